@@ -51,7 +51,9 @@ static void log_softmax_row(const float* z, int64_t A, double* lp) {
  *  - ratio R_t of Section 4.1 (R3 = pi_theta / max(pi_target, pi_worker / rho), Section 3.1)
  *    and the epsilon-clipped surrogate of Appendix E,
  *  - whether the gradient passes the clip (it does unless R lies strictly beyond the
- *    bound on the side where the clipped branch is the smaller one).
+ *    bound on the side where the clipped branch is the smaller one),
+ *  - adv_cond: sum of the absolute values of the terms that make up A_t (a conditioning
+ *    figure for the tests, no part of the loss).
  *
  * gamma_t = discounts[t] is the per-step discount, 0 where the episode ended at t.
  */
@@ -60,8 +62,8 @@ static void trajectory_terms(const double* lth, const double* ltg, const float* 
                              double bootstrap, double rho_bar, double c_bar, double clip_eps,
                              const oracle_coef* cf, int64_t T, const int8_t* flip,
                              double* adv, double* vtarget, double* ratio, double* surr,
-                             double* pass, double* rho_trunc) {
-    double next_adv = 0.0;
+                             double* pass, double* rho_trunc, double* adv_cond) {
+    double next_adv = 0.0, next_cond = 0.0;
     for (int64_t t = T - 1; t >= 0; --t) {
         double lw = (double)worker_logp[t];
         double x = (cf->is_source == 1 ? lth[t] : ltg[t]) - lw;
@@ -76,6 +78,11 @@ static void trajectory_terms(const double* lth, const double* ltg, const float* 
         adv[t] = a;
         vtarget[t] = v + a;
         rho_trunc[t] = (w > rho_bar) ? 1.0 : 0.0;
+        /* the same recursion on absolute values: the sum of |terms| of A_t, i.e. how much
+         * cancellation A_t hides.  Not part of the loss; tests scale their tolerance by it. */
+        next_cond = rho * (fabs((double)rewards[t]) + fabs(g * v_next) + fabs(v)) +
+                    fabs(cf->lambda * g * c) * next_cond;
+        adv_cond[t] = next_cond;
         next_adv = a;
     }
     for (int64_t t = 0; t < T; ++t) {
@@ -122,15 +129,16 @@ int oracle_impact_loss_categorical(
     double rho_bar, double c_bar, double clip_eps, const oracle_coef* cf,
     int64_t B, int64_t T, int64_t A, const int8_t* flip,
     double* loss_terms, double* dlogits, double* dvalues,
-    double* vtarget_out, double* advantage_out, double* ratio_out) {
+    double* vtarget_out, double* advantage_out, double* ratio_out, double* adv_cond_out) {
     if (B <= 0 || T <= 0 || A <= 0 || !cf) return -1;
     const double M = (double)B * (double)T;
     double* lp_th = (double*)malloc(sizeof(double) * (size_t)(T * A));
     double* lp_tg = (double*)malloc(sizeof(double) * (size_t)(T * A));
-    double* buf = (double*)malloc(sizeof(double) * (size_t)(T * 8));
+    double* buf = (double*)malloc(sizeof(double) * (size_t)(T * 9));
     if (!lp_th || !lp_tg || !buf) { free(lp_th); free(lp_tg); free(buf); return -1; }
     double *lth = buf, *ltg = buf + T, *adv = buf + 2 * T, *vt = buf + 3 * T,
-           *ratio = buf + 4 * T, *surr = buf + 5 * T, *pass = buf + 6 * T, *rtr = buf + 7 * T;
+           *ratio = buf + 4 * T, *surr = buf + 5 * T, *pass = buf + 6 * T, *rtr = buf + 7 * T,
+           *cond = buf + 8 * T;
     double s_surr = 0, s_val = 0, s_ent = 0, s_kl = 0, s_clip = 0, s_trunc = 0, s_ratio = 0;
 
     for (int64_t b = 0; b < B; ++b) {
@@ -147,7 +155,7 @@ int oracle_impact_loss_categorical(
         }
         trajectory_terms(lth, ltg, worker_logp + b * T, rewards + b * T, discounts + b * T,
                          values + b * T, (double)bootstrap_values[b], rho_bar, c_bar, clip_eps,
-                         cf, T, flip ? flip + b * T : NULL, adv, vt, ratio, surr, pass, rtr);
+                         cf, T, flip ? flip + b * T : NULL, adv, vt, ratio, surr, pass, rtr, cond);
         for (int64_t t = 0; t < T; ++t) {
             const double* lpl = lp_th + t * A;
             const double* lpt = lp_tg + t * A;
@@ -179,6 +187,7 @@ int oracle_impact_loss_categorical(
             if (vtarget_out) vtarget_out[b * T + t] = vt[t];
             if (advantage_out) advantage_out[b * T + t] = adv[t];
             if (ratio_out) ratio_out[b * T + t] = ratio[t];
+            if (adv_cond_out) adv_cond_out[b * T + t] = cond[t];
         }
     }
     if (loss_terms) {
@@ -212,14 +221,15 @@ int oracle_impact_loss_gaussian(
     const float* bootstrap_values, double rho_bar, double c_bar, double clip_eps,
     const oracle_coef* cf, int64_t B, int64_t T, int64_t D, const int8_t* flip,
     double* loss_terms, double* dmean, double* dlogstd, double* dvalues,
-    double* vtarget_out, double* advantage_out, double* ratio_out) {
+    double* vtarget_out, double* advantage_out, double* ratio_out, double* adv_cond_out) {
     if (B <= 0 || T <= 0 || D <= 0 || !cf) return -1;
     const double M = (double)B * (double)T;
     const double half_log_2pi = 0.5 * log(2.0 * 3.14159265358979323846);
-    double* buf = (double*)malloc(sizeof(double) * (size_t)(T * 8));
+    double* buf = (double*)malloc(sizeof(double) * (size_t)(T * 9));
     if (!buf) return -1;
     double *lth = buf, *ltg = buf + T, *adv = buf + 2 * T, *vt = buf + 3 * T,
-           *ratio = buf + 4 * T, *surr = buf + 5 * T, *pass = buf + 6 * T, *rtr = buf + 7 * T;
+           *ratio = buf + 4 * T, *surr = buf + 5 * T, *pass = buf + 6 * T, *rtr = buf + 7 * T,
+           *cond = buf + 8 * T;
     double s_surr = 0, s_val = 0, s_ent = 0, s_kl = 0, s_clip = 0, s_trunc = 0, s_ratio = 0;
 
     for (int64_t b = 0; b < B; ++b) {
@@ -238,7 +248,7 @@ int oracle_impact_loss_gaussian(
         }
         trajectory_terms(lth, ltg, worker_logp + b * T, rewards + b * T, discounts + b * T,
                          values + b * T, (double)bootstrap_values[b], rho_bar, c_bar, clip_eps,
-                         cf, T, flip ? flip + b * T : NULL, adv, vt, ratio, surr, pass, rtr);
+                         cf, T, flip ? flip + b * T : NULL, adv, vt, ratio, surr, pass, rtr, cond);
         for (int64_t t = 0; t < T; ++t) {
             int64_t o = (b * T + t) * D;
             double H = 0.0, KL = 0.0;
@@ -276,6 +286,7 @@ int oracle_impact_loss_gaussian(
             if (vtarget_out) vtarget_out[b * T + t] = vt[t];
             if (advantage_out) advantage_out[b * T + t] = adv[t];
             if (ratio_out) ratio_out[b * T + t] = ratio[t];
+            if (adv_cond_out) adv_cond_out[b * T + t] = cond[t];
         }
     }
     if (loss_terms) {

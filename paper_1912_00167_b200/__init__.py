@@ -1,0 +1,13 @@
+"""IMPACT learner hot path for B200: fused loss + gradient kernels and the circular buffer.
+
+The package is a thin binding over `libimpact.so` (built from `csrc/` for sm_100a); the
+library is loaded on first use and its absence is an error.
+"""
+from .binding import (  # noqa: F401
+    Coefficients, ImpactBuffer, ImpactError, PreparedCall, TERM_NAMES,
+    impact_gather_rows, impact_loss_fwd_bwd, impact_loss_fwd_bwd_gaussian,
+    impact_loss_workspace_bytes, impact_loss_workspace_init, impact_status_string,
+    impact_version, load_library, new_workspace, prepare_loss_fwd_bwd,
+    prepare_loss_fwd_bwd_gaussian,
+)
+from . import binding  # noqa: F401

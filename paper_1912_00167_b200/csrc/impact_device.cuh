@@ -1,0 +1,329 @@
+// Device building blocks of the fused IMPACT loss kernels (sm_100a).
+//
+// Work decomposition shared by the categorical and the Gaussian kernel:
+//   * one thread per time step ("row"); a block of NT threads owns a tile of up to NT
+//     consecutive rows of the row-major [B*T, width] tensors, which is one contiguous slab
+//     of global memory;
+//   * short trajectories (T <= NT) are packed, floor(NT/T) whole trajectories per tile;
+//     long ones (T > NT) are swept tile by tile from their END backwards, because the
+//     advantage recursion runs backward in time -- one scalar carry links the tiles, so
+//     every byte is still read once;
+//   * slabs are staged into shared memory with 16-byte streaming loads and re-laid out
+//     with an odd row stride, so that thread-per-row reads are bank-conflict free;
+//   * gradients overwrite the staged rows in place and leave with 16-byte streaming stores.
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace impact {
+namespace dev {
+
+constexpr int kNumSums = 7;  // surrogate, value, entropy, kl, clipped, rho-truncated, ratio
+
+// ---- 16-byte vectors of storage elements ---------------------------------------------
+template <typename T> struct Pack;
+template <> struct Pack<float> {
+    static constexpr int kElems = 4;
+    static __device__ __forceinline__ void unpack(const uint4& v, float (&f)[4]) {
+        f[0] = __uint_as_float(v.x); f[1] = __uint_as_float(v.y);
+        f[2] = __uint_as_float(v.z); f[3] = __uint_as_float(v.w);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[4]) {
+        return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]),
+                          __float_as_uint(f[2]), __float_as_uint(f[3]));
+    }
+    static __device__ __forceinline__ float to_float(float x) { return x; }
+    static __device__ __forceinline__ float from_float(float x) { return x; }
+};
+template <> struct Pack<__nv_bfloat16> {
+    static constexpr int kElems = 8;
+    static __device__ __forceinline__ void unpack(const uint4& v, float (&f)[8]) {
+        // a bf16 is the upper half of an fp32: widening is a shift, exact
+        f[0] = __uint_as_float(v.x << 16); f[1] = __uint_as_float(v.x & 0xFFFF0000u);
+        f[2] = __uint_as_float(v.y << 16); f[3] = __uint_as_float(v.y & 0xFFFF0000u);
+        f[4] = __uint_as_float(v.z << 16); f[5] = __uint_as_float(v.z & 0xFFFF0000u);
+        f[6] = __uint_as_float(v.w << 16); f[7] = __uint_as_float(v.w & 0xFFFF0000u);
+    }
+    static __device__ __forceinline__ uint32_t two(float lo, float hi) {
+        __nv_bfloat162 h = __floats2bfloat162_rn(lo, hi);  // round to nearest even
+        return *reinterpret_cast<uint32_t*>(&h);
+    }
+    static __device__ __forceinline__ uint4 pack(const float (&f)[8]) {
+        return make_uint4(two(f[0], f[1]), two(f[2], f[3]), two(f[4], f[5]), two(f[6], f[7]));
+    }
+    static __device__ __forceinline__ float to_float(__nv_bfloat16 x) { return __bfloat162float(x); }
+    static __device__ __forceinline__ __nv_bfloat16 from_float(float x) { return __float2bfloat16_rn(x); }
+};
+
+__device__ __forceinline__ uint4 ld_stream16(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.cs.v4.u32 {%0,%1,%2,%3}, [%4];"
+                 : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+__device__ __forceinline__ void st_stream16(uint4* p, const uint4& v) {
+    asm volatile("st.global.cs.v4.u32 [%0], {%1,%2,%3,%4};"
+                 :: "l"(p), "r"(v.x), "r"(v.y), "r"(v.z), "r"(v.w) : "memory");
+}
+
+// Walks (row, col) positions of a dense [rows, W] slab in steps of a fixed element count.
+struct RowCol {
+    int r, c;
+    __device__ __forceinline__ void init(int e, int W) { r = e / W; c = e - r * W; }
+    __device__ __forceinline__ void advance(int dq, int dr, int W) {
+        r += dq; c += dr;
+        if (c >= W) { c -= W; ++r; }
+    }
+};
+
+// Stage `nelem` consecutive elements of `src`, starting at element `base`, into shared
+// rows of stride `Ws` floats (element e of the slab lands at [e / W][e % W]).
+template <typename ST, int NT>
+__device__ __forceinline__ void stage_slab(float* __restrict__ dst, const ST* __restrict__ src,
+                                           long long base, int nelem, int W, int Ws) {
+    constexpr int VE = Pack<ST>::kElems;
+    const int tid = threadIdx.x;
+    int done = 0;
+    if ((base % VE) == 0) {
+        const int nvec = nelem / VE;
+        const uint4* s4 = reinterpret_cast<const uint4*>(src + base);
+        const int dq = (NT * VE) / W, dr = (NT * VE) % W;
+        RowCol rc; rc.init(tid * VE, W);
+        int v = tid;
+        constexpr int U = 4;
+        for (; v + (U - 1) * NT < nvec; v += U * NT) {
+            uint4 x[U];
+#pragma unroll
+            for (int u = 0; u < U; ++u) x[u] = ld_stream16(s4 + v + u * NT);
+#pragma unroll
+            for (int u = 0; u < U; ++u) {
+                float f[VE];
+                Pack<ST>::unpack(x[u], f);
+                int rr = rc.r, cc = rc.c;
+#pragma unroll
+                for (int j = 0; j < VE; ++j) {
+                    dst[rr * Ws + cc] = f[j];
+                    if (++cc == W) { cc = 0; ++rr; }
+                }
+                rc.advance(dq, dr, W);
+            }
+        }
+        for (; v < nvec; v += NT) {
+            uint4 x = ld_stream16(s4 + v);
+            float f[VE];
+            Pack<ST>::unpack(x, f);
+            int rr = rc.r, cc = rc.c;
+#pragma unroll
+            for (int j = 0; j < VE; ++j) {
+                dst[rr * Ws + cc] = f[j];
+                if (++cc == W) { cc = 0; ++rr; }
+            }
+            rc.advance(dq, dr, W);
+        }
+        done = nvec * VE;
+    }
+    if (done + tid < nelem) {  // unaligned slab, or the last few elements of an aligned one
+        const int dq = NT / W, dr = NT % W;
+        RowCol rc; rc.init(done + tid, W);
+        for (int e = done + tid; e < nelem; e += NT) {
+            dst[rc.r * Ws + rc.c] = Pack<ST>::to_float(src[base + e]);
+            rc.advance(dq, dr, W);
+        }
+    }
+}
+
+// The reverse of stage_slab: write the shared rows back to a dense global slab.
+template <typename ST, int NT>
+__device__ __forceinline__ void unstage_slab(ST* __restrict__ dst, const float* __restrict__ src,
+                                             long long base, int nelem, int W, int Ws) {
+    constexpr int VE = Pack<ST>::kElems;
+    const int tid = threadIdx.x;
+    int done = 0;
+    if ((base % VE) == 0) {
+        const int nvec = nelem / VE;
+        uint4* d4 = reinterpret_cast<uint4*>(dst + base);
+        const int dq = (NT * VE) / W, dr = (NT * VE) % W;
+        RowCol rc; rc.init(tid * VE, W);
+        for (int v = tid; v < nvec; v += NT) {
+            float f[VE];
+            int rr = rc.r, cc = rc.c;
+#pragma unroll
+            for (int j = 0; j < VE; ++j) {
+                f[j] = src[rr * Ws + cc];
+                if (++cc == W) { cc = 0; ++rr; }
+            }
+            st_stream16(d4 + v, Pack<ST>::pack(f));
+            rc.advance(dq, dr, W);
+        }
+        done = nvec * VE;
+    }
+    if (done + tid < nelem) {
+        const int dq = NT / W, dr = NT % W;
+        RowCol rc; rc.init(done + tid, W);
+        for (int e = done + tid; e < nelem; e += NT) {
+            dst[base + e] = Pack<ST>::from_float(src[rc.r * Ws + rc.c]);
+            rc.advance(dq, dr, W);
+        }
+    }
+}
+
+// ---- backward recursion as a suffix scan of affine maps ----------------------------------
+// Each thread i holds the map f_i(x) = a*x + b of its time step
+// (A_i = delta_i + (lambda gamma_i c_i) A_{i+1}).  Returns A_i = f_i(f_{i+1}(... f_{NT-1}(carry))).
+// Affine maps compose associatively, so the recursion is a scan: shuffles inside a warp,
+// one shared-memory hop across warps.  Contains one __syncthreads().
+template <int NT>
+__device__ __forceinline__ float suffix_affine_scan(float a, float b, float carry, float2* warp_agg) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float a2 = __shfl_down_sync(0xffffffffu, a, off);
+        const float b2 = __shfl_down_sync(0xffffffffu, b, off);
+        if (lane + off < 32) {
+            b = fmaf(a, b2, b);
+            a = a * a2;
+        }
+    }
+    if (lane == 0) warp_agg[warp] = make_float2(a, b);
+    __syncthreads();
+    float x = carry;
+#pragma unroll 1
+    for (int w = NT / 32 - 1; w > warp; --w) {
+        const float2 g = warp_agg[w];
+        x = fmaf(g.x, x, g.y);
+    }
+    return fmaf(a, x, b);
+}
+
+// Scalars of the loss that the kernels need; filled on the host.
+struct LossScalars {
+    float rho_bar, c_bar, clip_lo, clip_hi;
+    float vf_coef, ent_coef, kl_coef, lambda_, log_rho_tw;
+    float inv_M;
+    int is_source, ratio_mode;
+};
+
+// Per-step quantities once the three log-probabilities are known.
+struct StepIn {
+    float l_theta, l_target, l_worker;
+    float reward, discount, value, value_next;
+    bool last_step;  // t == T-1: the trace stops, V_{t+1} is the bootstrap value
+};
+
+// Truncated importance weights and the affine map of the advantage recursion
+// (Section 2.2; Section 3.1).  Returns whether exp(x) exceeded rho_bar.
+__device__ __forceinline__ bool recursion_map(const StepIn& s, const LossScalars& k, float& a, float& b) {
+    const float x = (k.is_source ? s.l_theta : s.l_target) - s.l_worker;
+    const float w = expf(x);
+    const float rho = fminf(k.rho_bar, w);
+    const float c = fminf(k.c_bar, w);
+    b = rho * (s.reward + s.discount * s.value_next - s.value);
+    a = s.last_step ? 0.0f : k.lambda_ * s.discount * c;
+    return w > k.rho_bar;
+}
+
+// Ratio of Section 4.1 and the eps-clipped surrogate of Appendix E.  Returns the weight
+// adv * R of the policy-gradient term (0 where the clip removes it).
+__device__ __forceinline__ float surrogate(const StepIn& s, const LossScalars& k, float adv,
+                                           float& surr, float& ratio, bool& clipped) {
+    float d;
+    if (k.ratio_mode == 1) d = s.l_target;
+    else if (k.ratio_mode == 2) d = s.l_worker;
+    else d = fmaxf(s.l_target, s.l_worker - k.log_rho_tw);
+    const float R = expf(s.l_theta - d);
+    const float Rc = fminf(fmaxf(R, k.clip_lo), k.clip_hi);
+    surr = fminf(R * adv, Rc * adv);
+    clipped = (adv > 0.0f && R > k.clip_hi) || (adv < 0.0f && R < k.clip_lo);
+    ratio = R;
+    return clipped ? 0.0f : adv * R;
+}
+
+// Sum the kNumSums per-thread values over the block (fixed order) and add them to `acc`,
+// which only thread 0 keeps.  `red` is [NT/32][8] shared floats.  The caller must place a
+// __syncthreads() between the write phase and the read phase: call stage 1, sync, stage 2.
+template <int NT>
+__device__ __forceinline__ void block_sums_stage1(float (&v)[kNumSums], float (*red)[8]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int j = 0; j < kNumSums; ++j) {
+        float x = v[j];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+        if (lane == 0) red[warp][j] = x;
+    }
+}
+template <int NT>
+__device__ __forceinline__ void block_sums_stage2(float (&acc)[kNumSums], float (*red)[8]) {
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int j = 0; j < kNumSums; ++j) {
+            float x = 0.0f;
+            for (int w = 0; w < NT / 32; ++w) x += red[w][j];
+            acc[j] += x;
+        }
+    }
+}
+
+// Last step of every loss kernel: publish this block's sums, and let the block that
+// finishes last add all blocks' sums in index order (fp64) and write the eight loss terms.
+// `counter` must be 0 on entry to the kernel and is 0 again on exit.
+template <int NT>
+__device__ __forceinline__ void finish_loss_terms(const float (&acc)[kNumSums], float* partials,
+                                                  unsigned int* counter, float* loss_terms,
+                                                  const LossScalars& k, double M) {
+    __shared__ bool is_last;
+    __shared__ double dred[NT / 32][kNumSums];
+    if (threadIdx.x == 0) {
+#pragma unroll
+        for (int j = 0; j < kNumSums; ++j) partials[(size_t)blockIdx.x * 8 + j] = acc[j];
+        __threadfence();
+        const unsigned int ticket = atomicAdd(counter, 1u);
+        is_last = (ticket == gridDim.x - 1);
+    }
+    __syncthreads();
+    if (!is_last) return;
+    __threadfence();
+    double s[kNumSums];
+#pragma unroll
+    for (int j = 0; j < kNumSums; ++j) s[j] = 0.0;
+    for (unsigned int blk = threadIdx.x; blk < gridDim.x; blk += NT) {
+        const float4 p0 = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)blk * 8));
+        const float4 p1 = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)blk * 8 + 4));
+        s[0] += p0.x; s[1] += p0.y; s[2] += p0.z; s[3] += p0.w;
+        s[4] += p1.x; s[5] += p1.y; s[6] += p1.z;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int j = 0; j < kNumSums; ++j) {
+        double x = s[j];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+        if (lane == 0) dred[warp][j] = x;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        double t[kNumSums];
+#pragma unroll
+        for (int j = 0; j < kNumSums; ++j) {
+            double x = 0.0;
+            for (int w = 0; w < NT / 32; ++w) x += dred[w][j];
+            t[j] = x / M;
+        }
+        const double l_pi = -t[0], l_v = t[1], ent = t[2], kl = t[3];
+        loss_terms[0] = (float)(l_pi + (double)k.vf_coef * l_v - (double)k.ent_coef * ent +
+                                (double)k.kl_coef * kl);
+        loss_terms[1] = (float)l_pi;
+        loss_terms[2] = (float)l_v;
+        loss_terms[3] = (float)ent;
+        loss_terms[4] = (float)kl;
+        loss_terms[5] = (float)t[4];
+        loss_terms[6] = (float)t[5];
+        loss_terms[7] = (float)t[6];
+        *counter = 0u;
+    }
+}
+
+}  // namespace dev
+}  // namespace impact

@@ -1,0 +1,610 @@
+// Fused IMPACT loss + gradient kernels and their host entry points.
+//
+// One launch per call does every step of the learner's "compute policy and value network
+// gradients" (Algorithm 1): log-probabilities under learner and target, truncated
+// importance weights, the backward V-trace GAE-lambda recursion (Section 3.1), the
+// target-worker-clipped, eps-clipped surrogate (Section 3.1, Appendix E), value / entropy /
+// KL terms, the gradients, and the batch means.  Each input byte is read from HBM once and
+// each output byte written once; nothing on this path is a matrix product, so no tensor
+// cores are involved -- the kernel is bound by HBM bandwidth.
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <math.h>
+
+#include "impact.h"
+#include "impact_device.cuh"
+#include "impact_internal.h"
+
+namespace impact {
+namespace {
+
+using dev::LossScalars;
+
+struct TileGeometry {
+    long long B, T;
+    long long nchunks;  // units of block-level work
+    int G;              // whole trajectories per chunk (T <= NT), else 1
+    int ntiles;         // tiles per trajectory (T > NT), else 1
+};
+
+struct CatParams {
+    const void* learner_logits;
+    const void* target_logits;
+    const float* worker_logp;
+    const int32_t* actions;
+    const float* rewards;
+    const float* discounts;
+    const float* values;
+    const float* bootstrap;
+    float* loss_terms;
+    void* dlogits;
+    float* dvalues;
+    float* vtarget;
+    float* advantage;
+    float* partials;
+    unsigned int* counter;
+    TileGeometry geo;
+    LossScalars k;
+    int A, As;
+};
+
+struct GaussParams {
+    const float* learner_mean;
+    const float* learner_logstd;
+    const float* target_mean;
+    const float* target_logstd;
+    const float* actions;
+    const float* worker_logp;
+    const float* rewards;
+    const float* discounts;
+    const float* values;
+    const float* bootstrap;
+    float* loss_terms;
+    float* dmean;
+    float* dlogstd;
+    float* dvalues;
+    float* vtarget;
+    float* advantage;
+    float* partials;
+    unsigned int* counter;
+    TileGeometry geo;
+    LossScalars k;
+    int D, Ds;
+};
+
+// Where a tile sits: its first global row, how many rows, and each thread's (b, t).
+struct TileRows {
+    long long row0;
+    int nrows;
+};
+
+template <int NT>
+__device__ __forceinline__ TileRows tile_rows(const TileGeometry& g, long long chunk, int tile) {
+    TileRows r;
+    if (g.ntiles > 1) {
+        const long long t0 = (long long)tile * NT;
+        const long long left = g.T - t0;
+        r.nrows = (int)(left < NT ? left : NT);
+        r.row0 = chunk * g.T + t0;
+    } else {
+        const long long traj0 = chunk * g.G;
+        long long ntraj = g.B - traj0;
+        if (ntraj > g.G) ntraj = g.G;
+        r.nrows = (int)(ntraj * g.T);
+        r.row0 = traj0 * g.T;
+    }
+    return r;
+}
+
+// ------------------------------------------------------------------------------------------
+// Categorical policy
+// ------------------------------------------------------------------------------------------
+template <typename LT, typename GT, int NT>
+__global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatParams p) {
+    extern __shared__ __align__(16) float smem[];
+    float* const sl = smem;                          // learner rows, then gradient rows
+    float* const st = smem + (size_t)NT * p.As;      // target rows
+    __shared__ float2 warp_agg[NT / 32];
+    __shared__ float red[NT / 32][8];
+    __shared__ float carry_s;
+
+    const int tid = threadIdx.x;
+    const int A = p.A, As = p.As;
+    const LossScalars k = p.k;
+    const TileGeometry g = p.geo;
+    const LT* const zl = static_cast<const LT*>(p.learner_logits);
+    const LT* const zt = static_cast<const LT*>(p.target_logits);
+    GT* const dz = static_cast<GT*>(p.dlogits);
+    const bool want_kl = (k.kl_coef != 0.0f);
+
+    float acc[dev::kNumSums];
+#pragma unroll
+    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = 0.0f;
+
+    for (long long chunk = blockIdx.x; chunk < g.nchunks; chunk += gridDim.x) {
+        float carry = 0.0f;
+        for (int tile = g.ntiles - 1; tile >= 0; --tile) {
+            const TileRows tr = tile_rows<NT>(g, chunk, tile);
+            const long long base = tr.row0 * A;
+            const int nelem = tr.nrows * A;
+            __syncthreads();  // the previous tile's rows, sums and carry have been consumed
+            dev::stage_slab<LT, NT>(sl, zl, base, nelem, A, As);
+            dev::stage_slab<LT, NT>(st, zt, base, nelem, A, As);
+            __syncthreads();
+
+            const bool active = tid < tr.nrows;
+            const long long row = tr.row0 + tid;
+            float* const rl = sl + tid * As;
+            const float* const rt = st + tid * As;
+            dev::StepIn s;
+            float fa = 1.0f, fb = 0.0f;  // identity map for idle threads
+            float lse_l = 0.0f, lse_t = 0.0f, ent = 0.0f, kl = 0.0f;
+            int a = 0;
+            bool truncated = false;
+            if (active) {
+                long long b, t;
+                if (g.ntiles > 1) { b = chunk; t = (long long)tile * NT + tid; }
+                else { const int q = tid / (int)g.T; b = chunk * g.G + q; t = tid - q * (int)g.T; }
+                a = p.actions[row];
+                a = a < 0 ? 0 : (a >= A ? A - 1 : a);
+                // log-softmax of the target row
+                float m = rt[0];
+                for (int j = 1; j < A; ++j) m = fmaxf(m, rt[j]);
+                float sum = 0.0f;
+                for (int j = 0; j < A; ++j) sum += expf(rt[j] - m);
+                lse_t = m + logf(sum);
+                s.l_target = rt[a] - lse_t;
+                // log-softmax and entropy of the learner row: H = ln S - sum e_j (z_j - m) / S
+                m = rl[0];
+                for (int j = 1; j < A; ++j) m = fmaxf(m, rl[j]);
+                sum = 0.0f;
+                float sez = 0.0f;
+                for (int j = 0; j < A; ++j) {
+                    const float d = rl[j] - m;
+                    const float e = expf(d);
+                    sum += e;
+                    sez = fmaf(e, d, sez);
+                }
+                const float ls = logf(sum);
+                lse_l = m + ls;
+                ent = ls - sez / sum;
+                s.l_theta = rl[a] - lse_l;
+                if (want_kl) {
+                    for (int j = 0; j < A; ++j) {
+                        const float lpt = rt[j] - lse_t;
+                        kl = fmaf(expf(lpt), lpt - (rl[j] - lse_l), kl);
+                    }
+                }
+                s.l_worker = p.worker_logp[row];
+                s.reward = p.rewards[row];
+                s.discount = p.discounts[row];
+                s.value = p.values[row];
+                s.last_step = (t == g.T - 1);
+                s.value_next = s.last_step ? p.bootstrap[b] : p.values[row + 1];
+                truncated = dev::recursion_map(s, k, fa, fb);
+            }
+            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
+            if (tid == 0) carry_s = adv;
+
+            float sums[dev::kNumSums];
+#pragma unroll
+            for (int j = 0; j < dev::kNumSums; ++j) sums[j] = 0.0f;
+            if (active) {
+                float surr, ratio;
+                bool clipped;
+                const float wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
+                // d total / d logit_j = [ wpg (pi_j - 1[j=a]) + ent_coef pi_j (lp_j + H)
+                //                         + kl_coef (pi_j - pi_target_j) ] / M
+                const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = k.kl_coef * k.inv_M;
+                for (int j = 0; j < A; ++j) {
+                    const float lp = rl[j] - lse_l;
+                    const float pi = expf(lp);
+                    float gj = pi * fmaf(ce, lp + ent, w1);
+                    if (want_kl) gj = fmaf(ck, pi - expf(rt[j] - lse_t), gj);
+                    rl[j] = gj;
+                }
+                rl[a] -= w1;
+                p.dvalues[row] = -k.vf_coef * k.inv_M * adv;  // V - Vhat = -A
+                if (p.vtarget) p.vtarget[row] = s.value + adv;
+                if (p.advantage) p.advantage[row] = adv;
+                sums[0] = surr;
+                sums[1] = 0.5f * adv * adv;
+                sums[2] = ent;
+                sums[3] = kl;
+                sums[4] = clipped ? 1.0f : 0.0f;
+                sums[5] = truncated ? 1.0f : 0.0f;
+                sums[6] = ratio;
+            }
+            dev::block_sums_stage1<NT>(sums, red);
+            __syncthreads();
+            carry = carry_s;
+            dev::unstage_slab<GT, NT>(dz, sl, base, nelem, A, As);
+            dev::block_sums_stage2<NT>(acc, red);
+        }
+    }
+    dev::finish_loss_terms<NT>(acc, p.partials, p.counter, p.loss_terms, k,
+                               (double)g.B * (double)g.T);
+}
+
+// ------------------------------------------------------------------------------------------
+// Diagonal-Gaussian policy
+// ------------------------------------------------------------------------------------------
+template <int NT>
+__global__ void __launch_bounds__(NT) impact_loss_gaussian_kernel(const GaussParams p) {
+    extern __shared__ __align__(16) float smem[];
+    const int D = p.D, Ds = p.Ds;
+    float* const s_mu = smem;                              // learner mean -> dmean
+    float* const s_ls = s_mu + (size_t)NT * Ds;            // learner logstd -> dlogstd
+    float* const s_mt = s_ls + (size_t)NT * Ds;            // target mean
+    float* const s_lt = s_mt + (size_t)NT * Ds;            // target logstd
+    float* const s_ac = s_lt + (size_t)NT * Ds;            // actions
+    __shared__ float2 warp_agg[NT / 32];
+    __shared__ float red[NT / 32][8];
+    __shared__ float carry_s;
+
+    const int tid = threadIdx.x;
+    const LossScalars k = p.k;
+    const TileGeometry g = p.geo;
+    const float half_log_2pi = 0.91893853320467274178f;
+
+    float acc[dev::kNumSums];
+#pragma unroll
+    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = 0.0f;
+
+    for (long long chunk = blockIdx.x; chunk < g.nchunks; chunk += gridDim.x) {
+        float carry = 0.0f;
+        for (int tile = g.ntiles - 1; tile >= 0; --tile) {
+            const TileRows tr = tile_rows<NT>(g, chunk, tile);
+            const long long base = tr.row0 * D;
+            const int nelem = tr.nrows * D;
+            __syncthreads();
+            dev::stage_slab<float, NT>(s_mu, p.learner_mean, base, nelem, D, Ds);
+            dev::stage_slab<float, NT>(s_ls, p.learner_logstd, base, nelem, D, Ds);
+            dev::stage_slab<float, NT>(s_mt, p.target_mean, base, nelem, D, Ds);
+            dev::stage_slab<float, NT>(s_lt, p.target_logstd, base, nelem, D, Ds);
+            dev::stage_slab<float, NT>(s_ac, p.actions, base, nelem, D, Ds);
+            __syncthreads();
+
+            const bool active = tid < tr.nrows;
+            const long long row = tr.row0 + tid;
+            float* const r_mu = s_mu + tid * Ds;
+            float* const r_ls = s_ls + tid * Ds;
+            const float* const r_mt = s_mt + tid * Ds;
+            const float* const r_lt = s_lt + tid * Ds;
+            const float* const r_ac = s_ac + tid * Ds;
+            dev::StepIn s;
+            float fa = 1.0f, fb = 0.0f;
+            float ent = 0.0f, kl = 0.0f;
+            bool truncated = false;
+            if (active) {
+                long long b, t;
+                if (g.ntiles > 1) { b = chunk; t = (long long)tile * NT + tid; }
+                else { const int q = tid / (int)g.T; b = chunk * g.G + q; t = tid - q * (int)g.T; }
+                // The log-probabilities are sums of D terms and reach magnitudes of tens; they
+                // enter exponentials, so their absolute error is the relative error of the
+                // ratios.  Accumulating them in fp64 (half-rate on this part, a few percent of
+                // the pipe here) keeps that error at the level of the fp32 terms themselves.
+                double lth = 0.0, ltg = 0.0;
+                for (int j = 0; j < D; ++j) {
+                    const float ls = r_ls[j], lt = r_lt[j], ac = r_ac[j];
+                    const float inv_s = expf(-ls), inv_st = expf(-lt);
+                    const float z1 = (ac - r_mu[j]) * inv_s;
+                    const float z2 = (ac - r_mt[j]) * inv_st;
+                    lth += (double)(fmaf(-0.5f * z1, z1, -ls) - half_log_2pi);
+                    ltg += (double)(fmaf(-0.5f * z2, z2, -lt) - half_log_2pi);
+                    ent += ls + (half_log_2pi + 0.5f);
+                    // KL(target || learner), per dimension
+                    const float dm = (r_mt[j] - r_mu[j]) * inv_s;
+                    const float sr = expf(lt - ls);  // sigma_target / sigma_learner
+                    kl += (ls - lt) + 0.5f * fmaf(sr, sr, dm * dm) - 0.5f;
+                }
+                // differences against the worker's log-probability are taken in fp64, then
+                // everything continues in fp32 relative to it
+                const float lw = p.worker_logp[row];
+                s.l_theta = (float)(lth - (double)lw);
+                s.l_target = (float)(ltg - (double)lw);
+                s.l_worker = 0.0f;
+                s.reward = p.rewards[row];
+                s.discount = p.discounts[row];
+                s.value = p.values[row];
+                s.last_step = (t == g.T - 1);
+                s.value_next = s.last_step ? p.bootstrap[b] : p.values[row + 1];
+                truncated = dev::recursion_map(s, k, fa, fb);
+            }
+            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
+            if (tid == 0) carry_s = adv;
+
+            float sums[dev::kNumSums];
+#pragma unroll
+            for (int j = 0; j < dev::kNumSums; ++j) sums[j] = 0.0f;
+            if (active) {
+                float surr, ratio;
+                bool clipped;
+                const float wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
+                const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = k.kl_coef * k.inv_M;
+                for (int j = 0; j < D; ++j) {
+                    const float ls = r_ls[j], lt = r_lt[j], mu = r_mu[j];
+                    const float inv_s = expf(-ls);
+                    const float z = (r_ac[j] - mu) * inv_s;       // (a - mu) / sigma
+                    const float dm = (mu - r_mt[j]) * inv_s;      // (mu - mu_target) / sigma
+                    const float sr = expf(lt - ls);
+                    // d log pi / d mu = z / sigma ; d KL / d mu = dm / sigma
+                    r_mu[j] = (ck * dm - w1 * z) * inv_s;
+                    // d log pi / d logstd = z^2 - 1 ; d H / d logstd = 1 ;
+                    // d KL / d logstd = 1 - (sigma_t^2 + (mu_t - mu)^2) / sigma^2
+                    r_ls[j] = -w1 * fmaf(z, z, -1.0f) - ce + ck * (1.0f - fmaf(sr, sr, dm * dm));
+                }
+                p.dvalues[row] = -k.vf_coef * k.inv_M * adv;
+                if (p.vtarget) p.vtarget[row] = s.value + adv;
+                if (p.advantage) p.advantage[row] = adv;
+                sums[0] = surr;
+                sums[1] = 0.5f * adv * adv;
+                sums[2] = ent;
+                sums[3] = kl;
+                sums[4] = clipped ? 1.0f : 0.0f;
+                sums[5] = truncated ? 1.0f : 0.0f;
+                sums[6] = ratio;
+            }
+            dev::block_sums_stage1<NT>(sums, red);
+            __syncthreads();
+            carry = carry_s;
+            dev::unstage_slab<float, NT>(p.dmean, s_mu, base, nelem, D, Ds);
+            dev::unstage_slab<float, NT>(p.dlogstd, s_ls, base, nelem, D, Ds);
+            dev::block_sums_stage2<NT>(acc, red);
+        }
+    }
+    dev::finish_loss_terms<NT>(acc, p.partials, p.counter, p.loss_terms, k,
+                               (double)g.B * (double)g.T);
+}
+
+// ------------------------------------------------------------------------------------------
+// Host side
+// ------------------------------------------------------------------------------------------
+constexpr int kMaxGridBlocks = 4096;  // upper bound on blocks of a loss launch (sizes the workspace)
+constexpr size_t kCounterBytes = 256; // counter lives in its own 256-byte line after the partials
+
+int pad_odd(int w) { return (w & 1) ? w : w + 1; }
+
+// Threads per block = rows per tile: as many as keep a tile's staged slabs within
+// `budget` bytes of shared memory, so that several blocks stay resident per SM.
+int pick_nt(int width_padded, int n_slabs, size_t budget) {
+    for (int nt : {128, 64}) {
+        if ((size_t)nt * width_padded * n_slabs * sizeof(float) <= budget) return nt;
+    }
+    return 32;
+}
+
+TileGeometry make_geometry(int64_t B, int64_t T, int nt) {
+    TileGeometry g;
+    g.B = B;
+    g.T = T;
+    if (T <= nt) {
+        g.G = (int)(nt / T);
+        g.ntiles = 1;
+        g.nchunks = (B + g.G - 1) / g.G;
+    } else {
+        g.G = 1;
+        g.ntiles = (int)((T + nt - 1) / nt);
+        g.nchunks = B;
+    }
+    return g;
+}
+
+bool bad_scalar(float x) { return !(x >= 0.0f); }  // negative or NaN
+
+int32_t fill_scalars(LossScalars& k, float rho_bar, float c_bar, float clip_eps,
+                     const impact_coefficients* coef, int64_t B, int64_t T) {
+    if (bad_scalar(rho_bar) || bad_scalar(c_bar) || bad_scalar(clip_eps)) return IMPACT_ERR_INVALID_ARG;
+    if (!(coef->rho_tw > 0.0f) || !isfinite(coef->vf_coef) || !isfinite(coef->ent_coef) ||
+        !isfinite(coef->kl_coef) || !isfinite(coef->lambda_) || coef->reserved != 0)
+        return IMPACT_ERR_INVALID_ARG;
+    if (coef->is_source != IMPACT_IS_TARGET_OVER_WORKER && coef->is_source != IMPACT_IS_LEARNER_OVER_WORKER)
+        return IMPACT_ERR_INVALID_ARG;
+    if (coef->ratio_mode < IMPACT_RATIO_R3 || coef->ratio_mode > IMPACT_RATIO_R2) return IMPACT_ERR_INVALID_ARG;
+    k.rho_bar = rho_bar;
+    k.c_bar = c_bar;
+    k.clip_lo = 1.0f - clip_eps;
+    k.clip_hi = 1.0f + clip_eps;
+    k.vf_coef = coef->vf_coef;
+    k.ent_coef = coef->ent_coef;
+    k.kl_coef = coef->kl_coef;
+    k.lambda_ = coef->lambda_;
+    k.log_rho_tw = (float)log((double)coef->rho_tw);
+    k.inv_M = (float)(1.0 / ((double)B * (double)T));
+    k.is_source = coef->is_source;
+    k.ratio_mode = coef->ratio_mode;
+    return IMPACT_OK;
+}
+
+// Blocks to launch: every chunk gets its own block while all of them can be resident at
+// once; beyond that, a resident-sized grid walks the chunks.
+template <typename Kernel>
+int32_t grid_for(Kernel kernel, int nt, size_t smem, long long nchunks, const DeviceInfo* di, int* grid) {
+    struct Key { const void* fn; size_t smem; int dev; int per_sm; };
+    static thread_local Key cache[16];
+    static thread_local int ncache = 0;
+    int per_sm = -1;
+    for (int i = 0; i < ncache; ++i)
+        if (cache[i].fn == (const void*)kernel && cache[i].smem == smem && cache[i].dev == di->device)
+            per_sm = cache[i].per_sm;
+    if (per_sm < 0) {
+        if (smem > 48 * 1024)
+            IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        IMPACT_CUDA_TRY(cudaOccupancyMaxActiveBlocksPerMultiprocessor(&per_sm, kernel, nt, smem));
+        if (per_sm < 1) return IMPACT_ERR_UNSUPPORTED;
+        if (ncache < 16) cache[ncache++] = Key{(const void*)kernel, smem, di->device, per_sm};
+    }
+    long long resident = (long long)per_sm * di->sm_count;
+    if (resident > kMaxGridBlocks) resident = kMaxGridBlocks;
+    *grid = (int)(nchunks < resident ? nchunks : resident);
+    return IMPACT_OK;
+}
+
+template <typename LT, typename GT, int NT>
+int32_t launch_categorical(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
+    auto kernel = impact_loss_categorical_kernel<LT, GT, NT>;
+    const size_t smem = (size_t)2 * NT * p.As * sizeof(float);
+    int grid = 0;
+    int32_t st = grid_for(kernel, NT, smem, p.geo.nchunks, di, &grid);
+    if (st != IMPACT_OK) return st;
+    kernel<<<grid, NT, smem, stream>>>(p);
+    IMPACT_CUDA_TRY(cudaGetLastError());
+    return IMPACT_OK;
+}
+
+template <typename LT, typename GT>
+int32_t dispatch_nt(const CatParams& p, int nt, const DeviceInfo* di, cudaStream_t stream) {
+    switch (nt) {
+        case 128: return launch_categorical<LT, GT, 128>(p, di, stream);
+        case 64: return launch_categorical<LT, GT, 64>(p, di, stream);
+        default: return launch_categorical<LT, GT, 32>(p, di, stream);
+    }
+}
+
+template <int NT>
+int32_t launch_gaussian(const GaussParams& p, const DeviceInfo* di, cudaStream_t stream) {
+    auto kernel = impact_loss_gaussian_kernel<NT>;
+    const size_t smem = (size_t)5 * NT * p.Ds * sizeof(float);
+    int grid = 0;
+    int32_t st = grid_for(kernel, NT, smem, p.geo.nchunks, di, &grid);
+    if (st != IMPACT_OK) return st;
+    kernel<<<grid, NT, smem, stream>>>(p);
+    IMPACT_CUDA_TRY(cudaGetLastError());
+    return IMPACT_OK;
+}
+
+}  // namespace
+}  // namespace impact
+
+using namespace impact;
+
+extern "C" size_t impact_loss_workspace_bytes(int64_t B, int64_t T) {
+    if (B <= 0 || T <= 0) return 0;
+    return (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes;
+}
+
+extern "C" int32_t impact_loss_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
+    if (!workspace || !aligned16(workspace) || workspace_bytes == 0) return IMPACT_ERR_INVALID_ARG;
+    IMPACT_CUDA_TRY(cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)));
+    return IMPACT_OK;
+}
+
+extern "C" int32_t impact_loss_fwd_bwd(
+    const void* learner_logits, const void* target_logits, const float* worker_logp,
+    const int32_t* actions, const float* rewards, const float* discounts, const float* values,
+    const float* bootstrap_values, float rho_bar, float c_bar, float clip_eps,
+    const impact_coefficients* coef, int64_t B, int64_t T, int32_t A, int32_t logits_dtype,
+    float* loss_terms, void* dlogits, float* dvalues, float* vtarget, float* advantage,
+    void* workspace, size_t workspace_bytes, void* stream) {
+    if (!learner_logits || !target_logits || !worker_logp || !actions || !rewards || !discounts ||
+        !values || !bootstrap_values || !coef || !loss_terms || !dlogits || !dvalues || !workspace)
+        return IMPACT_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || A <= 0) return IMPACT_ERR_INVALID_ARG;
+    const void* ptrs[] = {learner_logits, target_logits, worker_logp, actions, rewards, discounts,
+                          values, bootstrap_values, loss_terms, dlogits, dvalues, workspace};
+    for (const void* q : ptrs)
+        if (!aligned16(q)) return IMPACT_ERR_INVALID_ARG;
+    if ((vtarget && !aligned16(vtarget)) || (advantage && !aligned16(advantage))) return IMPACT_ERR_INVALID_ARG;
+    if (logits_dtype != IMPACT_DTYPE_F32 && logits_dtype != IMPACT_DTYPE_BF16) return IMPACT_ERR_INVALID_ARG;
+    if (coef->dlogits_dtype != IMPACT_DTYPE_F32 && coef->dlogits_dtype != IMPACT_DTYPE_BF16)
+        return IMPACT_ERR_INVALID_ARG;
+    if (A > 512) return IMPACT_ERR_UNSUPPORTED;
+    if ((double)B * (double)T * (double)A >= 1099511627776.0 || (double)B * (double)T >= 4.0e12)
+        return IMPACT_ERR_UNSUPPORTED;
+    if (workspace_bytes < impact_loss_workspace_bytes(B, T)) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
+
+    CatParams p;
+    int32_t st = fill_scalars(p.k, rho_bar, c_bar, clip_eps, coef, B, T);
+    if (st != IMPACT_OK) return st;
+    const DeviceInfo* di = current_device_info();
+    if (!di) return IMPACT_ERR_CUDA;
+
+    p.learner_logits = learner_logits;
+    p.target_logits = target_logits;
+    p.worker_logp = worker_logp;
+    p.actions = actions;
+    p.rewards = rewards;
+    p.discounts = discounts;
+    p.values = values;
+    p.bootstrap = bootstrap_values;
+    p.loss_terms = loss_terms;
+    p.dlogits = dlogits;
+    p.dvalues = dvalues;
+    p.vtarget = vtarget;
+    p.advantage = advantage;
+    p.partials = static_cast<float*>(workspace);
+    p.counter = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) +
+                                                (size_t)kMaxGridBlocks * 8 * sizeof(float));
+    p.A = A;
+    p.As = pad_odd(A);
+    const int nt = pick_nt(p.As, 2, 72 * 1024);
+    p.geo = make_geometry(B, T, nt);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const bool lb = logits_dtype == IMPACT_DTYPE_BF16, gb = coef->dlogits_dtype == IMPACT_DTYPE_BF16;
+    if (!lb && !gb) return dispatch_nt<float, float>(p, nt, di, s);
+    if (!lb && gb) return dispatch_nt<float, __nv_bfloat16>(p, nt, di, s);
+    if (lb && !gb) return dispatch_nt<__nv_bfloat16, float>(p, nt, di, s);
+    return dispatch_nt<__nv_bfloat16, __nv_bfloat16>(p, nt, di, s);
+}
+
+extern "C" int32_t impact_loss_fwd_bwd_gaussian(
+    const float* learner_mean, const float* learner_logstd, const float* target_mean,
+    const float* target_logstd, const float* worker_logp, const float* actions,
+    const float* rewards, const float* discounts, const float* values,
+    const float* bootstrap_values, float rho_bar, float c_bar, float clip_eps,
+    const impact_coefficients* coef, int64_t B, int64_t T, int32_t D,
+    float* loss_terms, float* dmean, float* dlogstd, float* dvalues, float* vtarget,
+    float* advantage, void* workspace, size_t workspace_bytes, void* stream) {
+    if (!learner_mean || !learner_logstd || !target_mean || !target_logstd || !worker_logp ||
+        !actions || !rewards || !discounts || !values || !bootstrap_values || !coef || !loss_terms ||
+        !dmean || !dlogstd || !dvalues || !workspace)
+        return IMPACT_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || D <= 0) return IMPACT_ERR_INVALID_ARG;
+    const void* ptrs[] = {learner_mean, learner_logstd, target_mean, target_logstd, worker_logp,
+                          actions, rewards, discounts, values, bootstrap_values, loss_terms,
+                          dmean, dlogstd, dvalues, workspace};
+    for (const void* q : ptrs)
+        if (!aligned16(q)) return IMPACT_ERR_INVALID_ARG;
+    if ((vtarget && !aligned16(vtarget)) || (advantage && !aligned16(advantage))) return IMPACT_ERR_INVALID_ARG;
+    if (coef->dlogits_dtype != IMPACT_DTYPE_F32) return IMPACT_ERR_INVALID_ARG;
+    if (D > 256) return IMPACT_ERR_UNSUPPORTED;
+    if ((double)B * (double)T * (double)D >= 1099511627776.0 || (double)B * (double)T >= 4.0e12)
+        return IMPACT_ERR_UNSUPPORTED;
+    if (workspace_bytes < impact_loss_workspace_bytes(B, T)) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
+
+    GaussParams p;
+    int32_t st = fill_scalars(p.k, rho_bar, c_bar, clip_eps, coef, B, T);
+    if (st != IMPACT_OK) return st;
+    const DeviceInfo* di = current_device_info();
+    if (!di) return IMPACT_ERR_CUDA;
+
+    p.learner_mean = learner_mean;
+    p.learner_logstd = learner_logstd;
+    p.target_mean = target_mean;
+    p.target_logstd = target_logstd;
+    p.actions = actions;
+    p.worker_logp = worker_logp;
+    p.rewards = rewards;
+    p.discounts = discounts;
+    p.values = values;
+    p.bootstrap = bootstrap_values;
+    p.loss_terms = loss_terms;
+    p.dmean = dmean;
+    p.dlogstd = dlogstd;
+    p.dvalues = dvalues;
+    p.vtarget = vtarget;
+    p.advantage = advantage;
+    p.partials = static_cast<float*>(workspace);
+    p.counter = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) +
+                                                (size_t)kMaxGridBlocks * 8 * sizeof(float));
+    p.D = D;
+    p.Ds = pad_odd(D);
+    const int nt = pick_nt(p.Ds, 5, 100 * 1024);
+    p.geo = make_geometry(B, T, nt);
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    switch (nt) {
+        case 128: return launch_gaussian<128>(p, di, s);
+        case 64: return launch_gaussian<64>(p, di, s);
+        default: return launch_gaussian<32>(p, di, s);
+    }
+}

@@ -1,0 +1,191 @@
+"""Helpers shared by the GPU parity tests: run both sides on the same seeded batch and compare.
+
+Tolerances (fp32 path): per-element outputs within 1e-5 relative or 1e-6 absolute, where
+the absolute part is taken on the natural scale of the output -- gradients carry a 1/M
+factor, so they are compared after multiplying by M; reduced scalars within 1e-4 relative.
+bf16-stored variants: 2e-2 relative (plus the same absolute floor).
+"""
+import dataclasses
+
+import numpy as np
+import torch
+
+import impact_inputs as ii
+
+RTOL_ELEM, ATOL_ELEM = 1e-5, 1e-6
+RTOL_SCALAR, ATOL_SCALAR = 1e-4, 1e-7
+RTOL_BF16, ATOL_BF16 = 2e-2, 2e-3
+COND_ADV = 4e-6  # ~64 fp32 unit roundoffs (2^-24) of the advantage's condition sum
+
+
+def f32_hyper(h: ii.LossHyper) -> ii.LossHyper:
+    """The hyper-parameters as the fp32 values the C ABI receives."""
+    r = lambda x: float(np.float32(x))
+    return dataclasses.replace(h, rho_bar=r(h.rho_bar), c_bar=r(h.c_bar), clip_eps=r(h.clip_eps),
+                               vf_coef=r(h.vf_coef), ent_coef=r(h.ent_coef), kl_coef=r(h.kl_coef),
+                               lam=r(h.lam), rho_tw=r(h.rho_tw))
+
+
+def to_coef(h: ii.LossHyper):
+    import paper_1912_00167_b200 as ip
+    return ip.Coefficients(rho_bar=h.rho_bar, c_bar=h.c_bar, clip_eps=h.clip_eps, vf_coef=h.vf_coef,
+                           ent_coef=h.ent_coef, kl_coef=h.kl_coef, lam=h.lam, rho_tw=h.rho_tw,
+                           is_source=h.is_source, ratio_mode=h.ratio_mode)
+
+
+def run_gpu_categorical(batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, extra=True):
+    import paper_1912_00167_b200 as ip
+    dev = "cuda"
+    t = {k: torch.from_numpy(np.ascontiguousarray(v)).to(dev) for k, v in batch.items()}
+    zl = t["learner_logits"].to(logits_dtype)
+    zt = t["target_logits"].to(logits_dtype)
+    B, T, A = zl.shape
+    out = dict(loss_terms=torch.full((8,), float("nan"), device=dev),
+               dlogits=torch.full((B, T, A), float("nan"), device=dev, dtype=dlogits_dtype),
+               dvalues=torch.full((B, T), float("nan"), device=dev))
+    if extra:
+        out["vtarget"] = torch.full((B, T), float("nan"), device=dev)
+        out["advantage"] = torch.full((B, T), float("nan"), device=dev)
+    ws = ip.new_workspace(B, T)
+    ip.impact_loss_fwd_bwd(zl, zt, t["worker_logp"], t["actions"], t["rewards"], t["discounts"], t["values"],
+                           t["bootstrap_values"], to_coef(h), workspace=ws, **out)
+    torch.cuda.synchronize()
+    return {k: v.float().cpu().numpy().astype(np.float64) for k, v in out.items()}
+
+
+def run_gpu_gaussian(batch, h, extra=True):
+    import paper_1912_00167_b200 as ip
+    dev = "cuda"
+    t = {k: torch.from_numpy(np.ascontiguousarray(v)).to(dev) for k, v in batch.items()}
+    B, T, D = t["learner_mean"].shape
+    out = dict(loss_terms=torch.full((8,), float("nan"), device=dev),
+               dmean=torch.full((B, T, D), float("nan"), device=dev),
+               dlogstd=torch.full((B, T, D), float("nan"), device=dev),
+               dvalues=torch.full((B, T), float("nan"), device=dev))
+    if extra:
+        out["vtarget"] = torch.full((B, T), float("nan"), device=dev)
+        out["advantage"] = torch.full((B, T), float("nan"), device=dev)
+    ws = ip.new_workspace(B, T)
+    ip.impact_loss_fwd_bwd_gaussian(t["learner_mean"], t["learner_logstd"], t["target_mean"], t["target_logstd"],
+                                    t["worker_logp"], t["actions"], t["rewards"], t["discounts"], t["values"],
+                                    t["bootstrap_values"], to_coef(h), workspace=ws, **out)
+    torch.cuda.synchronize()
+    return {k: v.cpu().numpy().astype(np.float64) for k, v in out.items()}
+
+
+def near_clip_bound(ref, h, rel=2e-5):
+    """Steps whose ratio sits on a clip bound to within rounding: either branch is valid."""
+    R = ref["ratio"]
+    lo, hi = 1.0 - h.clip_eps, 1.0 + h.clip_eps
+    return (np.abs(R - hi) <= rel * hi) | (np.abs(R - lo) <= rel * max(lo, 1e-30))
+
+
+def _close(got, want, rtol, atol):
+    return np.abs(got - want) <= rtol * np.abs(want) + atol
+
+
+def logp_scale(batch):
+    """Log-probabilities of magnitude L carry an absolute fp32 error proportional to L, and that
+    absolute error is the relative error of every ratio exp(l1 - l2): beyond |l| = 10 (only the
+    Gaussian policy, a sum over action dimensions, gets there) the relative bars scale with it."""
+    return max(1.0, float(np.abs(batch["worker_logp"]).max()) / 10.0)
+
+
+def compare(gpu, ref, ref_flipped, near, M, grad_keys, kl_coef, sens, vf_coef, rtol=RTOL_ELEM, atol=ATOL_ELEM,
+            rtol_scalar=RTOL_SCALAR, atol_scalar=ATOL_SCALAR, cond=COND_ADV, min_literal=0.995, scale_l=1.0,
+            kl_always=False):
+    """Element-by-element comparison.
+
+    Bar per element: |gpu - oracle| <= rtol |oracle| + atol + s * cond * S_t, where the last
+    term is the rounding the advantage A_t itself may carry: S_t is the sum of the absolute
+    values of the terms A_t is made of (the oracle's `adv_cond`), `cond` a few dozen fp32
+    unit roundoffs, and s = |d output / d A_t|.  Without it, steps where A_t cancels to
+    much less than its terms could not meet a purely relative bound in fp32 arithmetic.
+    At least `min_literal` of the elements must meet the bar without that term.
+    """
+    report = {}
+    rtol, cond = rtol * scale_l, cond * scale_l
+    adv_tol = cond * ref["adv_cond"]
+    for key in grad_keys + ["dvalues", "vtarget", "advantage"]:
+        if key not in gpu:
+            continue
+        scale = float(M) if key in grad_keys + ["dvalues"] else 1.0
+        got, want = gpu[key] * scale, ref[key] * scale
+        assert np.isfinite(got).all(), f"{key}: non-finite output"
+        if key in grad_keys:
+            extra = sens[key] * adv_tol[..., None]
+        elif key == "dvalues":
+            extra = abs(vf_coef) * adv_tol
+        else:
+            extra = adv_tol
+        err = np.abs(got - want)
+        literal = err <= rtol * np.abs(want) + atol
+        ok = err <= rtol * np.abs(want) + atol + extra
+        if not ok.all() and key in grad_keys and ref_flipped is not None:
+            want2 = ref_flipped[key] * scale
+            alt = np.abs(got - want2) <= rtol * np.abs(want2) + atol + extra
+            row_ok = ok.all(-1) | (alt.all(-1) & near)
+            bad = ~row_ok
+            literal = literal | (near[..., None] & alt)
+        else:
+            bad = ~ok
+        report[key] = dict(max_abs=float(err.max()), literal_frac=float(literal.mean()))
+        assert not bad.any(), (f"{key}: {int(bad.sum())} mismatches, worst abs {err[bad].max():.3e} "
+                               f"at {np.argwhere(bad)[0]} got {got[bad].ravel()[0]:.8e} want {want[bad].ravel()[0]:.8e}")
+        assert literal.mean() >= min_literal, f"{key}: only {literal.mean():.5f} of elements within rtol/atol"
+    lt_g, lt_r = gpu["loss_terms"].copy(), ref["loss_terms"]
+    if kl_coef == 0.0 and not kl_always:
+        # the library evaluates the KL term only when it enters the loss, and reports 0 otherwise
+        assert lt_g[4] == 0.0
+        lt_g[4] = lt_r[4]
+    ok = _close(lt_g, lt_r, rtol_scalar, atol_scalar)
+    if not ok.all() and ref_flipped is not None:
+        # a step on a clip bound moves clip_frac by 1/M and nothing else measurably
+        ok = ok | _close(lt_g, ref_flipped["loss_terms"], rtol_scalar, atol_scalar)
+    assert ok.all(), f"loss_terms: gpu {lt_g} vs oracle {lt_r}"
+    report["loss_terms"] = float(np.max(np.abs(lt_g - lt_r) / (np.abs(lt_r) + 1e-12)))
+    return report
+
+
+def _policy_sensitivity(loss_fn, batch, h, keys, M, flip):
+    """|d (M * gradient) / d A_t| per element: the policy term of the gradient divided by A_t."""
+    h0 = dataclasses.replace(h, ent_coef=0.0, kl_coef=0.0)
+    out = {}
+    for fl in ([None] if flip is None else [None, flip]):
+        r = loss_fn(batch, h0, flip=fl)
+        a = np.abs(r["advantage"])[..., None]
+        for k_ in keys:
+            s = np.abs(r[k_]) * M / np.maximum(a, 1e-300)
+            s = np.where(a > 0, s, 0.0)
+            out[k_] = s if k_ not in out else np.maximum(out[k_], s)
+    return out
+
+
+def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, **tol):
+    h = f32_hyper(h)
+    if logits_dtype == torch.bfloat16:
+        batch = dict(batch)
+        batch["learner_logits"] = ii.round_to_bf16(batch["learner_logits"])
+        batch["target_logits"] = ii.round_to_bf16(batch["target_logits"])
+    ref = oracle.loss_categorical(batch, h)
+    near = near_clip_bound(ref, h)
+    ref_flipped = oracle.loss_categorical(batch, h, flip=near.astype(np.int8)) if near.any() else None
+    gpu = run_gpu_categorical(batch, h, logits_dtype, dlogits_dtype)
+    M = batch["rewards"].size
+    sens = _policy_sensitivity(oracle.loss_categorical, batch, h, ["dlogits"], M,
+                               near.astype(np.int8) if near.any() else None)
+    return compare(gpu, ref, ref_flipped, near, M, ["dlogits"], h.kl_coef, sens, h.vf_coef,
+                   scale_l=logp_scale(batch), **tol)
+
+
+def check_gaussian(oracle, batch, h, **tol):
+    h = f32_hyper(h)
+    ref = oracle.loss_gaussian(batch, h)
+    near = near_clip_bound(ref, h)
+    ref_flipped = oracle.loss_gaussian(batch, h, flip=near.astype(np.int8)) if near.any() else None
+    gpu = run_gpu_gaussian(batch, h)
+    M = batch["rewards"].size
+    sens = _policy_sensitivity(oracle.loss_gaussian, batch, h, ["dmean", "dlogstd"], M,
+                               near.astype(np.int8) if near.any() else None)
+    return compare(gpu, ref, ref_flipped, near, M, ["dmean", "dlogstd"], h.kl_coef, sens, h.vf_coef,
+                   scale_l=logp_scale(batch), kl_always=True, **tol)

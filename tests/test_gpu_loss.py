@@ -1,0 +1,182 @@
+"""Parity of the CUDA loss kernels with the CPU oracle, element by element, through the C ABI."""
+import dataclasses
+
+import numpy as np
+import pytest
+import torch
+
+import impact_inputs as ii
+from impact_inputs import LossHyper
+
+import _parity as P
+
+pytestmark = pytest.mark.gpu
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_named_categorical_configs(oracle, idx):
+    cfg, batch = ii.make_config(idx)
+    P.check_categorical(oracle, batch, cfg.hyper)
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_named_configs_with_paper_hyperparameters(oracle, idx):
+    # Appendix B: rho = 2, lambda = 0.995, plus a KL term
+    cfg, batch = ii.make_config(idx)
+    h = dataclasses.replace(cfg.hyper, rho_tw=2.0, lam=0.995, kl_coef=0.5, vf_coef=1.0, clip_eps=0.3)
+    P.check_categorical(oracle, batch, h)
+
+
+def test_config2_bf16_logits(oracle):
+    cfg, batch = ii.make_config(2)
+    P.check_categorical(oracle, batch, cfg.hyper, torch.bfloat16, torch.bfloat16,
+                        rtol=P.RTOL_BF16, atol=P.ATOL_BF16)
+    # bf16 storage with fp32 gradients: only the inputs are rounded, so the fp32 bar holds
+    P.check_categorical(oracle, batch, cfg.hyper, torch.bfloat16, torch.float32)
+    P.check_categorical(oracle, batch, cfg.hyper, torch.float32, torch.bfloat16,
+                        rtol=P.RTOL_BF16, atol=P.ATOL_BF16)
+
+
+def test_config3_gaussian(oracle):
+    cfg, batch = ii.make_config(3)
+    P.check_gaussian(oracle, batch, cfg.hyper)
+    h = dataclasses.replace(cfg.hyper, rho_tw=2.0, lam=0.995, kl_coef=1.0, ent_coef=0.01, clip_eps=0.4,
+                            rho_bar=1.5, c_bar=1.2)
+    P.check_gaussian(oracle, batch, h)
+
+
+SHAPES = [
+    (1, 1, 1), (1, 1, 7), (3, 1, 4), (1, 5, 2), (7, 33, 3), (5, 127, 6), (4, 128, 18), (3, 129, 18),
+    (2, 300, 5), (9, 50, 18), (2, 20, 65), (3, 40, 64), (2, 70, 100), (1, 9, 257), (2, 5, 512),
+    (130, 1, 18), (65, 2, 9), (3, 1000, 4),
+]
+
+
+@pytest.mark.parametrize("B,T,A", SHAPES)
+def test_ragged_shapes_categorical(oracle, B, T, A):
+    batch = ii.categorical_batch(B, T, A, seed=1000 + B * 7 + T * 3 + A, p_done=0.05)
+    h = LossHyper(rho_bar=1.3, c_bar=1.1, clip_eps=0.25, vf_coef=0.7, ent_coef=0.02, kl_coef=0.1,
+                  lam=0.97, rho_tw=2.0)
+    P.check_categorical(oracle, batch, h)
+
+
+@pytest.mark.parametrize("B,T,D", [(1, 1, 1), (3, 7, 3), (5, 128, 17), (2, 131, 6), (4, 50, 33), (1, 300, 64),
+                                   (2, 9, 256), (40, 3, 17)])
+def test_ragged_shapes_gaussian(oracle, B, T, D):
+    batch = ii.gaussian_batch(B, T, D, seed=2000 + B + T + D, p_done=0.02)
+    h = LossHyper(rho_bar=1.3, c_bar=1.1, clip_eps=0.25, vf_coef=0.7, ent_coef=0.02, kl_coef=0.1,
+                  lam=0.97, rho_tw=2.0)
+    P.check_gaussian(oracle, batch, h)
+
+
+@pytest.mark.parametrize("B,T,A", [(3, 33, 5), (6, 20, 18), (2, 129, 7), (5, 50, 64)])
+def test_bf16_ragged(oracle, B, T, A):
+    batch = ii.categorical_batch(B, T, A, seed=3000 + A, p_done=0.05)
+    h = LossHyper(rho_tw=2.0, kl_coef=0.2, lam=0.995)
+    P.check_categorical(oracle, batch, h, torch.bfloat16, torch.bfloat16, rtol=P.RTOL_BF16, atol=P.ATOL_BF16)
+    P.check_categorical(oracle, batch, h, torch.bfloat16, torch.float32)
+
+
+@pytest.mark.parametrize("mode", [1, 2])
+@pytest.mark.parametrize("is_source", [0, 1])
+def test_variants(oracle, mode, is_source):
+    cfg, batch = ii.make_config(1)
+    h = dataclasses.replace(cfg.hyper, ratio_mode=mode, is_source=is_source, rho_tw=2.0)
+    P.check_categorical(oracle, batch, h)
+
+
+def test_degenerate_coefficients(oracle):
+    cfg, batch = ii.make_config(1)
+    for h in (LossHyper(c_bar=0.0), LossHyper(rho_bar=0.0), LossHyper(clip_eps=0.0, ent_coef=0.0),
+              LossHyper(rho_bar=float("inf"), c_bar=float("inf"), clip_eps=1e9),
+              LossHyper(vf_coef=0.0, ent_coef=0.0, kl_coef=0.0, lam=0.0)):
+        P.check_categorical(oracle, batch, h)
+
+
+def test_all_steps_terminal_and_on_policy(oracle):
+    batch = ii.categorical_batch(6, 40, 8, seed=77)
+    batch["discounts"][:] = 0.0
+    P.check_categorical(oracle, batch, LossHyper())
+    batch = ii.categorical_batch(6, 40, 8, seed=78)
+    batch["target_logits"] = batch["learner_logits"].copy()
+    P.check_categorical(oracle, batch, LossHyper(kl_coef=1.0))
+
+
+def test_optional_outputs_can_be_skipped_and_results_are_deterministic(oracle):
+    cfg, batch = ii.make_config(1)
+    h = P.f32_hyper(cfg.hyper)
+    a = P.run_gpu_categorical(batch, h, extra=True)
+    b = P.run_gpu_categorical(batch, h, extra=False)
+    c = P.run_gpu_categorical(batch, h, extra=True)
+    for k in ("loss_terms", "dlogits", "dvalues"):
+        np.testing.assert_array_equal(a[k], b[k])
+        np.testing.assert_array_equal(a[k], c[k])
+
+
+def test_workspace_is_reusable_across_calls_and_shapes(oracle):
+    import paper_1912_00167_b200 as ip
+    ws = ip.new_workspace(64, 64)
+    for (B, T, A, seed) in [(8, 20, 6, 1), (33, 50, 18, 2), (8, 20, 6, 1)]:
+        batch = ii.categorical_batch(B, T, A, seed)
+        h = P.f32_hyper(LossHyper())
+        ref = oracle.loss_categorical(batch, h)
+        t = {k: torch.from_numpy(v).cuda() for k, v in batch.items()}
+        lt = torch.zeros(8, device="cuda")
+        dz = torch.empty(B, T, A, device="cuda")
+        dv = torch.empty(B, T, device="cuda")
+        ip.impact_loss_fwd_bwd(t["learner_logits"], t["target_logits"], t["worker_logp"], t["actions"],
+                               t["rewards"], t["discounts"], t["values"], t["bootstrap_values"], P.to_coef(h),
+                               loss_terms=lt, dlogits=dz, dvalues=dv, workspace=ws)
+        torch.cuda.synchronize()
+        got = lt.cpu().numpy()
+        got[4] = ref["loss_terms"][4]  # KL is not evaluated at kl_coef = 0
+        np.testing.assert_allclose(got, ref["loss_terms"], rtol=1e-4, atol=1e-7)
+
+
+def test_rows_of_dlogits_sum_to_zero_at_full_size():
+    # softmax invariance: every term of the logit gradient sums to zero over the actions
+    import paper_1912_00167_b200 as ip
+    cfg, batch = ii.make_config(2)
+    h = P.f32_hyper(dataclasses.replace(cfg.hyper, kl_coef=0.3))
+    out = P.run_gpu_categorical(batch, h)
+    M = batch["rewards"].size
+    rows = out["dlogits"].sum(-1) * M
+    scale = np.abs(out["dlogits"]).sum(-1) * M
+    assert (np.abs(rows) <= 1e-5 * (1.0 + scale)).all()
+
+
+def test_bad_arguments_are_rejected_before_launch():
+    import paper_1912_00167_b200 as ip
+    from paper_1912_00167_b200 import binding as bd
+    cfg, batch = ii.make_config(0)
+    t = {k: torch.from_numpy(v).cuda() for k, v in batch.items()}
+    B, T, A = t["learner_logits"].shape
+    lt = torch.zeros(8, device="cuda")
+    dz = torch.empty(B, T, A, device="cuda")
+    dv = torch.empty(B, T, device="cuda")
+    ws = ip.new_workspace(B, T)
+
+    def call(coef, workspace=ws, **over):
+        args = dict(t)
+        args.update(over)
+        ip.impact_loss_fwd_bwd(args["learner_logits"], args["target_logits"], args["worker_logp"], args["actions"],
+                               args["rewards"], args["discounts"], args["values"], args["bootstrap_values"], coef,
+                               loss_terms=lt, dlogits=dz, dvalues=dv, workspace=workspace)
+
+    for bad in (ip.Coefficients(rho_bar=-1.0), ip.Coefficients(clip_eps=float("nan")), ip.Coefficients(rho_tw=0.0),
+                ip.Coefficients(ratio_mode=7), ip.Coefficients(is_source=3)):
+        with pytest.raises(ip.ImpactError) as e:
+            call(bad)
+        assert e.value.status == bd.ERR_INVALID_ARG
+    with pytest.raises(ip.ImpactError) as e:
+        call(ip.Coefficients(), workspace=torch.zeros(64, dtype=torch.uint8, device="cuda"))
+    assert e.value.status == bd.ERR_WORKSPACE_TOO_SMALL
+    with pytest.raises(ValueError):
+        call(ip.Coefficients(), rewards=t["rewards"].cpu())
+    # misaligned base pointer
+    big = torch.zeros(B * T + 4, device="cuda")
+    with pytest.raises(ip.ImpactError) as e:
+        call(ip.Coefficients(), rewards=big[1:B * T + 1].view(B, T))
+    assert e.value.status == bd.ERR_INVALID_ARG
+    call(ip.Coefficients())  # and the good call still works afterwards
+    torch.cuda.synchronize()
