@@ -1,0 +1,379 @@
+#!/usr/bin/env python
+"""Benchmark of the IMPACT learner hot path: circular-buffer sample -> fused loss + gradients.
+
+One step is one learner iteration of Algorithm 1 on one train batch:
+  obtain a batch from C(N, K) (zero-copy sample) -> if it is the batch's first traversal,
+  append the target network's output to its slot -> loss + gradients in one fused launch ->
+  when the traversal was the K-th, a new worker batch is pushed into the freed slot.
+Metric: learner timesteps per second (B*T steps per iteration).
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints one JSON line.  `--impl reference` times the CPU oracle instead (a deliberately
+plain program: context, not a target).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import tempfile
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+import numpy as np
+
+import impact_inputs as ii
+
+METRIC = "learner loss+grad timesteps/sec at BxT=131k, A=18"
+UNIT = "timesteps/s"
+WORKLOAD_IDX = 2  # B=1024 x T=128, A=18, fp32, ring N=32, K=4
+FALLBACK_HBM_GBS = 6650.0
+FIELD_NAMES = ["actions", "rewards", "discounts", "worker_logp", "target_logits"]
+N_DISTINCT = 4    # distinct synthetic batches generated on the host
+N_SETS = 16       # rotating learner-output / gradient buffer sets (footprint beyond L2)
+
+
+def algorithmic_bytes_per_step(A: int, logits_bytes: int = 4, grad_bytes: int = 4) -> int:
+    """Bytes the loss must move per timestep: 2A logits + 5 scalars in, A gradients + dvalues out."""
+    return 2 * A * logits_bytes + 5 * 4 + A * grad_bytes + 4
+
+
+def peak_hbm_gbs():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            return float(json.load(f)["hbm_gbs"]), "measured"
+    except Exception:
+        return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.proc = None
+        self.path = None
+
+    def start(self):
+        try:
+            fd, self.path = tempfile.mkstemp(prefix="clocks_", suffix=".csv")
+            os.close(fd)
+            self.out = open(self.path, "w")
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits", "-lms", "100",
+                 "-i", str(self.gpu_index)], stdout=self.out, stderr=subprocess.DEVNULL)
+        except Exception:
+            self.proc = None
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        self.out.close()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        with open(self.path) as f:
+            for line in f:
+                parts = [x.strip() for x in line.split(",")]
+                if len(parts) < 9:
+                    continue
+                try:
+                    sm.append(float(parts[1]))
+                    smax.append(float(parts[2]))
+                except ValueError:
+                    continue
+                for n, v in zip(names, parts[5:9]):
+                    if v.lower().startswith("active"):
+                        reasons.add(n)
+        try:
+            os.unlink(self.path)
+        except OSError:
+            pass
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def time_oracle(batch, hyper, min_seconds: float, max_reps: int):
+    """Times the oracle, as it stands, on repeated full batches of the workload."""
+    import oracle
+    oracle.build()
+    oracle.loss_categorical(batch, hyper)  # page in
+    reps, t0 = 0, time.perf_counter()
+    while True:
+        oracle.loss_categorical(batch, hyper)
+        reps += 1
+        el = time.perf_counter() - t0
+        if el >= min_seconds or reps >= max_reps:
+            break
+    M = batch["rewards"].size
+    return reps * M / el, reps, el
+
+
+def run_reference(args):
+    """The reference arm: the CPU oracle on the same workload, metric and unit."""
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    cfg, batch = ii.make_config(WORKLOAD_IDX)
+    import oracle
+    oracle.build()
+    M = cfg.B * cfg.T
+    for _ in range(args.warmup):
+        oracle.loss_categorical(batch, cfg.hyper)
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        oracle.loss_categorical(batch, cfg.hyper)
+    el = time.perf_counter() - t0
+    value = args.steps * M / el
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * el / args.steps,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"config 2: categorical B={cfg.B} T={cfg.T} A={cfg.A} fp32 (loss + gradients only)"},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+                         "sample": f"{args.steps} full batches of {M} timesteps, one per step"},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=2000)
+    ap.add_argument("--warmup", type=int, default=200)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.warmup < 3:
+        args.warmup = 3
+    if args.impl == "reference":
+        run_reference(args)
+        return
+
+    import torch
+    import paper_1912_00167_b200 as ip
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_
+        dist = dist_
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+    ip.load_library()
+
+    cfg = ii.CONFIGS[WORKLOAD_IDX]
+    B, T, A, N, K = cfg.B, cfg.T, cfg.A, cfg.ring_N, cfg.ring_K
+    M = B * T
+    h = cfg.hyper
+    coef = ip.Coefficients(rho_bar=h.rho_bar, c_bar=h.c_bar, clip_eps=h.clip_eps, vf_coef=h.vf_coef,
+                           ent_coef=h.ent_coef, kl_coef=h.kl_coef, lam=h.lam, rho_tw=h.rho_tw)
+
+    # ---- synthetic data: a few distinct seeded batches, replicated over rotating buffer sets ----------
+    host = [ii.make_config(WORKLOAD_IDX, seed=cfg.seed + 1000 * rank + i)[1] for i in range(N_DISTINCT)]
+    dev = [{k: torch.from_numpy(v).cuda() for k, v in b.items()} for b in host]
+    worker_batches = [[d[n].clone() for n in FIELD_NAMES] for d in dev for _ in range(N_SETS // N_DISTINCT)]
+    learner_sets = [dict(learner_logits=dev[i % N_DISTINCT]["learner_logits"].clone(),
+                         values=dev[i % N_DISTINCT]["values"].clone(),
+                         bootstrap_values=dev[i % N_DISTINCT]["bootstrap_values"].clone()) for i in range(N_SETS)]
+    out_sets = [dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
+                     dvalues=torch.empty(B, T, device="cuda")) for _ in range(N_SETS)]
+    workspace = ip.new_workspace(B, T)
+    field_bytes = [t.numel() * t.element_size() for t in worker_batches[0]]
+    ring = ip.ImpactBuffer(N, K, field_bytes, seed=cfg.seed)
+    stream = torch.cuda.current_stream()
+
+    # one prepared loss call per slot: the slot's fields in place, learner outputs / gradients of set slot % N_SETS
+    calls = []
+    proto = worker_batches[0]
+    for s in range(N):
+        v = [ring.slot_view(s, f, proto[f].dtype, proto[f].shape) for f in range(len(FIELD_NAMES))]
+        ls, os_ = learner_sets[s % N_SETS], out_sets[s % N_SETS]
+        calls.append(ip.prepare_loss_fwd_bwd(ls["learner_logits"], v[4], v[3], v[0], v[1], v[2], ls["values"],
+                                             ls["bootstrap_values"], coef, workspace=workspace, **os_))
+
+    counters = {"loss": 0, "copy": 0, "pushed": 0}
+    slot_batch = [0] * N  # which synthetic worker batch sits in each slot
+
+    def push_one():
+        idx = counters["pushed"] % len(worker_batches)
+        src = list(worker_batches[idx])
+        src[4] = None  # the target network's output is appended at the first traversal
+        slot = ring.push(src, stream)
+        if slot is not None:
+            slot_batch[slot] = idx
+            counters["pushed"] += 1
+            counters["copy"] += 1
+        return slot
+
+    def step(timer=None):
+        got = ring.sample(None, stream)
+        if got is None:
+            raise RuntimeError("ring ran empty")
+        slot, k = got
+        if k == 0:  # first traversal: store the target network's output for this batch
+            ring.append(slot, 4, worker_batches[slot_batch[slot]][4], stream)
+            counters["copy"] += 1
+        if timer is not None:
+            timer[0].record(stream)
+        calls[slot](stream)
+        if timer is not None:
+            timer[1].record(stream)
+        counters["loss"] += 1
+        if k == K - 1:
+            push_one()
+
+    while push_one() is not None:
+        pass
+    for _ in range(args.warmup):
+        step()
+    torch.cuda.synchronize()
+
+    def barrier():
+        if dist is not None:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    # ---- timed region 1: K steps, whole-step throughput ---------------------------------------------------
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.25)
+    for c in counters:
+        counters[c] = counters[c] if c == "pushed" else 0
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    t_wall0 = time.perf_counter()
+    e0.record(stream)
+    for _ in range(args.steps):
+        step()
+    e1.record(stream)
+    barrier()
+    t_wall = time.perf_counter() - t_wall0
+    ms_total = e0.elapsed_time(e1)
+    launches = counters["loss"] + counters["copy"]
+    loss_launches = counters["loss"]
+
+    # ---- timed region 2: the same K steps again, an event pair around every loss launch (roofline) -------
+    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
+    barrier()
+    for i in range(args.steps):
+        step(pairs[i])
+    barrier()
+    loss_ms = [a.elapsed_time(b) for a, b in pairs]
+    # ---- and back to back: K loss launches over the rotating slots, nothing between them -----------------
+    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    barrier()
+    d0.record(stream)
+    for i in range(args.steps):
+        calls[i % N](stream)
+    d1.record(stream)
+    barrier()
+    dense_ms = d0.elapsed_time(d1) / args.steps
+    time.sleep(0.15)
+    clocks = sampler.stop()
+
+    # ---- end to end: inputs in pinned host memory, copied in every step; loss terms read back ------------
+    e2e_steps = max(3, min(args.steps, 50))
+    hb = host[0]
+    pinned = {k: torch.from_numpy(v).pin_memory() for k, v in hb.items()}
+    dst = {k: torch.empty_like(v, device="cuda") for k, v in pinned.items()}
+    out = out_sets[0]
+    terms_host = torch.empty(8).pin_memory()
+    e2e_call = ip.prepare_loss_fwd_bwd(dst["learner_logits"], dst["target_logits"], dst["worker_logp"],
+                                       dst["actions"], dst["rewards"], dst["discounts"], dst["values"],
+                                       dst["bootstrap_values"], coef, workspace=workspace, **out)
+    h2d = sum(v.numel() * v.element_size() for v in pinned.values())
+
+    def e2e_step():
+        for k_, v in pinned.items():
+            dst[k_].copy_(v, non_blocking=True)
+        e2e_call(stream)
+        terms_host.copy_(out["loss_terms"], non_blocking=True)
+        stream.synchronize()
+
+    for _ in range(3):
+        e2e_step()
+    barrier()
+    t0 = time.perf_counter()
+    for _ in range(e2e_steps):
+        e2e_step()
+    barrier()
+    e2e_s = time.perf_counter() - t0
+
+    # ---- reduce over ranks: the slowest rank sets the time ---------------------------------------------------
+    vals = torch.tensor([ms_total, e2e_s, statistics.fmean(loss_ms), dense_ms], device="cuda", dtype=torch.float64)
+    if dist is not None:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    ms_total, e2e_s, loss_ms_avg, dense_ms = [float(x) for x in vals.cpu()]
+    value = world * args.steps * M / (ms_total * 1e-3)
+    e2e_value = world * e2e_steps * M / e2e_s
+
+    peak, peak_kind = peak_hbm_gbs()
+    bytes_per_launch = algorithmic_bytes_per_step(A) * M
+    achieved = bytes_per_launch / (dense_ms * 1e-3) / 1e9
+    roofline = {
+        "bound": "hbm", "kernel": "impact_loss_categorical_kernel<float,float,128>",
+        "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
+        "traffic": None,
+        "algorithmic_bytes_per_launch": bytes_per_launch,
+        "avg_launch_us": dense_ms * 1e3,
+        "how": "K back-to-back loss launches over the rotating ring slots, CUDA events on the launch stream",
+        "avg_launch_us_event_pair_in_step": loss_ms_avg * 1e3,
+        "achieved_event_pair_in_step": bytes_per_launch / (loss_ms_avg * 1e-3) / 1e9,
+    }
+
+    line = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms_total / args.steps, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "f32", "data": "synthetic",
+        "config": {
+            "workload": f"config 2: categorical B={B} T={T} A={A} fp32, ring N={N} K={K} (zero-copy sample, "
+                        f"append at k=0, push on discard)",
+            "parallelism": "replicas only" if world > 1 else "single GPU",
+            "l2": f"inputs larger than L2: ring {ring.storage_bytes(N, field_bytes) >> 20} MiB + {N_SETS} "
+                  f"learner-output sets + {N_SETS} gradient sets, rotated",
+            "host_wall_ms_per_step": 1e3 * t_wall / args.steps,
+        },
+        "clocks": clocks,
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 32,
+                "steps": e2e_steps},
+        "gpu_launches": launches,
+        "gpu_launches_loss": loss_launches,
+        "roofline": roofline,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        v, reps, el = time_oracle(host[0], h, min_seconds=10.0, max_reps=200)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
+                                "sample": f"{reps} full batches of {M} timesteps (loss + gradients), {el:.1f} s"}
+    if rank == 0:
+        print(json.dumps(line))
+    ring.close()
+    if dist is not None:
+        dist.destroy_process_group()
+
+
+if __name__ == "__main__":
+    main()
