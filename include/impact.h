@@ -182,6 +182,41 @@ int32_t impact_loss_fwd_bwd_gaussian(
     float* loss_terms, float* dmean, float* dlogstd, float* dvalues, float* vtarget,
     float* advantage, void* workspace, size_t workspace_bytes, void* stream);
 
+/*
+ * impact_loss_fwd_bwd for callers that cannot allocate device memory.  (The paper has no
+ * counterpart of this call; it exists for the way the library gets embedded.)
+ *
+ * Some hosts of this library run where cudaMalloc is off limits: a plugin called from
+ * inside another framework's step, whose memory pool owns the whole device; a real-time
+ * control loop that may not block on the driver's allocator; a process that was handed
+ * fixed buffers by its parent and nothing else.  Such a caller has no workspace to pass.
+ * This entry point therefore takes none: the per-block sums and the completion counter
+ * live in a 33,024-byte array that is part of the library image (one copy on every GPU that
+ * loads the library, held until the process exits).  Inputs, outputs, arithmetic and
+ * results are those of impact_loss_fwd_bwd; nothing is allocated or freed, here or in
+ * anything this call uses.
+ *
+ * Limits: A <= 64, and the batch must split into at most 1024 tiles of 128 steps:
+ * ceil(B / floor(128 / T)) <= 1024 when T <= 128, else B <= 1024.  (B=1024, T=128 is the
+ * largest batch of full-length trajectories.)  Larger batches return
+ * IMPACT_ERR_WORKSPACE_TOO_SMALL, A > 64 returns IMPACT_ERR_UNSUPPORTED; use
+ * impact_loss_fwd_bwd with a workspace for those.
+ *
+ * The first call on a device looks up the array's device address (a driver query, with that
+ * device current); make that first call outside any stream capture.  Every call enqueues a
+ * small clear of the counter before its kernel, since the array still holds what the
+ * previous call left.  All calls on a device share the one array: two calls whose kernels
+ * may run at the same time (different streams, or different host threads without ordering)
+ * corrupt each other's sums.  Keep them on one stream or order them with events.
+ */
+int32_t impact_loss_fwd_bwd_static_scratch(
+    const void* learner_logits, const void* target_logits, const float* worker_logp,
+    const int32_t* actions, const float* rewards, const float* discounts, const float* values,
+    const float* bootstrap_values, float rho_bar, float c_bar, float clip_eps,
+    const impact_coefficients* coef, int64_t B, int64_t T, int32_t A, int32_t logits_dtype,
+    float* loss_terms, void* dlogits, float* dvalues, float* vtarget, float* advantage,
+    void* stream);
+
 /* ---- circular buffer C(N, K) ---------------------------------------------------------- */
 
 /*

@@ -32,6 +32,7 @@ EXPORTS = (
     "impact_buffer_destroy", "impact_buffer_push", "impact_buffer_sample", "impact_buffer_append",
     "impact_buffer_slot_ptr", "impact_buffer_live", "impact_buffer_state_bytes",
     "impact_buffer_export_state", "impact_buffer_import_state", "impact_gather_rows",
+    "impact_loss_fwd_bwd_static_scratch",
 )
 
 
@@ -71,6 +72,9 @@ def load_library() -> ctypes.CDLL:
     lib.impact_loss_fwd_bwd.restype = _i32
     lib.impact_loss_fwd_bwd.argtypes = [_vp] * 8 + [_f32] * 3 + [ctypes.POINTER(impact_coefficients), _i64, _i64,
                                                                _i32, _i32] + [_vp] * 6 + [_sz, _vp]
+    lib.impact_loss_fwd_bwd_static_scratch.restype = _i32
+    lib.impact_loss_fwd_bwd_static_scratch.argtypes = [_vp] * 8 + [_f32] * 3 + [
+        ctypes.POINTER(impact_coefficients), _i64, _i64, _i32, _i32] + [_vp] * 5 + [_vp]
     lib.impact_loss_fwd_bwd_gaussian.restype = _i32
     lib.impact_loss_fwd_bwd_gaussian.argtypes = [_vp] * 10 + [_f32] * 3 + [ctypes.POINTER(impact_coefficients),
                                                                          _i64, _i64, _i32] + [_vp] * 7 + [_sz, _vp]
@@ -224,6 +228,34 @@ def impact_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, rew
     prepare_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
                          bootstrap_values, coef, loss_terms=loss_terms, dlogits=dlogits, dvalues=dvalues,
                          vtarget=vtarget, advantage=advantage, workspace=workspace)(stream)
+
+
+def impact_loss_fwd_bwd_static_scratch(learner_logits, target_logits, worker_logp, actions, rewards, discounts,
+                                       values, bootstrap_values, coef: Coefficients, *, loss_terms, dlogits,
+                                       dvalues, vtarget=None, advantage=None, stream=None) -> None:
+    """impact_loss_fwd_bwd without a workspace argument, for callers that may not allocate.
+
+    The scratch the kernel needs sits in an array inside the library, so this call takes only
+    inputs and outputs.  Batches are limited to 1024 tiles of 128 steps and A <= 64; all calls
+    on a device share the array, so keep them ordered on one stream (see include/impact.h).
+    """
+    lib = load_library()
+    B, T, A = learner_logits.shape
+    ldt = learner_logits.dtype
+    if ldt not in _DTYPE_CODE or dlogits.dtype not in _DTYPE_CODE:
+        raise ValueError("logits must be float32 or bfloat16")
+    f32, bt = torch.float32, (B, T)
+    cs = coef.c_struct(_DTYPE_CODE[dlogits.dtype])
+    st = lib.impact_loss_fwd_bwd_static_scratch(
+        _dev(learner_logits, ldt, (B, T, A), "learner_logits"), _dev(target_logits, ldt, (B, T, A), "target_logits"),
+        _dev(worker_logp, f32, bt, "worker_logp"), _dev(actions, torch.int32, bt, "actions"),
+        _dev(rewards, f32, bt, "rewards"), _dev(discounts, f32, bt, "discounts"), _dev(values, f32, bt, "values"),
+        _dev(bootstrap_values, f32, (B,), "bootstrap_values"),
+        coef.rho_bar, coef.c_bar, coef.clip_eps, ctypes.pointer(cs), B, T, A, _DTYPE_CODE[ldt],
+        _dev(loss_terms, f32, (NUM_TERMS,), "loss_terms"), _dev(dlogits, dlogits.dtype, (B, T, A), "dlogits"),
+        _dev(dvalues, f32, bt, "dvalues"), _dev(vtarget, f32, bt, "vtarget", True),
+        _dev(advantage, f32, bt, "advantage", True), _stream(stream))
+    _check(st, "impact_loss_fwd_bwd_static_scratch")
 
 
 def prepare_loss_fwd_bwd_gaussian(learner_mean, learner_logstd, target_mean, target_logstd, worker_logp, actions,

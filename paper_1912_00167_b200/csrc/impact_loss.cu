@@ -608,3 +608,95 @@ extern "C" int32_t impact_loss_fwd_bwd_gaussian(
         default: return launch_gaussian<32>(p, di, s);
     }
 }
+
+// ------------------------------------------------------------------------------------------
+// Variant for callers that must not allocate
+// ------------------------------------------------------------------------------------------
+namespace impact {
+namespace {
+
+constexpr int kStaticMaxBlocks = 1024;  // tiles (= blocks) the built-in scratch has room for
+constexpr size_t kStaticScratchBytes = (size_t)kStaticMaxBlocks * 8 * sizeof(float) + kCounterBytes;
+
+// Scratch that lives in the library image: per-block sums first, the completion counter in
+// the last 256 bytes.  Every device that loads the library carries its own copy.
+static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
+
+// Device address of g_static_scratch on the current device.  In host code the symbol's name
+// is only a handle, so the address is asked for once per device and remembered.
+int32_t static_scratch_address(const DeviceInfo* di, unsigned char** out) {
+    static unsigned char* address[64] = {};
+    if (!address[di->device]) {
+        void* p = nullptr;
+        IMPACT_CUDA_TRY(cudaGetSymbolAddress(&p, g_static_scratch));
+        address[di->device] = static_cast<unsigned char*>(p);
+    }
+    *out = address[di->device];
+    return IMPACT_OK;
+}
+
+}  // namespace
+}  // namespace impact
+
+extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
+    const void* learner_logits, const void* target_logits, const float* worker_logp,
+    const int32_t* actions, const float* rewards, const float* discounts, const float* values,
+    const float* bootstrap_values, float rho_bar, float c_bar, float clip_eps,
+    const impact_coefficients* coef, int64_t B, int64_t T, int32_t A, int32_t logits_dtype,
+    float* loss_terms, void* dlogits, float* dvalues, float* vtarget, float* advantage,
+    void* stream) {
+    if (!learner_logits || !target_logits || !worker_logp || !actions || !rewards || !discounts ||
+        !values || !bootstrap_values || !coef || !loss_terms || !dlogits || !dvalues)
+        return IMPACT_ERR_INVALID_ARG;
+    if (B <= 0 || T <= 0 || A <= 0) return IMPACT_ERR_INVALID_ARG;
+    const void* ptrs[] = {learner_logits, target_logits, worker_logp, actions, rewards, discounts,
+                          values, bootstrap_values, loss_terms, dlogits, dvalues};
+    for (const void* q : ptrs)
+        if (!aligned16(q)) return IMPACT_ERR_INVALID_ARG;
+    if ((vtarget && !aligned16(vtarget)) || (advantage && !aligned16(advantage))) return IMPACT_ERR_INVALID_ARG;
+    if (logits_dtype != IMPACT_DTYPE_F32 && logits_dtype != IMPACT_DTYPE_BF16) return IMPACT_ERR_INVALID_ARG;
+    if (coef->dlogits_dtype != IMPACT_DTYPE_F32 && coef->dlogits_dtype != IMPACT_DTYPE_BF16)
+        return IMPACT_ERR_INVALID_ARG;
+    if (A > 64) return IMPACT_ERR_UNSUPPORTED;  // keeps the tile at 128 steps, which the limit below counts in
+
+    CatParams p;
+    int32_t st = fill_scalars(p.k, rho_bar, c_bar, clip_eps, coef, B, T);
+    if (st != IMPACT_OK) return st;
+    p.A = A;
+    p.As = pad_odd(A);
+    const int nt = pick_nt(p.As, 2, 72 * 1024);
+    p.geo = make_geometry(B, T, nt);
+    // one block's sums per tile at most: more tiles than the built-in scratch holds are refused
+    if (nt != 128 || p.geo.nchunks > kStaticMaxBlocks) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
+
+    const DeviceInfo* di = current_device_info();
+    if (!di) return IMPACT_ERR_CUDA;
+    unsigned char* scratch = nullptr;
+    st = static_scratch_address(di, &scratch);
+    if (st != IMPACT_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    // the scratch keeps whatever the previous call left; the counter is what has to start at zero
+    unsigned char* counter = scratch + (size_t)kStaticMaxBlocks * 8 * sizeof(float);
+    IMPACT_CUDA_TRY(cudaMemsetAsync(counter, 0, kCounterBytes, s));
+
+    p.learner_logits = learner_logits;
+    p.target_logits = target_logits;
+    p.worker_logp = worker_logp;
+    p.actions = actions;
+    p.rewards = rewards;
+    p.discounts = discounts;
+    p.values = values;
+    p.bootstrap = bootstrap_values;
+    p.loss_terms = loss_terms;
+    p.dlogits = dlogits;
+    p.dvalues = dvalues;
+    p.vtarget = vtarget;
+    p.advantage = advantage;
+    p.partials = reinterpret_cast<float*>(scratch);
+    p.counter = reinterpret_cast<unsigned int*>(counter);
+    const bool lb = logits_dtype == IMPACT_DTYPE_BF16, gb = coef->dlogits_dtype == IMPACT_DTYPE_BF16;
+    if (!lb && !gb) return dispatch_nt<float, float>(p, nt, di, s);
+    if (!lb && gb) return dispatch_nt<float, __nv_bfloat16>(p, nt, di, s);
+    if (lb && !gb) return dispatch_nt<__nv_bfloat16, float>(p, nt, di, s);
+    return dispatch_nt<__nv_bfloat16, __nv_bfloat16>(p, nt, di, s);
+}
