@@ -227,6 +227,295 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
 }
 
 // ------------------------------------------------------------------------------------------
+// Categorical policy, action count known at compile time (the hot variant)
+// ------------------------------------------------------------------------------------------
+// Same decomposition as the kernel above (128 steps per block, one thread per step), but:
+//   * the two logits slabs of a tile arrive by ONE bulk asynchronous copy each, issued by a
+//     single thread and signalled through an mbarrier, and the gradient slab leaves by one
+//     bulk store: staging costs no per-element instructions and all of a tile's bytes are
+//     in flight at once;
+//   * the slabs keep their dense global layout in shared memory; a thread reads its row
+//     with the widest vector access the row pitch allows, which is bank-conflict free for
+//     the action counts compiled here (pitch/width odd);
+//   * A is a template parameter, rows live in registers, every loop is unrolled;
+//   * the softmax runs on exp2 of pre-scaled differences (one multiply + one MUFU each).
+// With ~19 KB of shared memory and <= 72 registers, 7 blocks fit an SM, so the 1024 tiles of
+// a B*T = 131072 batch are all resident at once on 148 SMs and every load is issued up front.
+template <typename ST, int W> struct RowIO;
+
+template <int W> struct RowIO<float, W> {
+    static constexpr int VW = (W % 4 == 0) ? 4 : ((W % 2 == 0) ? 2 : 1);
+    static __device__ __forceinline__ void load(const unsigned char* slab, int row, float (&z)[W]) {
+        const float* r = reinterpret_cast<const float*>(slab) + row * W;
+        if constexpr (VW == 4) {
+#pragma unroll
+            for (int j = 0; j < W / 4; ++j) {
+                const float4 v = reinterpret_cast<const float4*>(r)[j];
+                z[4 * j] = v.x; z[4 * j + 1] = v.y; z[4 * j + 2] = v.z; z[4 * j + 3] = v.w;
+            }
+        } else if constexpr (VW == 2) {
+#pragma unroll
+            for (int j = 0; j < W / 2; ++j) {
+                const float2 v = reinterpret_cast<const float2*>(r)[j];
+                z[2 * j] = v.x; z[2 * j + 1] = v.y;
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < W; ++j) z[j] = r[j];
+        }
+    }
+    static __device__ __forceinline__ void store(unsigned char* slab, int row, const float (&g)[W]) {
+        float* r = reinterpret_cast<float*>(slab) + row * W;
+        if constexpr (VW == 4) {
+#pragma unroll
+            for (int j = 0; j < W / 4; ++j)
+                reinterpret_cast<float4*>(r)[j] = make_float4(g[4 * j], g[4 * j + 1], g[4 * j + 2], g[4 * j + 3]);
+        } else if constexpr (VW == 2) {
+#pragma unroll
+            for (int j = 0; j < W / 2; ++j) reinterpret_cast<float2*>(r)[j] = make_float2(g[2 * j], g[2 * j + 1]);
+        } else {
+#pragma unroll
+            for (int j = 0; j < W; ++j) r[j] = g[j];
+        }
+    }
+    static __device__ __forceinline__ float at(const unsigned char* slab, int row, int col) {
+        return reinterpret_cast<const float*>(slab)[row * W + col];
+    }
+};
+
+template <int W> struct RowIO<__nv_bfloat16, W> {
+    static __device__ __forceinline__ void load(const unsigned char* slab, int row, float (&z)[W]) {
+        if constexpr (W % 2 == 0) {
+            const uint32_t* r = reinterpret_cast<const uint32_t*>(slab) + row * (W / 2);
+#pragma unroll
+            for (int j = 0; j < W / 2; ++j) {
+                const uint32_t w = r[j];
+                z[2 * j] = __uint_as_float(w << 16);
+                z[2 * j + 1] = __uint_as_float(w & 0xFFFF0000u);
+            }
+        } else {
+            const unsigned short* r = reinterpret_cast<const unsigned short*>(slab) + row * W;
+#pragma unroll
+            for (int j = 0; j < W; ++j) z[j] = __uint_as_float((uint32_t)r[j] << 16);
+        }
+    }
+    static __device__ __forceinline__ void store(unsigned char* slab, int row, const float (&g)[W]) {
+        if constexpr (W % 2 == 0) {
+            uint32_t* r = reinterpret_cast<uint32_t*>(slab) + row * (W / 2);
+#pragma unroll
+            for (int j = 0; j < W / 2; ++j) r[j] = dev::Pack<__nv_bfloat16>::two(g[2 * j], g[2 * j + 1]);
+        } else {
+            __nv_bfloat16* r = reinterpret_cast<__nv_bfloat16*>(slab) + row * W;
+#pragma unroll
+            for (int j = 0; j < W; ++j) r[j] = __float2bfloat16_rn(g[j]);
+        }
+    }
+    static __device__ __forceinline__ float at(const unsigned char* slab, int row, int col) {
+        return __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(slab)[row * W + col] << 16);
+    }
+};
+
+constexpr int kRegTileRows = 128;
+
+template <typename LT, typename GT, int A>
+constexpr size_t reg_kernel_smem() {
+    constexpr size_t in_row = A * sizeof(LT), out_row = A * sizeof(GT);
+    return kRegTileRows * ((in_row > out_row ? in_row : out_row) + in_row);
+}
+
+template <typename LT, typename GT, int A>
+__global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_kernel(const CatParams p) {
+    constexpr int NT = kRegTileRows;
+    constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
+    constexpr int kRegion0 = NT * (kInRow > kOutRow ? kInRow : kOutRow);
+    constexpr float kLog2e = 1.4426950408889634f;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    unsigned char* const s0 = smem_raw;             // learner logits in, gradients out
+    unsigned char* const s1 = smem_raw + kRegion0;  // target logits
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ float2 warp_agg[NT / 32];
+    __shared__ float red[NT / 32][8];
+    __shared__ float carry_s;
+
+    const int tid = threadIdx.x;
+    const LossScalars k = p.k;
+    const TileGeometry g = p.geo;
+    const LT* const zl = static_cast<const LT*>(p.learner_logits);
+    const LT* const zt = static_cast<const LT*>(p.target_logits);
+    GT* const dz = static_cast<GT*>(p.dlogits);
+    const bool want_kl = (k.kl_coef != 0.0f);
+
+    if (tid == 0) dev::mbarrier_init(&bar, 1);
+    __syncthreads();
+    uint32_t parity = 0;
+
+    float acc[dev::kNumSums];
+#pragma unroll
+    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = 0.0f;
+
+    for (long long chunk = blockIdx.x; chunk < g.nchunks; chunk += gridDim.x) {
+        float carry = 0.0f;
+        for (int tile = g.ntiles - 1; tile >= 0; --tile) {
+            const TileRows tr = tile_rows<NT>(g, chunk, tile);
+            const long long base = tr.row0 * A;
+            const LT* const gl = zl + base;
+            const LT* const gt = zt + base;
+            GT* const gd = dz + base;
+            const uint32_t in_bytes = (uint32_t)tr.nrows * kInRow, out_bytes = (uint32_t)tr.nrows * kOutRow;
+            const bool bulk_in = (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | in_bytes) & 15u) == 0);
+            const bool bulk_out = (((reinterpret_cast<uintptr_t>(gd) | out_bytes) & 15u) == 0);
+            // shared memory is free here: the previous tile's rows were read into registers before
+            // its scan barrier, and its store was drained before the barrier that ended the tile
+            if (bulk_in) {
+                if (tid == 0) {
+                    dev::mbarrier_expect_tx(&bar, 2 * in_bytes);
+                    dev::bulk_load(s0, gl, in_bytes, &bar);
+                    dev::bulk_load(s1, gt, in_bytes, &bar);
+                }
+            } else {  // ragged or unaligned slab: plain element copies
+                const int nelem = tr.nrows * A;
+                for (int e = tid; e < nelem; e += NT) {
+                    reinterpret_cast<LT*>(s0)[e] = gl[e];
+                    reinterpret_cast<LT*>(s1)[e] = gt[e];
+                }
+            }
+
+            // per-step scalars straight from global memory (coalesced), in flight with the slabs
+            const bool active = tid < tr.nrows;
+            const long long row = tr.row0 + tid;
+            dev::StepIn s;
+            int a = 0;
+            if (active) {
+                long long b, t;
+                if (g.ntiles > 1) { b = chunk; t = (long long)tile * NT + tid; }
+                else { const int q = tid / (int)g.T; b = chunk * g.G + q; t = tid - q * (int)g.T; }
+                a = p.actions[row];
+                a = a < 0 ? 0 : (a >= A ? A - 1 : a);
+                s.l_worker = p.worker_logp[row];
+                s.reward = p.rewards[row];
+                s.discount = p.discounts[row];
+                s.value = p.values[row];
+                s.last_step = (t == g.T - 1);
+                s.value_next = s.last_step ? p.bootstrap[b] : p.values[row + 1];
+            }
+
+            if (bulk_in) {
+                if (!dev::mbarrier_wait(&bar, parity)) atomicExch(p.counter + 1, 1u);
+                parity ^= 1u;
+            } else {
+                __syncthreads();
+            }
+
+            float fa = 1.0f, fb = 0.0f;
+            float d[A], e[A];  // learner row: z - max, and 2^((z - max) log2 e)
+            float ln_s = 0.0f, inv_s = 0.0f, lse_t = 0.0f, ent = 0.0f, kl = 0.0f;
+            bool truncated = false;
+            if (active) {
+                {   // target row: only its log-sum-exp and the taken action's logit are needed
+                    float zr[A];
+                    RowIO<LT, A>::load(s1, tid, zr);
+                    float m = zr[0];
+#pragma unroll
+                    for (int j = 1; j < A; ++j) m = fmaxf(m, zr[j]);
+                    float sum = 0.0f;
+#pragma unroll
+                    for (int j = 0; j < A; ++j) sum += dev::exp2_fast((zr[j] - m) * kLog2e);
+                    lse_t = m + logf(sum);
+                    s.l_target = RowIO<LT, A>::at(s1, tid, a) - lse_t;
+                }
+                RowIO<LT, A>::load(s0, tid, d);
+                float m = d[0];
+#pragma unroll
+                for (int j = 1; j < A; ++j) m = fmaxf(m, d[j]);
+                float sum = 0.0f, sed = 0.0f;
+#pragma unroll
+                for (int j = 0; j < A; ++j) {
+                    d[j] -= m;
+                    e[j] = dev::exp2_fast(d[j] * kLog2e);
+                    sum += e[j];
+                    sed = fmaf(e[j], d[j], sed);
+                }
+                ln_s = logf(sum);
+                inv_s = 1.0f / sum;
+                ent = ln_s - sed * inv_s;  // H = ln S - sum_j e_j (z_j - m) / S
+                s.l_theta = (RowIO<LT, A>::at(s0, tid, a) - m) - ln_s;
+                if (want_kl) {
+                    float zr[A];
+                    RowIO<LT, A>::load(s1, tid, zr);
+#pragma unroll
+                    for (int j = 0; j < A; ++j) {
+                        const float lpt = zr[j] - lse_t;
+                        kl = fmaf(dev::exp2_fast(lpt * kLog2e), lpt - (d[j] - ln_s), kl);
+                    }
+                }
+                truncated = dev::recursion_map(s, k, fa, fb);
+            }
+            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
+            if (tid == 0) carry_s = adv;
+
+            float sums[dev::kNumSums];
+#pragma unroll
+            for (int j = 0; j < dev::kNumSums; ++j) sums[j] = 0.0f;
+            if (active) {
+                float surr, ratio;
+                bool clipped;
+                const float wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
+                // d total / d logit_j = [ wpg (pi_j - 1[j=a]) + ent_coef pi_j (lp_j + H)
+                //                         + kl_coef (pi_j - pi_target_j) ] / M
+                const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = k.kl_coef * k.inv_M;
+                const float h_minus_lns = ent - ln_s;  // lp_j + H = d_j + (H - ln S)
+#pragma unroll
+                for (int j = 0; j < A; ++j) {
+                    const float pi = e[j] * inv_s;
+                    float gj = pi * fmaf(ce, d[j] + h_minus_lns, w1);
+                    gj -= (j == a) ? w1 : 0.0f;
+                    e[j] = gj;
+                }
+                if (want_kl) {
+                    float zr[A];
+                    RowIO<LT, A>::load(s1, tid, zr);
+#pragma unroll
+                    for (int j = 0; j < A; ++j) {
+                        const float pt = dev::exp2_fast((zr[j] - lse_t) * kLog2e);
+                        // e[j] holds the gradient so far; pi_j is recovered from d_j
+                        const float pi = dev::exp2_fast(d[j] * kLog2e) * inv_s;
+                        e[j] = fmaf(ck, pi - pt, e[j]);
+                    }
+                }
+                p.dvalues[row] = -k.vf_coef * k.inv_M * adv;  // V - Vhat = -A
+                if (p.vtarget) p.vtarget[row] = s.value + adv;
+                if (p.advantage) p.advantage[row] = adv;
+                sums[0] = surr;
+                sums[1] = 0.5f * adv * adv;
+                sums[2] = ent;
+                sums[3] = kl;
+                sums[4] = clipped ? 1.0f : 0.0f;
+                sums[5] = truncated ? 1.0f : 0.0f;
+                sums[6] = ratio;
+            }
+            // every thread has its rows in registers (the scan's barrier is behind us), so the
+            // learner slab can be overwritten with the gradient slab
+            if (active) RowIO<GT, A>::store(s0, tid, e);
+            dev::block_sums_stage1<NT>(sums, red);
+            if (bulk_out) dev::fence_async_shared();
+            __syncthreads();
+            carry = carry_s;
+            if (bulk_out) {
+                if (tid == 0) dev::bulk_store(gd, s0, out_bytes);
+            } else {
+                const int nelem = tr.nrows * A;
+                for (int i = tid; i < nelem; i += NT) gd[i] = reinterpret_cast<const GT*>(s0)[i];
+            }
+            dev::block_sums_stage2<NT>(acc, red);
+            if (bulk_out && tid == 0) dev::bulk_store_wait_read();
+            __syncthreads();  // slabs, sums and carry are free for the next tile
+        }
+    }
+    dev::finish_loss_terms<NT>(acc, p.partials, p.counter, p.loss_terms, k,
+                               (double)g.B * (double)g.T);
+}
+
+// ------------------------------------------------------------------------------------------
 // Diagonal-Gaussian policy
 // ------------------------------------------------------------------------------------------
 template <int NT>
@@ -461,6 +750,52 @@ int32_t dispatch_nt(const CatParams& p, int nt, const DeviceInfo* di, cudaStream
     }
 }
 
+template <typename LT, typename GT, int A>
+int32_t launch_categorical_reg(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
+    auto kernel = impact_loss_categorical_reg_kernel<LT, GT, A>;
+    const size_t smem = reg_kernel_smem<LT, GT, A>();
+    int grid = 0;
+    int32_t st = grid_for(kernel, kRegTileRows, smem, p.geo.nchunks, di, &grid);
+    if (st != IMPACT_OK) return st;
+    kernel<<<grid, kRegTileRows, smem, stream>>>(p);
+    IMPACT_CUDA_TRY(cudaGetLastError());
+    return IMPACT_OK;
+}
+
+// Action counts with a compiled register-resident kernel (the Atari action sets).
+constexpr bool has_reg_kernel(int A) { return A == 4 || A == 6 || A == 9 || A == 18; }
+
+template <typename LT, typename GT>
+int32_t dispatch_reg(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
+    switch (p.A) {
+        case 4: return launch_categorical_reg<LT, GT, 4>(p, di, stream);
+        case 6: return launch_categorical_reg<LT, GT, 6>(p, di, stream);
+        case 9: return launch_categorical_reg<LT, GT, 9>(p, di, stream);
+        default: return launch_categorical_reg<LT, GT, 18>(p, di, stream);
+    }
+}
+
+// Picks the kernel for a categorical call: the register-resident one where it exists, else
+// the generic one.  `p` arrives complete except for As and geo.
+int32_t run_categorical(CatParams& p, int64_t B, int64_t T, bool logits_bf16, bool grads_bf16,
+                        const DeviceInfo* di, cudaStream_t s) {
+    if (has_reg_kernel(p.A)) {
+        p.As = p.A;
+        p.geo = make_geometry(B, T, kRegTileRows);
+        if (!logits_bf16 && !grads_bf16) return dispatch_reg<float, float>(p, di, s);
+        if (!logits_bf16 && grads_bf16) return dispatch_reg<float, __nv_bfloat16>(p, di, s);
+        if (logits_bf16 && !grads_bf16) return dispatch_reg<__nv_bfloat16, float>(p, di, s);
+        return dispatch_reg<__nv_bfloat16, __nv_bfloat16>(p, di, s);
+    }
+    p.As = pad_odd(p.A);
+    const int nt = pick_nt(p.As, 2, 72 * 1024);
+    p.geo = make_geometry(B, T, nt);
+    if (!logits_bf16 && !grads_bf16) return dispatch_nt<float, float>(p, nt, di, s);
+    if (!logits_bf16 && grads_bf16) return dispatch_nt<float, __nv_bfloat16>(p, nt, di, s);
+    if (logits_bf16 && !grads_bf16) return dispatch_nt<__nv_bfloat16, float>(p, nt, di, s);
+    return dispatch_nt<__nv_bfloat16, __nv_bfloat16>(p, nt, di, s);
+}
+
 template <int NT>
 int32_t launch_gaussian(const GaussParams& p, const DeviceInfo* di, cudaStream_t stream) {
     auto kernel = impact_loss_gaussian_kernel<NT>;
@@ -536,15 +871,8 @@ extern "C" int32_t impact_loss_fwd_bwd(
     p.counter = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) +
                                                 (size_t)kMaxGridBlocks * 8 * sizeof(float));
     p.A = A;
-    p.As = pad_odd(A);
-    const int nt = pick_nt(p.As, 2, 72 * 1024);
-    p.geo = make_geometry(B, T, nt);
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const bool lb = logits_dtype == IMPACT_DTYPE_BF16, gb = coef->dlogits_dtype == IMPACT_DTYPE_BF16;
-    if (!lb && !gb) return dispatch_nt<float, float>(p, nt, di, s);
-    if (!lb && gb) return dispatch_nt<float, __nv_bfloat16>(p, nt, di, s);
-    if (lb && !gb) return dispatch_nt<__nv_bfloat16, float>(p, nt, di, s);
-    return dispatch_nt<__nv_bfloat16, __nv_bfloat16>(p, nt, di, s);
+    return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
+                           di, static_cast<cudaStream_t>(stream));
 }
 
 extern "C" int32_t impact_loss_fwd_bwd_gaussian(
@@ -663,11 +991,9 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     int32_t st = fill_scalars(p.k, rho_bar, c_bar, clip_eps, coef, B, T);
     if (st != IMPACT_OK) return st;
     p.A = A;
-    p.As = pad_odd(A);
-    const int nt = pick_nt(p.As, 2, 72 * 1024);
-    p.geo = make_geometry(B, T, nt);
     // one block's sums per tile at most: more tiles than the built-in scratch holds are refused
-    if (nt != 128 || p.geo.nchunks > kStaticMaxBlocks) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
+    // (every kernel serving A <= 64 works on tiles of 128 steps)
+    if (make_geometry(B, T, 128).nchunks > kStaticMaxBlocks) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
 
     const DeviceInfo* di = current_device_info();
     if (!di) return IMPACT_ERR_CUDA;
@@ -694,9 +1020,7 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     p.advantage = advantage;
     p.partials = reinterpret_cast<float*>(scratch);
     p.counter = reinterpret_cast<unsigned int*>(counter);
-    const bool lb = logits_dtype == IMPACT_DTYPE_BF16, gb = coef->dlogits_dtype == IMPACT_DTYPE_BF16;
-    if (!lb && !gb) return dispatch_nt<float, float>(p, nt, di, s);
-    if (!lb && gb) return dispatch_nt<float, __nv_bfloat16>(p, nt, di, s);
-    if (lb && !gb) return dispatch_nt<__nv_bfloat16, float>(p, nt, di, s);
-    return dispatch_nt<__nv_bfloat16, __nv_bfloat16>(p, nt, di, s);
+    // the same kernels, chosen the same way, as impact_loss_fwd_bwd
+    return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
+                           di, s);
 }
