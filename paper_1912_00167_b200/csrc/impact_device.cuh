@@ -377,5 +377,86 @@ __device__ __forceinline__ void finish_loss_terms(const float (&acc)[kNumSums], 
     }
 }
 
+// ---- early publication of a block's sums ---------------------------------------------------
+// Thread 0 calls this as soon as its block's last sums are final, long before the block's
+// stores are done: the fence and the counter's round trip then overlap the rest of the
+// block's work instead of extending it.  Returns the block's ticket (0-based arrival order).
+__device__ __forceinline__ unsigned int publish_block_sums(const float (&acc)[kNumSums], float* partials,
+                                                           unsigned int* counter) {
+    float4* row = reinterpret_cast<float4*>(partials + (size_t)blockIdx.x * 8);
+    row[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
+    row[1] = make_float4(acc[4], acc[5], acc[6], 0.0f);
+    __threadfence();
+    return atomicAdd(counter, 1u);
+}
+
+// Run by every thread of the block that drew the last ticket: add all blocks' sums in index
+// order (fp64), write the eight loss terms, and leave the counter at 0 for the next launch.
+template <int NT>
+__device__ __forceinline__ void reduce_published_sums(const float* partials, unsigned int* counter,
+                                                      float* loss_terms, const LossScalars& k, double M) {
+    __shared__ double dred[NT / 32][kNumSums];
+    __threadfence();
+    double s[kNumSums];
+#pragma unroll
+    for (int j = 0; j < kNumSums; ++j) s[j] = 0.0;
+    for (unsigned int blk = threadIdx.x; blk < gridDim.x; blk += NT) {
+        const float4 p0 = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)blk * 8));
+        const float4 p1 = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)blk * 8 + 4));
+        s[0] += p0.x; s[1] += p0.y; s[2] += p0.z; s[3] += p0.w;
+        s[4] += p1.x; s[5] += p1.y; s[6] += p1.z;
+    }
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+#pragma unroll
+    for (int j = 0; j < kNumSums; ++j) {
+        double x = s[j];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+        if (lane == 0) dred[warp][j] = x;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const double inv_m = 1.0 / M;
+        double t[kNumSums];
+#pragma unroll
+        for (int j = 0; j < kNumSums; ++j) {
+            double x = 0.0;
+            for (int w = 0; w < NT / 32; ++w) x += dred[w][j];
+            t[j] = x * inv_m;
+        }
+        const double l_pi = -t[0], l_v = t[1], ent = t[2], kl = t[3];
+        loss_terms[0] = (float)(l_pi + (double)k.vf_coef * l_v - (double)k.ent_coef * ent +
+                                (double)k.kl_coef * kl);
+        loss_terms[1] = (float)l_pi;
+        loss_terms[2] = (float)l_v;
+        loss_terms[3] = (float)ent;
+        loss_terms[4] = (float)kl;
+        loss_terms[5] = (float)t[4];
+        loss_terms[6] = (float)t[5];
+        loss_terms[7] = (float)t[6];
+        *counter = 0u;
+    }
+}
+
+// Block sums when two of the seven are counts of a per-thread flag: five float sums by
+// shuffles, the two counts by one ballot each.
+template <int NT>
+__device__ __forceinline__ void block_sums_stage1_flags(const float (&v)[5], bool f0, bool f1, float (*red)[8]) {
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    float x[5];
+#pragma unroll
+    for (int j = 0; j < 5; ++j) x[j] = v[j];
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) {
+#pragma unroll
+        for (int j = 0; j < 5; ++j) x[j] += __shfl_xor_sync(0xffffffffu, x[j], off);
+    }
+    const unsigned int b0 = __ballot_sync(0xffffffffu, f0), b1 = __ballot_sync(0xffffffffu, f1);
+    if (lane == 0) {
+        red[warp][0] = x[0]; red[warp][1] = x[1]; red[warp][2] = x[2]; red[warp][3] = x[3];
+        red[warp][4] = (float)__popc(b0); red[warp][5] = (float)__popc(b1); red[warp][6] = x[4];
+    }
+}
+
 }  // namespace dev
 }  // namespace impact

@@ -243,99 +243,147 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
 // a B*T = 131072 batch are all resident at once on 148 SMs and every load is issued up front.
 template <typename ST, int W> struct RowIO;
 
+// Rows are handled as NP = ceil(W/2) pairs; for odd W the second lane of the last pair is
+// padding (loaded as 0, never stored).
 template <int W> struct RowIO<float, W> {
-    static constexpr int VW = (W % 4 == 0) ? 4 : ((W % 2 == 0) ? 2 : 1);
-    static __device__ __forceinline__ void load(const unsigned char* slab, int row, float (&z)[W]) {
+    static constexpr int NP = (W + 1) / 2;
+    static __device__ __forceinline__ void load(const unsigned char* slab, int row, float2 (&v)[NP]) {
         const float* r = reinterpret_cast<const float*>(slab) + row * W;
-        if constexpr (VW == 4) {
+        if constexpr (W % 4 == 0) {
 #pragma unroll
             for (int j = 0; j < W / 4; ++j) {
-                const float4 v = reinterpret_cast<const float4*>(r)[j];
-                z[4 * j] = v.x; z[4 * j + 1] = v.y; z[4 * j + 2] = v.z; z[4 * j + 3] = v.w;
+                const float4 q = reinterpret_cast<const float4*>(r)[j];
+                v[2 * j] = make_float2(q.x, q.y);
+                v[2 * j + 1] = make_float2(q.z, q.w);
             }
-        } else if constexpr (VW == 2) {
+        } else if constexpr (W % 2 == 0) {
 #pragma unroll
-            for (int j = 0; j < W / 2; ++j) {
-                const float2 v = reinterpret_cast<const float2*>(r)[j];
-                z[2 * j] = v.x; z[2 * j + 1] = v.y;
-            }
+            for (int j = 0; j < W / 2; ++j) v[j] = reinterpret_cast<const float2*>(r)[j];
         } else {
 #pragma unroll
-            for (int j = 0; j < W; ++j) z[j] = r[j];
+            for (int j = 0; j < W / 2; ++j) v[j] = make_float2(r[2 * j], r[2 * j + 1]);
+            v[NP - 1] = make_float2(r[W - 1], 0.0f);
         }
     }
-    static __device__ __forceinline__ void store(unsigned char* slab, int row, const float (&g)[W]) {
+    static __device__ __forceinline__ void store(unsigned char* slab, int row, const float2 (&v)[NP]) {
         float* r = reinterpret_cast<float*>(slab) + row * W;
-        if constexpr (VW == 4) {
+        if constexpr (W % 4 == 0) {
 #pragma unroll
             for (int j = 0; j < W / 4; ++j)
-                reinterpret_cast<float4*>(r)[j] = make_float4(g[4 * j], g[4 * j + 1], g[4 * j + 2], g[4 * j + 3]);
-        } else if constexpr (VW == 2) {
+                reinterpret_cast<float4*>(r)[j] = make_float4(v[2 * j].x, v[2 * j].y, v[2 * j + 1].x, v[2 * j + 1].y);
+        } else if constexpr (W % 2 == 0) {
 #pragma unroll
-            for (int j = 0; j < W / 2; ++j) reinterpret_cast<float2*>(r)[j] = make_float2(g[2 * j], g[2 * j + 1]);
+            for (int j = 0; j < W / 2; ++j) reinterpret_cast<float2*>(r)[j] = v[j];
         } else {
 #pragma unroll
-            for (int j = 0; j < W; ++j) r[j] = g[j];
+            for (int j = 0; j < W / 2; ++j) { r[2 * j] = v[j].x; r[2 * j + 1] = v[j].y; }
+            r[W - 1] = v[NP - 1].x;
         }
     }
     static __device__ __forceinline__ float at(const unsigned char* slab, int row, int col) {
         return reinterpret_cast<const float*>(slab)[row * W + col];
     }
+    // Overwrites one element after `store` wrote the row; an explicit shared-memory store
+    // keeps it ordered behind the vector stores to the same bytes.
+    static __device__ __forceinline__ void put(unsigned char* slab, int row, int col, float x) {
+        asm volatile("st.shared.f32 [%0], %1;" ::"r"(dev::smem_addr(slab) + (uint32_t)(row * W + col) * 4u), "f"(x)
+                     : "memory");
+    }
 };
 
 template <int W> struct RowIO<__nv_bfloat16, W> {
-    static __device__ __forceinline__ void load(const unsigned char* slab, int row, float (&z)[W]) {
+    static constexpr int NP = (W + 1) / 2;
+    static __device__ __forceinline__ float widen(unsigned short h) { return __uint_as_float((uint32_t)h << 16); }
+    static __device__ __forceinline__ void load(const unsigned char* slab, int row, float2 (&v)[NP]) {
         if constexpr (W % 2 == 0) {
             const uint32_t* r = reinterpret_cast<const uint32_t*>(slab) + row * (W / 2);
 #pragma unroll
             for (int j = 0; j < W / 2; ++j) {
                 const uint32_t w = r[j];
-                z[2 * j] = __uint_as_float(w << 16);
-                z[2 * j + 1] = __uint_as_float(w & 0xFFFF0000u);
+                v[j] = make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
             }
         } else {
             const unsigned short* r = reinterpret_cast<const unsigned short*>(slab) + row * W;
 #pragma unroll
-            for (int j = 0; j < W; ++j) z[j] = __uint_as_float((uint32_t)r[j] << 16);
+            for (int j = 0; j < W / 2; ++j) v[j] = make_float2(widen(r[2 * j]), widen(r[2 * j + 1]));
+            v[NP - 1] = make_float2(widen(r[W - 1]), 0.0f);
         }
     }
-    static __device__ __forceinline__ void store(unsigned char* slab, int row, const float (&g)[W]) {
+    static __device__ __forceinline__ void store(unsigned char* slab, int row, const float2 (&v)[NP]) {
         if constexpr (W % 2 == 0) {
             uint32_t* r = reinterpret_cast<uint32_t*>(slab) + row * (W / 2);
 #pragma unroll
-            for (int j = 0; j < W / 2; ++j) r[j] = dev::Pack<__nv_bfloat16>::two(g[2 * j], g[2 * j + 1]);
+            for (int j = 0; j < W / 2; ++j) r[j] = dev::Pack<__nv_bfloat16>::two(v[j].x, v[j].y);
         } else {
             __nv_bfloat16* r = reinterpret_cast<__nv_bfloat16*>(slab) + row * W;
 #pragma unroll
-            for (int j = 0; j < W; ++j) r[j] = __float2bfloat16_rn(g[j]);
+            for (int j = 0; j < W / 2; ++j) {
+                r[2 * j] = __float2bfloat16_rn(v[j].x);
+                r[2 * j + 1] = __float2bfloat16_rn(v[j].y);
+            }
+            r[W - 1] = __float2bfloat16_rn(v[NP - 1].x);
         }
     }
     static __device__ __forceinline__ float at(const unsigned char* slab, int row, int col) {
-        return __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(slab)[row * W + col] << 16);
+        return widen(reinterpret_cast<const unsigned short*>(slab)[row * W + col]);
+    }
+    static __device__ __forceinline__ void put(unsigned char* slab, int row, int col, float x) {
+        const unsigned short h = __bfloat16_as_ushort(__float2bfloat16_rn(x));
+        asm volatile("st.shared.u16 [%0], %1;" ::"r"(dev::smem_addr(slab) + (uint32_t)(row * W + col) * 2u), "h"(h)
+                     : "memory");
     }
 };
 
 constexpr int kRegTileRows = 128;
 
+// Shared memory of the register-resident kernel: the two input slabs, plus a separate
+// gradient slab only when gradients and logits differ in element size (otherwise each
+// thread's gradient row replaces its own logits row).
 template <typename LT, typename GT, int A>
 constexpr size_t reg_kernel_smem() {
     constexpr size_t in_row = A * sizeof(LT), out_row = A * sizeof(GT);
-    return kRegTileRows * ((in_row > out_row ? in_row : out_row) + in_row);
+    return kRegTileRows * (2 * in_row + (sizeof(LT) == sizeof(GT) ? 0 : out_row));
+}
+
+// A row of A logits in registers, as pairs: Blackwell's packed fp32 instructions (two lanes
+// per instruction for add, mul and fma) halve the arithmetic issue slots of the row passes.
+// Odd A carries its last element in a pair whose second lane is padding.
+template <int A> struct RowRegs {
+    static constexpr int NP = (A + 1) / 2;
+    float2 v[NP];
+    __device__ __forceinline__ float get(int j) const { return (j & 1) ? v[j >> 1].y : v[j >> 1].x; }
+};
+
+template <typename ST, int A>
+__device__ __forceinline__ void load_row_pairs(const unsigned char* slab, int row, RowRegs<A>& r) {
+    RowIO<ST, A>::load(slab, row, r.v);
+}
+
+template <int A>
+__device__ __forceinline__ float row_max(const RowRegs<A>& r) {
+    float m = r.v[0].x;
+#pragma unroll
+    for (int j = 1; j < A; ++j) m = fmaxf(m, r.get(j));
+    return m;
 }
 
 template <typename LT, typename GT, int A>
 __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_kernel(const CatParams p) {
     constexpr int NT = kRegTileRows;
+    constexpr int NP = RowRegs<A>::NP;
+    constexpr bool kOdd = (A & 1) != 0;
     constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
-    constexpr int kRegion0 = NT * (kInRow > kOutRow ? kInRow : kOutRow);
     constexpr float kLog2e = 1.4426950408889634f;
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* const s0 = smem_raw;             // learner logits in, gradients out
-    unsigned char* const s1 = smem_raw + kRegion0;  // target logits
+    unsigned char* const s0 = smem_raw;                // learner logits
+    unsigned char* const s1 = smem_raw + NT * kInRow;  // target logits
+    // gradient rows: over the thread's own logits row when the element sizes agree
+    unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : smem_raw + 2 * NT * kInRow;
     __shared__ __align__(8) uint64_t bar;
     __shared__ float2 warp_agg[NT / 32];
     __shared__ float red[NT / 32][8];
     __shared__ float carry_s;
+    __shared__ int is_last_s;
 
     const int tid = threadIdx.x;
     const LossScalars k = p.k;
@@ -344,8 +392,12 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
     const LT* const zt = static_cast<const LT*>(p.target_logits);
     GT* const dz = static_cast<GT*>(p.dlogits);
     const bool want_kl = (k.kl_coef != 0.0f);
+    const float2 log2e2 = make_float2(kLog2e, kLog2e);
 
-    if (tid == 0) dev::mbarrier_init(&bar, 1);
+    if (tid == 0) {
+        dev::mbarrier_init(&bar, 1);
+        is_last_s = 0;
+    }
     __syncthreads();
     uint32_t parity = 0;
 
@@ -356,6 +408,7 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
     for (long long chunk = blockIdx.x; chunk < g.nchunks; chunk += gridDim.x) {
         float carry = 0.0f;
         for (int tile = g.ntiles - 1; tile >= 0; --tile) {
+            const bool final_tile = (tile == 0) && (chunk + gridDim.x >= g.nchunks);
             const TileRows tr = tile_rows<NT>(g, chunk, tile);
             const long long base = tr.row0 * A;
             const LT* const gl = zl + base;
@@ -364,8 +417,8 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
             const uint32_t in_bytes = (uint32_t)tr.nrows * kInRow, out_bytes = (uint32_t)tr.nrows * kOutRow;
             const bool bulk_in = (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | in_bytes) & 15u) == 0);
             const bool bulk_out = (((reinterpret_cast<uintptr_t>(gd) | out_bytes) & 15u) == 0);
-            // shared memory is free here: the previous tile's rows were read into registers before
-            // its scan barrier, and its store was drained before the barrier that ended the tile
+            // shared memory is free here: the previous tile ended with a barrier, after its rows
+            // had been consumed and its gradient store had finished reading the slab
             if (bulk_in) {
                 if (tid == 0) {
                     dev::mbarrier_expect_tx(&bar, 2 * in_bytes);
@@ -407,45 +460,53 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
             }
 
             float fa = 1.0f, fb = 0.0f;
-            float d[A], e[A];  // learner row: z - max, and 2^((z - max) log2 e)
-            float ln_s = 0.0f, inv_s = 0.0f, lse_t = 0.0f, ent = 0.0f, kl = 0.0f;
+            RowRegs<A> e;  // learner row: exp(z - max); the row itself is re-read where needed
+            float m_l = 0.0f, ln_s = 0.0f, inv_s = 0.0f, lse_t = 0.0f, ent = 0.0f, kl = 0.0f;
             bool truncated = false;
             if (active) {
                 {   // target row: only its log-sum-exp and the taken action's logit are needed
-                    float zr[A];
-                    RowIO<LT, A>::load(s1, tid, zr);
-                    float m = zr[0];
+                    RowRegs<A> zr;
+                    load_row_pairs<LT, A>(s1, tid, zr);
+                    const float m = row_max<A>(zr);
+                    const float2 neg_m = make_float2(-m, -m);
+                    float2 sum2 = make_float2(0.0f, 0.0f);
 #pragma unroll
-                    for (int j = 1; j < A; ++j) m = fmaxf(m, zr[j]);
-                    float sum = 0.0f;
-#pragma unroll
-                    for (int j = 0; j < A; ++j) sum += dev::exp2_fast((zr[j] - m) * kLog2e);
-                    lse_t = m + logf(sum);
+                    for (int j = 0; j < NP; ++j) {
+                        const float2 t2 = __fmul2_rn(__fadd2_rn(zr.v[j], neg_m), log2e2);
+                        float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
+                        if (kOdd && j == NP - 1) ex.y = 0.0f;
+                        sum2 = __fadd2_rn(sum2, ex);
+                    }
+                    lse_t = m + logf(sum2.x + sum2.y);
                     s.l_target = RowIO<LT, A>::at(s1, tid, a) - lse_t;
                 }
-                RowIO<LT, A>::load(s0, tid, d);
-                float m = d[0];
+                RowRegs<A> d;
+                load_row_pairs<LT, A>(s0, tid, d);
+                const float m = row_max<A>(d);
+                m_l = m;
+                const float2 neg_m = make_float2(-m, -m);
+                float2 sum2 = make_float2(0.0f, 0.0f), sed2 = make_float2(0.0f, 0.0f);
 #pragma unroll
-                for (int j = 1; j < A; ++j) m = fmaxf(m, d[j]);
-                float sum = 0.0f, sed = 0.0f;
-#pragma unroll
-                for (int j = 0; j < A; ++j) {
-                    d[j] -= m;
-                    e[j] = dev::exp2_fast(d[j] * kLog2e);
-                    sum += e[j];
-                    sed = fmaf(e[j], d[j], sed);
+                for (int j = 0; j < NP; ++j) {
+                    d.v[j] = __fadd2_rn(d.v[j], neg_m);
+                    const float2 t2 = __fmul2_rn(d.v[j], log2e2);
+                    e.v[j] = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
+                    if (kOdd && j == NP - 1) { e.v[j].y = 0.0f; d.v[j].y = 0.0f; }
+                    sum2 = __fadd2_rn(sum2, e.v[j]);
+                    sed2 = __ffma2_rn(e.v[j], d.v[j], sed2);
                 }
+                const float sum = sum2.x + sum2.y;
                 ln_s = logf(sum);
                 inv_s = 1.0f / sum;
-                ent = ln_s - sed * inv_s;  // H = ln S - sum_j e_j (z_j - m) / S
+                ent = ln_s - (sed2.x + sed2.y) * inv_s;  // H = ln S - sum_j e_j (z_j - m) / S
                 s.l_theta = (RowIO<LT, A>::at(s0, tid, a) - m) - ln_s;
                 if (want_kl) {
-                    float zr[A];
-                    RowIO<LT, A>::load(s1, tid, zr);
+                    RowRegs<A> zr;
+                    load_row_pairs<LT, A>(s1, tid, zr);
 #pragma unroll
                     for (int j = 0; j < A; ++j) {
-                        const float lpt = zr[j] - lse_t;
-                        kl = fmaf(dev::exp2_fast(lpt * kLog2e), lpt - (d[j] - ln_s), kl);
+                        const float lpt = zr.get(j) - lse_t;
+                        kl = fmaf(dev::exp2_fast(lpt * kLog2e), lpt - (d.get(j) - ln_s), kl);
                     }
                 }
                 truncated = dev::recursion_map(s, k, fa, fb);
@@ -453,66 +514,77 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
             const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
             if (tid == 0) carry_s = adv;
 
-            float sums[dev::kNumSums];
-#pragma unroll
-            for (int j = 0; j < dev::kNumSums; ++j) sums[j] = 0.0f;
+            float surr = 0.0f, ratio = 0.0f, wpg = 0.0f;
+            bool clipped = false;
+            if (active) wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
+            {
+                const float sums5[5] = {surr, active ? 0.5f * adv * adv : 0.0f, ent, kl, ratio};
+                dev::block_sums_stage1_flags<NT>(sums5, clipped, truncated, red);
+            }
+            __syncthreads();
+            unsigned int ticket = 0;
+            if (tid == 0) {
+                dev::block_sums_stage2<NT>(acc, red);
+                // sums of the block's last tile: publish now, the round trip hides behind the epilogue
+                if (final_tile) ticket = dev::publish_block_sums(acc, p.partials, p.counter);
+            }
+
             if (active) {
-                float surr, ratio;
-                bool clipped;
-                const float wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
                 // d total / d logit_j = [ wpg (pi_j - 1[j=a]) + ent_coef pi_j (lp_j + H)
-                //                         + kl_coef (pi_j - pi_target_j) ] / M
+                //                         + kl_coef (pi_j - pi_target_j) ] / M,   lp_j + H = d_j + (H - ln S)
                 const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = k.kl_coef * k.inv_M;
-                const float h_minus_lns = ent - ln_s;  // lp_j + H = d_j + (H - ln S)
+                const float h_minus_lns = ent - ln_s;
+                const float2 inv_s2 = make_float2(inv_s, inv_s);
+                // lp_j + H = z_j + (H - ln S - max)
+                const float2 hml2 = make_float2(h_minus_lns - m_l, h_minus_lns - m_l);
+                const float2 ce2 = make_float2(ce, ce), w12 = make_float2(w1, w1);
+                RowRegs<A> d;  // the learner row again (still untouched in shared memory)
+                load_row_pairs<LT, A>(s0, tid, d);
 #pragma unroll
-                for (int j = 0; j < A; ++j) {
-                    const float pi = e[j] * inv_s;
-                    float gj = pi * fmaf(ce, d[j] + h_minus_lns, w1);
-                    gj -= (j == a) ? w1 : 0.0f;
-                    e[j] = gj;
+                for (int j = 0; j < NP; ++j) {
+                    const float2 pi2 = __fmul2_rn(e.v[j], inv_s2);
+                    e.v[j] = __fmul2_rn(pi2, __ffma2_rn(ce2, __fadd2_rn(d.v[j], hml2), w12));
                 }
+                // the taken action's entry, from its own log-probability
+                const float pi_a = dev::exp2_fast(s.l_theta * kLog2e);
+                float g_a = fmaf(pi_a, fmaf(ce, s.l_theta + ent, w1), -w1);
                 if (want_kl) {
-                    float zr[A];
-                    RowIO<LT, A>::load(s1, tid, zr);
+                    RowRegs<A> zr;
+                    load_row_pairs<LT, A>(s1, tid, zr);
+                    const float2 ck2 = make_float2(ck, ck), neg_lse_t = make_float2(-lse_t, -lse_t);
 #pragma unroll
-                    for (int j = 0; j < A; ++j) {
-                        const float pt = dev::exp2_fast((zr[j] - lse_t) * kLog2e);
-                        // e[j] holds the gradient so far; pi_j is recovered from d_j
-                        const float pi = dev::exp2_fast(d[j] * kLog2e) * inv_s;
-                        e[j] = fmaf(ck, pi - pt, e[j]);
+                    for (int j = 0; j < NP; ++j) {
+                        const float2 tt = __fmul2_rn(__fadd2_rn(zr.v[j], neg_lse_t), log2e2);
+                        const float2 pt = make_float2(dev::exp2_fast(tt.x), dev::exp2_fast(tt.y));
+                        const float2 tl = __fmul2_rn(__fadd2_rn(d.v[j], make_float2(-m_l, -m_l)), log2e2);
+                        const float2 pi2 = __fmul2_rn(make_float2(dev::exp2_fast(tl.x), dev::exp2_fast(tl.y)), inv_s2);
+                        e.v[j] = __ffma2_rn(ck2, __fadd2_rn(pi2, make_float2(-pt.x, -pt.y)), e.v[j]);
                     }
+                    g_a = fmaf(ck, pi_a - dev::exp2_fast(s.l_target * kLog2e), g_a);
                 }
                 p.dvalues[row] = -k.vf_coef * k.inv_M * adv;  // V - Vhat = -A
                 if (p.vtarget) p.vtarget[row] = s.value + adv;
                 if (p.advantage) p.advantage[row] = adv;
-                sums[0] = surr;
-                sums[1] = 0.5f * adv * adv;
-                sums[2] = ent;
-                sums[3] = kl;
-                sums[4] = clipped ? 1.0f : 0.0f;
-                sums[5] = truncated ? 1.0f : 0.0f;
-                sums[6] = ratio;
+                RowIO<GT, A>::store(so, tid, e.v);
+                RowIO<GT, A>::put(so, tid, a, g_a);
             }
-            // every thread has its rows in registers (the scan's barrier is behind us), so the
-            // learner slab can be overwritten with the gradient slab
-            if (active) RowIO<GT, A>::store(s0, tid, e);
-            dev::block_sums_stage1<NT>(sums, red);
             if (bulk_out) dev::fence_async_shared();
+            if (tid == 0 && final_tile) is_last_s = (ticket == gridDim.x - 1) ? 1 : 0;
             __syncthreads();
             carry = carry_s;
             if (bulk_out) {
-                if (tid == 0) dev::bulk_store(gd, s0, out_bytes);
+                if (tid == 0) {
+                    dev::bulk_store(gd, so, out_bytes);
+                    dev::bulk_store_wait_read();
+                }
             } else {
                 const int nelem = tr.nrows * A;
-                for (int i = tid; i < nelem; i += NT) gd[i] = reinterpret_cast<const GT*>(s0)[i];
+                for (int i = tid; i < nelem; i += NT) gd[i] = reinterpret_cast<const GT*>(so)[i];
             }
-            dev::block_sums_stage2<NT>(acc, red);
-            if (bulk_out && tid == 0) dev::bulk_store_wait_read();
-            __syncthreads();  // slabs, sums and carry are free for the next tile
+            if (!final_tile) __syncthreads();  // slabs, sums and carry are free for the next tile
         }
     }
-    dev::finish_loss_terms<NT>(acc, p.partials, p.counter, p.loss_terms, k,
-                               (double)g.B * (double)g.T);
+    if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k, (double)g.B * (double)g.T);
 }
 
 // ------------------------------------------------------------------------------------------
