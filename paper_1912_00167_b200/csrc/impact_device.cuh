@@ -88,14 +88,16 @@ __device__ __forceinline__ void mbarrier_expect_tx(uint64_t* bar, uint32_t bytes
 // bytes never arrive the caller gets `false` instead of a hang.
 __device__ __forceinline__ bool mbarrier_wait(uint64_t* bar, uint32_t parity) {
     const uint32_t addr = smem_addr(bar);
-    for (uint32_t tries = 0; tries < (1u << 22); ++tries) {
+    constexpr uint32_t kSuspendHintNs = 100000;  // each try may sleep this long: few tries, no busy spinning
+    for (uint32_t tries = 0; tries < (1u << 20); ++tries) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
+            : "=r"(done) : "r"(addr), "r"(parity), "r"(kSuspendHintNs) : "memory");
         if (done) return true;
+        __nanosleep(64);  // a failed try returns early on this part: back off instead of spinning
     }
     return false;
 }
@@ -266,9 +268,13 @@ struct StepIn {
 
 // Truncated importance weights and the affine map of the advantage recursion
 // (Section 2.2; Section 3.1).  Returns whether exp(x) exceeded rho_bar.
+// exp of a log-probability difference.  Arguments are a few units at most, where the
+// multiply-then-exp2 form stays within ~3e-7 relative of the correctly rounded result.
+__device__ __forceinline__ float exp_of_logratio(float x) { return exp2_fast(x * 1.4426950408889634f); }
+
 __device__ __forceinline__ bool recursion_map(const StepIn& s, const LossScalars& k, float& a, float& b) {
     const float x = (k.is_source ? s.l_theta : s.l_target) - s.l_worker;
-    const float w = expf(x);
+    const float w = exp_of_logratio(x);
     const float rho = fminf(k.rho_bar, w);
     const float c = fminf(k.c_bar, w);
     b = rho * (s.reward + s.discount * s.value_next - s.value);
@@ -284,7 +290,7 @@ __device__ __forceinline__ float surrogate(const StepIn& s, const LossScalars& k
     if (k.ratio_mode == 1) d = s.l_target;
     else if (k.ratio_mode == 2) d = s.l_worker;
     else d = fmaxf(s.l_target, s.l_worker - k.log_rho_tw);
-    const float R = expf(s.l_theta - d);
+    const float R = exp_of_logratio(s.l_theta - d);
     const float Rc = fminf(fmaxf(R, k.clip_lo), k.clip_hi);
     surr = fminf(R * adv, Rc * adv);
     clipped = (adv > 0.0f && R > k.clip_hi) || (adv < 0.0f && R < k.clip_lo);
@@ -386,25 +392,41 @@ __device__ __forceinline__ unsigned int publish_block_sums(const float (&acc)[kN
     float4* row = reinterpret_cast<float4*>(partials + (size_t)blockIdx.x * 8);
     row[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
     row[1] = make_float4(acc[4], acc[5], acc[6], 0.0f);
-    __threadfence();
+    // release the row, then draw the ticket (acq_rel: the last drawer also acquires all rows)
+    asm volatile("fence.acq_rel.gpu;" ::: "memory");
     return atomicAdd(counter, 1u);
 }
 
 // Run by every thread of the block that drew the last ticket: add all blocks' sums in index
 // order (fp64), write the eight loss terms, and leave the counter at 0 for the next launch.
 template <int NT>
-__device__ __forceinline__ void reduce_published_sums(const float* partials, unsigned int* counter,
+__device__ __noinline__ void reduce_published_sums(const float* partials, unsigned int* counter,
                                                       float* loss_terms, const LossScalars& k, double M) {
     __shared__ double dred[NT / 32][kNumSums];
-    __threadfence();
+    asm volatile("fence.acq_rel.gpu;" ::: "memory");
     double s[kNumSums];
 #pragma unroll
     for (int j = 0; j < kNumSums; ++j) s[j] = 0.0;
-    for (unsigned int blk = threadIdx.x; blk < gridDim.x; blk += NT) {
-        const float4 p0 = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)blk * 8));
-        const float4 p1 = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)blk * 8 + 4));
-        s[0] += p0.x; s[1] += p0.y; s[2] += p0.z; s[3] += p0.w;
-        s[4] += p1.x; s[5] += p1.y; s[6] += p1.z;
+    // rows in batches of eight per thread, all loads of a batch in flight together
+    constexpr int kBatch = 8;
+    for (unsigned int first = threadIdx.x; first < gridDim.x; first += NT * kBatch) {
+        float4 p0[kBatch], p1[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const unsigned int blk = first + u * NT;
+            if (blk < gridDim.x) {
+                p0[u] = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)blk * 8));
+                p1[u] = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)blk * 8 + 4));
+            } else {
+                p0[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                p1[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            s[0] += p0[u].x; s[1] += p0[u].y; s[2] += p0[u].z; s[3] += p0[u].w;
+            s[4] += p1[u].x; s[5] += p1[u].y; s[6] += p1[u].z;
+        }
     }
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll

@@ -181,6 +181,7 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
                 s.value = p.values[row];
                 s.last_step = (t == g.T - 1);
                 s.value_next = s.last_step ? p.bootstrap[b] : p.values[row + 1];
+                asm volatile("" ::: "memory");
                 truncated = dev::recursion_map(s, k, fa, fb);
             }
             const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
@@ -239,8 +240,8 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
 //     the action counts compiled here (pitch/width odd);
 //   * A is a template parameter, rows live in registers, every loop is unrolled;
 //   * the softmax runs on exp2 of pre-scaled differences (one multiply + one MUFU each).
-// With ~19 KB of shared memory and <= 72 registers, 7 blocks fit an SM, so the 1024 tiles of
-// a B*T = 131072 batch are all resident at once on 148 SMs and every load is issued up front.
+// Five blocks per SM (<= 102 registers, no spills) measured faster than seven at 72 registers
+// with spills, even though a B*T = 131072 batch then runs as two waves of blocks.
 template <typename ST, int W> struct RowIO;
 
 // Rows are handled as NP = ceil(W/2) pairs; for odd W the second lane of the last pair is
@@ -368,7 +369,7 @@ __device__ __forceinline__ float row_max(const RowRegs<A>& r) {
 }
 
 template <typename LT, typename GT, int A>
-__global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_kernel(const CatParams p) {
+__global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_kernel(const CatParams p) {
     constexpr int NT = kRegTileRows;
     constexpr int NP = RowRegs<A>::NP;
     constexpr bool kOdd = (A & 1) != 0;
@@ -441,6 +442,7 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
             if (active) {
                 long long b, t;
                 if (g.ntiles > 1) { b = chunk; t = (long long)tile * NT + tid; }
+                else if (g.G == 1) { b = chunk; t = tid; }
                 else { const int q = tid / (int)g.T; b = chunk * g.G + q; t = tid - q * (int)g.T; }
                 a = p.actions[row];
                 a = a < 0 ? 0 : (a >= A ? A - 1 : a);
@@ -453,62 +455,71 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
             }
 
             if (bulk_in) {
-                if (!dev::mbarrier_wait(&bar, parity)) atomicExch(p.counter + 1, 1u);
+                // one warp watches the mbarrier; the others sleep at the block barrier
+                if (tid < 32) {
+                    if (!dev::mbarrier_wait(&bar, parity)) atomicExch(p.counter + 1, 1u);
+                }
                 parity ^= 1u;
-            } else {
-                __syncthreads();
             }
+            __syncthreads();
 
             float fa = 1.0f, fb = 0.0f;
-            RowRegs<A> e;  // learner row: exp(z - max); the row itself is re-read where needed
-            float m_l = 0.0f, ln_s = 0.0f, inv_s = 0.0f, lse_t = 0.0f, ent = 0.0f, kl = 0.0f;
+            // Nothing row-sized stays in registers across the scan: the epilogue re-reads the
+            // learner row from shared memory and re-forms its exponentials (18 more MUFU ops are
+            // cheaper than 36 registers held across the barrier).
+            float m2_l = 0.0f, ln_s = 0.0f, inv_s = 0.0f, lse_t = 0.0f, ent = 0.0f, kl = 0.0f;
             bool truncated = false;
             if (active) {
                 {   // target row: only its log-sum-exp and the taken action's logit are needed
                     RowRegs<A> zr;
                     load_row_pairs<LT, A>(s1, tid, zr);
                     const float m = row_max<A>(zr);
-                    const float2 neg_m = make_float2(-m, -m);
+                    const float2 neg_m2 = make_float2(-m * kLog2e, -m * kLog2e);
                     float2 sum2 = make_float2(0.0f, 0.0f);
 #pragma unroll
                     for (int j = 0; j < NP; ++j) {
-                        const float2 t2 = __fmul2_rn(__fadd2_rn(zr.v[j], neg_m), log2e2);
+                        const float2 t2 = __ffma2_rn(zr.v[j], log2e2, neg_m2);  // (z - m) log2 e
                         float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
                         if (kOdd && j == NP - 1) ex.y = 0.0f;
                         sum2 = __fadd2_rn(sum2, ex);
                     }
-                    lse_t = m + logf(sum2.x + sum2.y);
+                    lse_t = m + __logf(sum2.x + sum2.y);
                     s.l_target = RowIO<LT, A>::at(s1, tid, a) - lse_t;
                 }
-                RowRegs<A> d;
-                load_row_pairs<LT, A>(s0, tid, d);
-                const float m = row_max<A>(d);
-                m_l = m;
-                const float2 neg_m = make_float2(-m, -m);
-                float2 sum2 = make_float2(0.0f, 0.0f), sed2 = make_float2(0.0f, 0.0f);
+                // keep the compiler from hoisting the next row's loads over this one's arithmetic:
+                // one row in registers at a time
+                asm volatile("" ::: "memory");
+                RowRegs<A> z;
+                load_row_pairs<LT, A>(s0, tid, z);
+                const float m = row_max<A>(z);
+                m2_l = m * kLog2e;
+                const float2 neg_m2 = make_float2(-m2_l, -m2_l);
+                float2 sum2 = make_float2(0.0f, 0.0f), sez2 = make_float2(0.0f, 0.0f);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
-                    d.v[j] = __fadd2_rn(d.v[j], neg_m);
-                    const float2 t2 = __fmul2_rn(d.v[j], log2e2);
-                    e.v[j] = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
-                    if (kOdd && j == NP - 1) { e.v[j].y = 0.0f; d.v[j].y = 0.0f; }
-                    sum2 = __fadd2_rn(sum2, e.v[j]);
-                    sed2 = __ffma2_rn(e.v[j], d.v[j], sed2);
+                    const float2 t2 = __ffma2_rn(z.v[j], log2e2, neg_m2);
+                    float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
+                    if (kOdd && j == NP - 1) ex.y = 0.0f;
+                    sum2 = __fadd2_rn(sum2, ex);
+                    sez2 = __ffma2_rn(ex, z.v[j], sez2);
                 }
                 const float sum = sum2.x + sum2.y;
-                ln_s = logf(sum);
-                inv_s = 1.0f / sum;
-                ent = ln_s - (sed2.x + sed2.y) * inv_s;  // H = ln S - sum_j e_j (z_j - m) / S
+                ln_s = __logf(sum);
+                inv_s = __frcp_rn(sum);
+                // H = -sum_j pi_j lp_j = (m + ln S) - sum_j e_j z_j / S
+                ent = (m + ln_s) - (sez2.x + sez2.y) * inv_s;
                 s.l_theta = (RowIO<LT, A>::at(s0, tid, a) - m) - ln_s;
                 if (want_kl) {
                     RowRegs<A> zr;
                     load_row_pairs<LT, A>(s1, tid, zr);
+                    const float lse_l = m + ln_s;
 #pragma unroll
                     for (int j = 0; j < A; ++j) {
                         const float lpt = zr.get(j) - lse_t;
-                        kl = fmaf(dev::exp2_fast(lpt * kLog2e), lpt - (d.get(j) - ln_s), kl);
+                        kl = fmaf(dev::exp2_fast(lpt * kLog2e), lpt - (z.get(j) - lse_l), kl);
                     }
                 }
+                asm volatile("" ::: "memory");
                 truncated = dev::recursion_map(s, k, fa, fb);
             }
             const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
@@ -531,19 +542,21 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
 
             if (active) {
                 // d total / d logit_j = [ wpg (pi_j - 1[j=a]) + ent_coef pi_j (lp_j + H)
-                //                         + kl_coef (pi_j - pi_target_j) ] / M,   lp_j + H = d_j + (H - ln S)
+                //                         + kl_coef (pi_j - pi_target_j) ] / M
+                // with pi_j = 2^(z_j log2 e - m log2 e) / S and lp_j + H = z_j + (H - m - ln S)
                 const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = k.kl_coef * k.inv_M;
-                const float h_minus_lns = ent - ln_s;
-                const float2 inv_s2 = make_float2(inv_s, inv_s);
-                // lp_j + H = z_j + (H - ln S - max)
-                const float2 hml2 = make_float2(h_minus_lns - m_l, h_minus_lns - m_l);
+                const float h_off = ent - (m2_l * 0.6931471805599453f + ln_s);
+                const float2 inv_s2 = make_float2(inv_s, inv_s), hoff2 = make_float2(h_off, h_off);
                 const float2 ce2 = make_float2(ce, ce), w12 = make_float2(w1, w1);
-                RowRegs<A> d;  // the learner row again (still untouched in shared memory)
-                load_row_pairs<LT, A>(s0, tid, d);
+                const float2 neg_m2 = make_float2(-m2_l, -m2_l);
+                RowRegs<A> z, gr;
+                load_row_pairs<LT, A>(s0, tid, z);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
-                    const float2 pi2 = __fmul2_rn(e.v[j], inv_s2);
-                    e.v[j] = __fmul2_rn(pi2, __ffma2_rn(ce2, __fadd2_rn(d.v[j], hml2), w12));
+                    const float2 t2 = __ffma2_rn(z.v[j], log2e2, neg_m2);
+                    const float2 pi2 = __fmul2_rn(make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y)), inv_s2);
+                    gr.v[j] = __fmul2_rn(pi2, __ffma2_rn(ce2, __fadd2_rn(z.v[j], hoff2), w12));
+                    if (want_kl) z.v[j] = pi2;  // keep pi_j for the KL term below
                 }
                 // the taken action's entry, from its own log-probability
                 const float pi_a = dev::exp2_fast(s.l_theta * kLog2e);
@@ -551,21 +564,20 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
                 if (want_kl) {
                     RowRegs<A> zr;
                     load_row_pairs<LT, A>(s1, tid, zr);
-                    const float2 ck2 = make_float2(ck, ck), neg_lse_t = make_float2(-lse_t, -lse_t);
+                    const float2 ck2 = make_float2(ck, ck);
+                    const float2 neg_lse_t2 = make_float2(-lse_t * kLog2e, -lse_t * kLog2e);
 #pragma unroll
                     for (int j = 0; j < NP; ++j) {
-                        const float2 tt = __fmul2_rn(__fadd2_rn(zr.v[j], neg_lse_t), log2e2);
-                        const float2 pt = make_float2(dev::exp2_fast(tt.x), dev::exp2_fast(tt.y));
-                        const float2 tl = __fmul2_rn(__fadd2_rn(d.v[j], make_float2(-m_l, -m_l)), log2e2);
-                        const float2 pi2 = __fmul2_rn(make_float2(dev::exp2_fast(tl.x), dev::exp2_fast(tl.y)), inv_s2);
-                        e.v[j] = __ffma2_rn(ck2, __fadd2_rn(pi2, make_float2(-pt.x, -pt.y)), e.v[j]);
+                        const float2 tt = __ffma2_rn(zr.v[j], log2e2, neg_lse_t2);
+                        const float2 npt = make_float2(-dev::exp2_fast(tt.x), -dev::exp2_fast(tt.y));
+                        gr.v[j] = __ffma2_rn(ck2, __fadd2_rn(z.v[j], npt), gr.v[j]);
                     }
                     g_a = fmaf(ck, pi_a - dev::exp2_fast(s.l_target * kLog2e), g_a);
                 }
                 p.dvalues[row] = -k.vf_coef * k.inv_M * adv;  // V - Vhat = -A
                 if (p.vtarget) p.vtarget[row] = s.value + adv;
                 if (p.advantage) p.advantage[row] = adv;
-                RowIO<GT, A>::store(so, tid, e.v);
+                RowIO<GT, A>::store(so, tid, gr.v);
                 RowIO<GT, A>::put(so, tid, a, g_a);
             }
             if (bulk_out) dev::fence_async_shared();
@@ -575,7 +587,7 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
             if (bulk_out) {
                 if (tid == 0) {
                     dev::bulk_store(gd, so, out_bytes);
-                    dev::bulk_store_wait_read();
+                    if (!final_tile) dev::bulk_store_wait_read();  // the last store drains at the very end
                 }
             } else {
                 const int nelem = tr.nrows * A;
@@ -585,6 +597,7 @@ __global__ void __launch_bounds__(kRegTileRows, 7) impact_loss_categorical_reg_k
         }
     }
     if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k, (double)g.B * (double)g.T);
+    if (tid == 0) dev::bulk_store_wait_read();  // shared memory must outlive the store's reads
 }
 
 // ------------------------------------------------------------------------------------------
@@ -670,6 +683,7 @@ __global__ void __launch_bounds__(NT) impact_loss_gaussian_kernel(const GaussPar
                 s.value = p.values[row];
                 s.last_step = (t == g.T - 1);
                 s.value_next = s.last_step ? p.bootstrap[b] : p.values[row + 1];
+                asm volatile("" ::: "memory");
                 truncated = dev::recursion_map(s, k, fa, fb);
             }
             const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
