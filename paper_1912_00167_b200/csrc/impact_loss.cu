@@ -337,13 +337,17 @@ template <int W> struct RowIO<__nv_bfloat16, W> {
 
 constexpr int kRegTileRows = 128;
 
-// Shared memory of the register-resident kernel: the two input slabs, plus a separate
-// gradient slab only when gradients and logits differ in element size (otherwise each
-// thread's gradient row replaces its own logits row).
+// Shared memory of the register-resident kernel, per pipeline stage: the two input slabs,
+// plus a separate gradient slab only when gradients and logits differ in element size
+// (otherwise each thread's gradient row replaces its own logits row).
 template <typename LT, typename GT, int A>
-constexpr size_t reg_kernel_smem() {
+__host__ __device__ constexpr size_t reg_kernel_stage_bytes() {
     constexpr size_t in_row = A * sizeof(LT), out_row = A * sizeof(GT);
     return kRegTileRows * (2 * in_row + (sizeof(LT) == sizeof(GT) ? 0 : out_row));
+}
+template <typename LT, typename GT, int A>
+constexpr size_t reg_kernel_smem() {
+    return 2 * reg_kernel_stage_bytes<LT, GT, A>();  // two stages
 }
 
 // A row of A logits in registers, as pairs: Blackwell's packed fp32 instructions (two lanes
@@ -374,13 +378,12 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
     constexpr int NP = RowRegs<A>::NP;
     constexpr bool kOdd = (A & 1) != 0;
     constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
+    constexpr int kStageBytes = (int)reg_kernel_stage_bytes<LT, GT, A>();
     constexpr float kLog2e = 1.4426950408889634f;
+    // Two stages of slabs: while a tile is being worked on, the block's next tile is already
+    // streaming into the other stage (slabs by bulk copy, per-step scalars into registers).
     extern __shared__ __align__(128) unsigned char smem_raw[];
-    unsigned char* const s0 = smem_raw;                // learner logits
-    unsigned char* const s1 = smem_raw + NT * kInRow;  // target logits
-    // gradient rows: over the thread's own logits row when the element sizes agree
-    unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : smem_raw + 2 * NT * kInRow;
-    __shared__ __align__(8) uint64_t bar;
+    __shared__ __align__(8) uint64_t bar[2];
     __shared__ float2 warp_agg[NT / 32];
     __shared__ float red[NT / 32][8];
     __shared__ float carry_s;
@@ -396,70 +399,132 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
     const float2 log2e2 = make_float2(kLog2e, kLog2e);
 
     if (tid == 0) {
-        dev::mbarrier_init(&bar, 1);
+        dev::mbarrier_init(&bar[0], 1);
+        dev::mbarrier_init(&bar[1], 1);
         is_last_s = 0;
     }
     __syncthreads();
-    uint32_t parity = 0;
+
+    // This block's work: chunks blockIdx.x, blockIdx.x + gridDim.x, ...; within a chunk the tiles
+    // of a long trajectory from the last one backwards.  Iteration `it` of the block is
+    // (chunk, tile) = (blockIdx.x + (it / ntiles) * gridDim.x, ntiles - 1 - it % ntiles).
+    const long long n_iter = ((g.nchunks - blockIdx.x + gridDim.x - 1) / gridDim.x) * g.ntiles;
+
+    struct Tile {
+        long long chunk, row0;
+        int tile, nrows;
+        bool bulk_in;
+    };
+    auto tile_of = [&](long long it) {
+        Tile t;
+        const long long ci = it / g.ntiles;
+        t.chunk = blockIdx.x + ci * gridDim.x;
+        t.tile = g.ntiles - 1 - (int)(it - ci * g.ntiles);
+        const TileRows tr = tile_rows<NT>(g, t.chunk, t.tile);
+        t.row0 = tr.row0;
+        t.nrows = tr.nrows;
+        const uintptr_t a0 = reinterpret_cast<uintptr_t>(zl + tr.row0 * A), a1 = reinterpret_cast<uintptr_t>(zt + tr.row0 * A);
+        t.bulk_in = (((a0 | a1 | (uintptr_t)(tr.nrows * kInRow)) & 15u) == 0);
+        return t;
+    };
+    // Start the slab copies of a tile into a stage (whose previous contents are no longer needed).
+    auto fill_stage = [&](const Tile& t, int stage) {
+        unsigned char* const d0 = smem_raw + stage * kStageBytes;
+        unsigned char* const d1 = d0 + NT * kInRow;
+        const LT* const gl = zl + t.row0 * A;
+        const LT* const gt = zt + t.row0 * A;
+        if (t.bulk_in) {
+            if (tid == 0) {
+                const uint32_t bytes = (uint32_t)t.nrows * kInRow;
+                dev::mbarrier_expect_tx(&bar[stage], 2 * bytes);
+                dev::bulk_load(d0, gl, bytes, &bar[stage]);
+                dev::bulk_load(d1, gt, bytes, &bar[stage]);
+            }
+        } else {  // ragged or unaligned slab: plain element copies
+            const int nelem = t.nrows * A;
+            for (int e = tid; e < nelem; e += NT) {
+                reinterpret_cast<LT*>(d0)[e] = gl[e];
+                reinterpret_cast<LT*>(d1)[e] = gt[e];
+            }
+        }
+    };
+    // Per-step scalars of a tile, straight from global memory (coalesced).
+    struct StepRaw {
+        int a;
+        float l_worker, reward, discount, value, value_next;
+        bool last_step;
+    };
+    auto load_scalars = [&](const Tile& t) {
+        StepRaw r;
+        r.a = 0; r.l_worker = 0.f; r.reward = 0.f; r.discount = 0.f; r.value = 0.f; r.value_next = 0.f;
+        r.last_step = false;
+        if (tid < t.nrows) {
+            const long long row = t.row0 + tid;
+            long long b, ts;
+            if (g.ntiles > 1) { b = t.chunk; ts = (long long)t.tile * NT + tid; }
+            else if (g.G == 1) { b = t.chunk; ts = tid; }
+            else { const int q = tid / (int)g.T; b = t.chunk * g.G + q; ts = tid - q * (int)g.T; }
+            int a = p.actions[row];
+            r.a = a < 0 ? 0 : (a >= A ? A - 1 : a);
+            r.l_worker = p.worker_logp[row];
+            r.reward = p.rewards[row];
+            r.discount = p.discounts[row];
+            r.value = p.values[row];
+            r.last_step = (ts == g.T - 1);
+            r.value_next = r.last_step ? p.bootstrap[b] : p.values[row + 1];
+        }
+        return r;
+    };
 
     float acc[dev::kNumSums];
 #pragma unroll
     for (int j = 0; j < dev::kNumSums; ++j) acc[j] = 0.0f;
 
-    for (long long chunk = blockIdx.x; chunk < g.nchunks; chunk += gridDim.x) {
-        float carry = 0.0f;
-        for (int tile = g.ntiles - 1; tile >= 0; --tile) {
-            const bool final_tile = (tile == 0) && (chunk + gridDim.x >= g.nchunks);
-            const TileRows tr = tile_rows<NT>(g, chunk, tile);
-            const long long base = tr.row0 * A;
-            const LT* const gl = zl + base;
-            const LT* const gt = zt + base;
-            GT* const gd = dz + base;
-            const uint32_t in_bytes = (uint32_t)tr.nrows * kInRow, out_bytes = (uint32_t)tr.nrows * kOutRow;
-            const bool bulk_in = (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | in_bytes) & 15u) == 0);
+    Tile cur_tile = tile_of(0);
+    fill_stage(cur_tile, 0);
+    StepRaw cur = load_scalars(cur_tile);
+    uint32_t parity_bits = 0;  // bit s: phase parity the next wait on bar[s] expects
+    float carry = 0.0f;
+
+    for (long long it = 0; it < n_iter; ++it) {
+        {
+            const int stage = (int)(it & 1);
+            const bool final_tile = (it + 1 == n_iter);
+            const Tile tl = cur_tile;
+            if (tl.tile == g.ntiles - 1) carry = 0.0f;  // a new trajectory starts (from its end)
+            // prefetch: the other stage was released by the barrier that ended the previous tile
+            Tile next_tile = tl;
+            StepRaw nxt = cur;
+            if (!final_tile) {
+                next_tile = tile_of(it + 1);
+                fill_stage(next_tile, stage ^ 1);
+                nxt = load_scalars(next_tile);
+            }
+
+            unsigned char* const s0 = smem_raw + stage * kStageBytes;  // learner logits
+            unsigned char* const s1 = s0 + NT * kInRow;                // target logits
+            // gradient rows: over the thread's own logits row when the element sizes agree
+            unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : s0 + 2 * NT * kInRow;
+            GT* const gd = dz + tl.row0 * A;
+            const uint32_t out_bytes = (uint32_t)tl.nrows * kOutRow;
             const bool bulk_out = (((reinterpret_cast<uintptr_t>(gd) | out_bytes) & 15u) == 0);
-            // shared memory is free here: the previous tile ended with a barrier, after its rows
-            // had been consumed and its gradient store had finished reading the slab
-            if (bulk_in) {
-                if (tid == 0) {
-                    dev::mbarrier_expect_tx(&bar, 2 * in_bytes);
-                    dev::bulk_load(s0, gl, in_bytes, &bar);
-                    dev::bulk_load(s1, gt, in_bytes, &bar);
-                }
-            } else {  // ragged or unaligned slab: plain element copies
-                const int nelem = tr.nrows * A;
-                for (int e = tid; e < nelem; e += NT) {
-                    reinterpret_cast<LT*>(s0)[e] = gl[e];
-                    reinterpret_cast<LT*>(s1)[e] = gt[e];
-                }
-            }
-
-            // per-step scalars straight from global memory (coalesced), in flight with the slabs
-            const bool active = tid < tr.nrows;
-            const long long row = tr.row0 + tid;
+            const bool active = tid < tl.nrows;
+            const long long row = tl.row0 + tid;
+            const int a = cur.a;
             dev::StepIn s;
-            int a = 0;
-            if (active) {
-                long long b, t;
-                if (g.ntiles > 1) { b = chunk; t = (long long)tile * NT + tid; }
-                else if (g.G == 1) { b = chunk; t = tid; }
-                else { const int q = tid / (int)g.T; b = chunk * g.G + q; t = tid - q * (int)g.T; }
-                a = p.actions[row];
-                a = a < 0 ? 0 : (a >= A ? A - 1 : a);
-                s.l_worker = p.worker_logp[row];
-                s.reward = p.rewards[row];
-                s.discount = p.discounts[row];
-                s.value = p.values[row];
-                s.last_step = (t == g.T - 1);
-                s.value_next = s.last_step ? p.bootstrap[b] : p.values[row + 1];
-            }
+            s.l_worker = cur.l_worker;
+            s.reward = cur.reward;
+            s.discount = cur.discount;
+            s.value = cur.value;
+            s.value_next = cur.value_next;
+            s.last_step = cur.last_step;
 
-            if (bulk_in) {
+            if (tl.bulk_in) {
                 // one warp watches the mbarrier; the others sleep at the block barrier
                 if (tid < 32) {
-                    if (!dev::mbarrier_wait(&bar, parity)) atomicExch(p.counter + 1, 1u);
+                    if (!dev::mbarrier_wait(&bar[stage], (parity_bits >> stage) & 1u)) atomicExch(p.counter + 1, 1u);
                 }
-                parity ^= 1u;
+                parity_bits ^= (1u << stage);
             }
             __syncthreads();
 
@@ -590,10 +655,12 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
                     if (!final_tile) dev::bulk_store_wait_read();  // the last store drains at the very end
                 }
             } else {
-                const int nelem = tr.nrows * A;
+                const int nelem = tl.nrows * A;
                 for (int i = tid; i < nelem; i += NT) gd[i] = reinterpret_cast<const GT*>(so)[i];
             }
-            if (!final_tile) __syncthreads();  // slabs, sums and carry are free for the next tile
+            if (!final_tile) __syncthreads();  // this stage, the sums and the carry are free again
+            cur_tile = next_tile;
+            cur = nxt;
         }
     }
     if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k, (double)g.B * (double)g.T);
