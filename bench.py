@@ -38,6 +38,9 @@ FALLBACK_HBM_GBS = 6650.0
 FIELD_NAMES = ["actions", "rewards", "discounts", "worker_logp", "target_logits"]
 N_DISTINCT = 4    # distinct synthetic batches generated on the host
 N_SETS = 16       # rotating learner-output / gradient buffer sets (footprint beyond L2)
+# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel, from the ncu capture
+# summarised under profiles/ (None while the kernel has changed since the counters were taken)
+NCU_TRAFFIC_BYTES = None
 
 
 def algorithmic_bytes_per_step(A: int, logits_bytes: int = 4, grad_bytes: int = 4) -> int:
@@ -202,18 +205,23 @@ def main():
     out_sets = [dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
                      dvalues=torch.empty(B, T, device="cuda")) for _ in range(N_SETS)]
     workspace = ip.new_workspace(B, T)
+    workspace2 = ip.new_workspace(B, T)  # for launches that overlap the first stream's
     field_bytes = [t.numel() * t.element_size() for t in worker_batches[0]]
     ring = ip.ImpactBuffer(N, K, field_bytes, seed=cfg.seed)
     stream = torch.cuda.current_stream()
+    stream_id = stream.cuda_stream
 
     # one prepared loss call per slot: the slot's fields in place, learner outputs / gradients of set slot % N_SETS
-    calls = []
-    proto = worker_batches[0]
-    for s in range(N):
-        v = [ring.slot_view(s, f, proto[f].dtype, proto[f].shape) for f in range(len(FIELD_NAMES))]
-        ls, os_ = learner_sets[s % N_SETS], out_sets[s % N_SETS]
-        calls.append(ip.prepare_loss_fwd_bwd(ls["learner_logits"], v[4], v[3], v[0], v[1], v[2], ls["values"],
-                                             ls["bootstrap_values"], coef, workspace=workspace, **os_))
+    def prepared(ws):
+        out = []
+        proto = worker_batches[0]
+        for s in range(N):
+            v = [ring.slot_view(s, f, proto[f].dtype, proto[f].shape) for f in range(len(FIELD_NAMES))]
+            ls, os_ = learner_sets[s % N_SETS], out_sets[s % N_SETS]
+            out.append(ip.prepare_loss_fwd_bwd(ls["learner_logits"], v[4], v[3], v[0], v[1], v[2], ls["values"],
+                                               ls["bootstrap_values"], coef, workspace=ws, **os_))
+        return out
+    calls, calls2 = prepared(workspace), prepared(workspace2)
 
     counters = {"loss": 0, "copy": 0, "pushed": 0}
     slot_batch = [0] * N  # which synthetic worker batch sits in each slot
@@ -222,26 +230,22 @@ def main():
         idx = counters["pushed"] % len(worker_batches)
         src = list(worker_batches[idx])
         src[4] = None  # the target network's output is appended at the first traversal
-        slot = ring.push(src, stream)
+        slot = ring.push(src, stream_id)
         if slot is not None:
             slot_batch[slot] = idx
             counters["pushed"] += 1
             counters["copy"] += 1
         return slot
 
-    def step(timer=None):
-        got = ring.sample(None, stream)
+    def step():
+        got = ring.sample(None, stream_id)
         if got is None:
             raise RuntimeError("ring ran empty")
         slot, k = got
         if k == 0:  # first traversal: store the target network's output for this batch
-            ring.append(slot, 4, worker_batches[slot_batch[slot]][4], stream)
+            ring.append(slot, 4, worker_batches[slot_batch[slot]][4], stream_id)
             counters["copy"] += 1
-        if timer is not None:
-            timer[0].record(stream)
-        calls[slot](stream)
-        if timer is not None:
-            timer[1].record(stream)
+        calls[slot].on_stream(stream_id)
         counters["loss"] += 1
         if k == K - 1:
             push_one()
@@ -257,41 +261,102 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    # ---- timed region 1: K steps, whole-step throughput ---------------------------------------------------
+    def time_on_stream(fn):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        a.record(stream)
+        fn()
+        b.record(stream)
+        barrier()
+        return a.elapsed_time(b)
+
+    # ---- timed region: K learner iterations, whole-step throughput -----------------------------------------
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.25)
     for c in counters:
         counters[c] = counters[c] if c == "pushed" else 0
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
     t_wall0 = time.perf_counter()
-    e0.record(stream)
-    for _ in range(args.steps):
-        step()
-    e1.record(stream)
-    barrier()
+
+    def run_steps():
+        for _ in range(args.steps):
+            step()
+    ms_total = time_on_stream(run_steps)
     t_wall = time.perf_counter() - t_wall0
-    ms_total = e0.elapsed_time(e1)
     launches = counters["loss"] + counters["copy"]
     loss_launches = counters["loss"]
 
-    # ---- timed region 2: the same K steps again, an event pair around every loss launch (roofline) -------
-    pairs = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    barrier()
-    for i in range(args.steps):
-        step(pairs[i])
-    barrier()
-    loss_ms = [a.elapsed_time(b) for a, b in pairs]
-    # ---- and back to back: K loss launches over the rotating slots, nothing between them -----------------
-    d0, d1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    barrier()
-    d0.record(stream)
-    for i in range(args.steps):
-        calls[i % N](stream)
-    d1.record(stream)
-    barrier()
-    dense_ms = d0.elapsed_time(d1) / args.steps
+    # ---- the loss kernel alone: back-to-back launches over the rotating slots ---------------------------------
+    # (a) issued from this host loop; (b) the same launches captured once in a CUDA graph, so that no host
+    # time sits between them; (c) alternating between two streams (a workspace each), so that one launch's
+    # fixed start-up and drain overlap the other's transfers: throughput with two batches in flight.
+    n_dense = max(args.steps, 64)
+
+    def dense_loop():
+        for i in range(n_dense):
+            calls[i % N].on_stream(stream_id)
+    loop_ms = time_on_stream(dense_loop) / n_dense
+
+    side, side2 = torch.cuda.Stream(), torch.cuda.Stream()
+    graph1 = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph1, stream=side):
+            for i in range(n_dense):
+                calls[i % N].on_stream(side.cuda_stream)
+    graph2 = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph2, stream=side):
+            fork = torch.cuda.Event()
+            fork.record(side)
+            side2.wait_event(fork)
+            for i in range(n_dense):
+                if i % 2 == 0:
+                    calls[i % N].on_stream(side.cuda_stream)
+                else:
+                    calls2[i % N].on_stream(side2.cuda_stream)
+            join = torch.cuda.Event()
+            join.record(side2)
+            side.wait_event(join)
+    torch.cuda.synchronize()
+    graph1.replay()
+    graph2.replay()
+    dense_ms = min(time_on_stream(graph1.replay) for _ in range(5)) / n_dense
+    overlap_ms = min(time_on_stream(graph2.replay) for _ in range(5)) / n_dense
+
+    # ---- the same kernel on a batch eight times as large (B*T = 1,048,576): start-up and drain amortised ----
+    big = None
+    try:
+        bigB = 8 * B
+        big_calls = []
+        for i in range(3):
+            g_ = torch.Generator(device="cuda").manual_seed(1234 + i)
+            zl_ = torch.randn(bigB, T, A, device="cuda", generator=g_)
+            zt_ = zl_ + 0.1 * torch.randn(bigB, T, A, device="cuda", generator=g_)
+            zw_ = zl_ + 0.5 * torch.randn(bigB, T, A, device="cuda", generator=g_)
+            act_ = torch.distributions.Categorical(logits=zw_).sample().to(torch.int32)
+            wl_ = torch.log_softmax(zw_, -1).gather(-1, act_.long().unsqueeze(-1)).squeeze(-1).contiguous()
+            del zw_
+            u_ = torch.rand(bigB, T, device="cuda", generator=g_)
+            rew_ = (u_ < 0.05).float() * torch.where(u_ < 0.025, -1.0, 1.0)
+            dis_ = torch.where(torch.rand(bigB, T, device="cuda", generator=g_) < cfg.p_done, 0.0, cfg.gamma).float()
+            val_ = torch.randn(bigB, T, device="cuda", generator=g_)
+            boot_ = torch.randn(bigB, device="cuda", generator=g_)
+            o_ = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(bigB, T, A, device="cuda"),
+                      dvalues=torch.empty(bigB, T, device="cuda"))
+            big_calls.append(ip.prepare_loss_fwd_bwd(zl_, zt_, wl_, act_, rew_, dis_, val_, boot_, coef,
+                                                     workspace=workspace, **o_))
+        n_big = 48
+        for c_ in big_calls:
+            c_.on_stream(stream_id)
+
+        def big_loop():
+            for i in range(n_big):
+                big_calls[i % 3].on_stream(stream_id)
+        big_ms = min(time_on_stream(big_loop) for _ in range(3)) / n_big
+        big = {"timesteps": bigB * T, "avg_launch_us": big_ms * 1e3}
+        del big_calls
+    except RuntimeError as exc:  # out of memory on a small device: report without the large batch
+        big = {"error": str(exc)[:80]}
     time.sleep(0.15)
     clocks = sampler.stop()
 
@@ -310,7 +375,7 @@ def main():
     def e2e_step():
         for k_, v in pinned.items():
             dst[k_].copy_(v, non_blocking=True)
-        e2e_call(stream)
+        e2e_call.on_stream(stream_id)
         terms_host.copy_(out["loss_terms"], non_blocking=True)
         stream.synchronize()
 
@@ -324,26 +389,37 @@ def main():
     e2e_s = time.perf_counter() - t0
 
     # ---- reduce over ranks: the slowest rank sets the time ---------------------------------------------------
-    vals = torch.tensor([ms_total, e2e_s, statistics.fmean(loss_ms), dense_ms], device="cuda", dtype=torch.float64)
+    vals = torch.tensor([ms_total, e2e_s, loop_ms, dense_ms, overlap_ms], device="cuda", dtype=torch.float64)
     if dist is not None:
         dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    ms_total, e2e_s, loss_ms_avg, dense_ms = [float(x) for x in vals.cpu()]
+    ms_total, e2e_s, loop_ms, dense_ms, overlap_ms = [float(x) for x in vals.cpu()]
     value = world * args.steps * M / (ms_total * 1e-3)
     e2e_value = world * e2e_steps * M / e2e_s
 
     peak, peak_kind = peak_hbm_gbs()
     bytes_per_launch = algorithmic_bytes_per_step(A) * M
     achieved = bytes_per_launch / (dense_ms * 1e-3) / 1e9
+    gbs = lambda ms: bytes_per_launch / (ms * 1e-3) / 1e9
     roofline = {
-        "bound": "hbm", "kernel": "impact_loss_categorical_kernel<float,float,128>",
+        "bound": "hbm", "kernel": "impact_loss_categorical_reg_kernel<float,float,18>",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
-        "traffic": None,
+        "traffic": NCU_TRAFFIC_BYTES,
         "algorithmic_bytes_per_launch": bytes_per_launch,
         "avg_launch_us": dense_ms * 1e3,
-        "how": "K back-to-back loss launches over the rotating ring slots, CUDA events on the launch stream",
-        "avg_launch_us_event_pair_in_step": loss_ms_avg * 1e3,
-        "achieved_event_pair_in_step": bytes_per_launch / (loss_ms_avg * 1e-3) / 1e9,
+        "how": f"{n_dense} back-to-back loss launches over the rotating ring slots, captured in one CUDA graph; "
+               "CUDA events on the launch stream around the replay, best of 5",
+        "host_loop": {"avg_launch_us": loop_ms * 1e3, "achieved": gbs(loop_ms), "frac": gbs(loop_ms) / peak,
+                      "how": "the same launches issued one by one from the Python loop"},
+        "two_streams": {"avg_launch_us": overlap_ms * 1e3, "achieved": gbs(overlap_ms), "frac": gbs(overlap_ms) / peak,
+                        "how": "the same launches alternating between two streams (a workspace each): "
+                               "throughput with two batches in flight, not one launch's duration"},
     }
+    if big and "avg_launch_us" in big:
+        big_bytes = algorithmic_bytes_per_step(A) * big["timesteps"]
+        big["achieved"] = big_bytes / (big["avg_launch_us"] * 1e-6) / 1e9
+        big["frac"] = big["achieved"] / peak
+        big["how"] = "same kernel, B*T = 1,048,576 timesteps per launch, 3 rotating buffer sets, host loop"
+    roofline["large_batch"] = big
 
     line = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,

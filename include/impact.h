@@ -163,6 +163,38 @@ int32_t impact_loss_fwd_bwd(
     void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * The arguments of impact_loss_fwd_bwd as one plain struct, for callers that issue the same
+ * call many times (a learner loop over fixed buffers): fill it once, then pass its HOST
+ * address to impact_loss_fwd_bwd_call.  Field meanings, layouts, limits and errors are those
+ * of impact_loss_fwd_bwd; `coef` is embedded by value.
+ */
+typedef struct impact_loss_call {
+    const void* learner_logits;
+    const void* target_logits;
+    const float* worker_logp;
+    const int32_t* actions;
+    const float* rewards;
+    const float* discounts;
+    const float* values;
+    const float* bootstrap_values;
+    float rho_bar, c_bar, clip_eps;
+    int32_t logits_dtype;
+    impact_coefficients coef;
+    int32_t A;
+    int64_t B, T;
+    float* loss_terms;
+    void* dlogits;
+    float* dvalues;
+    float* vtarget;
+    float* advantage;
+    void* workspace;
+    size_t workspace_bytes;
+} impact_loss_call;
+
+/* impact_loss_fwd_bwd with its arguments taken from `call` (Algorithm 1, gradient step). */
+int32_t impact_loss_fwd_bwd_call(const impact_loss_call* call, void* stream);
+
+/*
  * The same loss for a diagonal-Gaussian policy with D action dimensions (continuous
  * control, Section 4.3; Appendix E).  sigma = exp(logstd), per step:
  *   log pi(a|s)  = sum_d [ -1/2 ((a_d - mu_d)/sigma_d)^2 - logstd_d - 1/2 ln 2pi ]

@@ -32,7 +32,7 @@ EXPORTS = (
     "impact_buffer_destroy", "impact_buffer_push", "impact_buffer_sample", "impact_buffer_append",
     "impact_buffer_slot_ptr", "impact_buffer_live", "impact_buffer_state_bytes",
     "impact_buffer_export_state", "impact_buffer_import_state", "impact_gather_rows",
-    "impact_loss_fwd_bwd_static_scratch",
+    "impact_loss_fwd_bwd_static_scratch", "impact_loss_fwd_bwd_call",
 )
 
 
@@ -47,6 +47,17 @@ class impact_coefficients(ctypes.Structure):
                 ("lambda_", ctypes.c_float), ("rho_tw", ctypes.c_float), ("is_source", ctypes.c_int32),
                 ("ratio_mode", ctypes.c_int32), ("dlogits_dtype", ctypes.c_int32),
                 ("reserved", ctypes.c_int32)]
+
+
+class impact_loss_call(ctypes.Structure):
+    _fields_ = [("learner_logits", ctypes.c_void_p), ("target_logits", ctypes.c_void_p),
+                ("worker_logp", ctypes.c_void_p), ("actions", ctypes.c_void_p), ("rewards", ctypes.c_void_p),
+                ("discounts", ctypes.c_void_p), ("values", ctypes.c_void_p), ("bootstrap_values", ctypes.c_void_p),
+                ("rho_bar", ctypes.c_float), ("c_bar", ctypes.c_float), ("clip_eps", ctypes.c_float),
+                ("logits_dtype", ctypes.c_int32), ("coef", impact_coefficients), ("A", ctypes.c_int32),
+                ("B", ctypes.c_int64), ("T", ctypes.c_int64), ("loss_terms", ctypes.c_void_p),
+                ("dlogits", ctypes.c_void_p), ("dvalues", ctypes.c_void_p), ("vtarget", ctypes.c_void_p),
+                ("advantage", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
 
 
 _lib = None
@@ -72,6 +83,8 @@ def load_library() -> ctypes.CDLL:
     lib.impact_loss_fwd_bwd.restype = _i32
     lib.impact_loss_fwd_bwd.argtypes = [_vp] * 8 + [_f32] * 3 + [ctypes.POINTER(impact_coefficients), _i64, _i64,
                                                                _i32, _i32] + [_vp] * 6 + [_sz, _vp]
+    lib.impact_loss_fwd_bwd_call.restype = _i32
+    lib.impact_loss_fwd_bwd_call.argtypes = [ctypes.POINTER(impact_loss_call), _vp]
     lib.impact_loss_fwd_bwd_static_scratch.restype = _i32
     lib.impact_loss_fwd_bwd_static_scratch.argtypes = [_vp] * 8 + [_f32] * 3 + [
         ctypes.POINTER(impact_coefficients), _i64, _i64, _i32, _i32] + [_vp] * 5 + [_vp]
@@ -196,6 +209,13 @@ class PreparedCall:
         if st != OK:
             _check(st, self._what)
 
+    def on_stream(self, cuda_stream: int) -> None:
+        """Same as `()`, for a raw cudaStream_t value (skips the torch stream lookup)."""
+        self._args[-1] = cuda_stream
+        st = self._fn(*self._args)
+        if st != OK:
+            _check(st, self._what)
+
 
 def prepare_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
                          bootstrap_values, coef: Coefficients, *, loss_terms, dlogits, dvalues,
@@ -207,18 +227,17 @@ def prepare_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, re
         raise ValueError("logits must be float32 or bfloat16")
     f32, bt = torch.float32, (B, T)
     cs = coef.c_struct(_DTYPE_CODE[dlogits.dtype])
-    args = [
+    call = impact_loss_call(
         _dev(learner_logits, ldt, (B, T, A), "learner_logits"), _dev(target_logits, ldt, (B, T, A), "target_logits"),
         _dev(worker_logp, f32, bt, "worker_logp"), _dev(actions, torch.int32, bt, "actions"),
         _dev(rewards, f32, bt, "rewards"), _dev(discounts, f32, bt, "discounts"), _dev(values, f32, bt, "values"),
         _dev(bootstrap_values, f32, (B,), "bootstrap_values"),
-        coef.rho_bar, coef.c_bar, coef.clip_eps, ctypes.pointer(cs), B, T, A, _DTYPE_CODE[ldt],
+        coef.rho_bar, coef.c_bar, coef.clip_eps, _DTYPE_CODE[ldt], cs, A, B, T,
         _dev(loss_terms, f32, (NUM_TERMS,), "loss_terms"), _dev(dlogits, dlogits.dtype, (B, T, A), "dlogits"),
         _dev(dvalues, f32, bt, "dvalues"), _dev(vtarget, f32, bt, "vtarget", True),
         _dev(advantage, f32, bt, "advantage", True),
-        _dev(workspace, torch.uint8, workspace.shape, "workspace"), workspace.numel(), 0,
-    ]
-    return PreparedCall(lib.impact_loss_fwd_bwd, args, "impact_loss_fwd_bwd", (cs,))
+        _dev(workspace, torch.uint8, workspace.shape, "workspace"), workspace.numel())
+    return PreparedCall(lib.impact_loss_fwd_bwd_call, [ctypes.byref(call), 0], "impact_loss_fwd_bwd_call", (call,))
 
 
 def impact_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,

@@ -1028,6 +1028,14 @@ extern "C" int32_t impact_loss_fwd_bwd(
                            di, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" int32_t impact_loss_fwd_bwd_call(const impact_loss_call* c, void* stream) {
+    if (!c) return IMPACT_ERR_INVALID_ARG;
+    return impact_loss_fwd_bwd(c->learner_logits, c->target_logits, c->worker_logp, c->actions, c->rewards,
+                               c->discounts, c->values, c->bootstrap_values, c->rho_bar, c->c_bar, c->clip_eps,
+                               &c->coef, c->B, c->T, c->A, c->logits_dtype, c->loss_terms, c->dlogits,
+                               c->dvalues, c->vtarget, c->advantage, c->workspace, c->workspace_bytes, stream);
+}
+
 extern "C" int32_t impact_loss_fwd_bwd_gaussian(
     const float* learner_mean, const float* learner_logstd, const float* target_mean,
     const float* target_logstd, const float* worker_logp, const float* actions,
