@@ -22,6 +22,36 @@ struct DeviceInfo {
 // Returns nullptr (and records the error) when no CUDA device is usable.
 const DeviceInfo* current_device_info();
 
+// Launch with programmatic stream serialization: the grid may be set up on the device while
+// the previous kernel of the stream is still running.  Every kernel of this library starts
+// with grid_dependency_wait(), which returns only once that previous kernel has completed
+// and its writes are visible, so stream order is kept exactly; what is saved is the launch
+// latency between consecutive kernels.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_serialized(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem,
+                                     cudaStream_t stream, Args&&... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+
+#ifdef __CUDACC__
+// First statement of every kernel: wait for the kernel before this one on the stream (a
+// no-op when there is none), then let the kernel after this one begin its own set-up.
+__device__ __forceinline__ void grid_dependency_wait() {
+    asm volatile("griddepcontrol.wait;" ::: "memory");
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+}
+#endif
+
 }  // namespace impact
 
 #define IMPACT_CUDA_TRY(expr)                                        \

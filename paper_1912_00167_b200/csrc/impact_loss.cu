@@ -101,6 +101,7 @@ __device__ __forceinline__ TileRows tile_rows(const TileGeometry& g, long long c
 // ------------------------------------------------------------------------------------------
 template <typename LT, typename GT, int NT>
 __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatParams p) {
+    grid_dependency_wait();
     extern __shared__ __align__(16) float smem[];
     float* const sl = smem;                          // learner rows, then gradient rows
     float* const st = smem + (size_t)NT * p.As;      // target rows
@@ -374,6 +375,7 @@ __device__ __forceinline__ float row_max(const RowRegs<A>& r) {
 
 template <typename LT, typename GT, int A>
 __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_kernel(const CatParams p) {
+    grid_dependency_wait();
     constexpr int NT = kRegTileRows;
     constexpr int NP = RowRegs<A>::NP;
     constexpr bool kOdd = (A & 1) != 0;
@@ -672,6 +674,7 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
 // ------------------------------------------------------------------------------------------
 template <int NT>
 __global__ void __launch_bounds__(NT) impact_loss_gaussian_kernel(const GaussParams p) {
+    grid_dependency_wait();
     extern __shared__ __align__(16) float smem[];
     const int D = p.D, Ds = p.Ds;
     float* const s_mu = smem;                              // learner mean -> dmean
@@ -889,8 +892,7 @@ int32_t launch_categorical(const CatParams& p, const DeviceInfo* di, cudaStream_
     int grid = 0;
     int32_t st = grid_for(kernel, NT, smem, p.geo.nchunks, di, &grid);
     if (st != IMPACT_OK) return st;
-    kernel<<<grid, NT, smem, stream>>>(p);
-    IMPACT_CUDA_TRY(cudaGetLastError());
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3(grid), dim3(NT), smem, stream, p));
     return IMPACT_OK;
 }
 
@@ -910,8 +912,7 @@ int32_t launch_categorical_reg(const CatParams& p, const DeviceInfo* di, cudaStr
     int grid = 0;
     int32_t st = grid_for(kernel, kRegTileRows, smem, p.geo.nchunks, di, &grid);
     if (st != IMPACT_OK) return st;
-    kernel<<<grid, kRegTileRows, smem, stream>>>(p);
-    IMPACT_CUDA_TRY(cudaGetLastError());
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3(grid), dim3(kRegTileRows), smem, stream, p));
     return IMPACT_OK;
 }
 
@@ -956,8 +957,7 @@ int32_t launch_gaussian(const GaussParams& p, const DeviceInfo* di, cudaStream_t
     int grid = 0;
     int32_t st = grid_for(kernel, NT, smem, p.geo.nchunks, di, &grid);
     if (st != IMPACT_OK) return st;
-    kernel<<<grid, NT, smem, stream>>>(p);
-    IMPACT_CUDA_TRY(cudaGetLastError());
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3(grid), dim3(NT), smem, stream, p));
     return IMPACT_OK;
 }
 

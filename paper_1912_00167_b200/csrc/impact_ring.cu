@@ -32,6 +32,7 @@ struct CopySegments {
 // Copies up to kMaxFields byte ranges in one launch.  Every range is walked in 16-byte
 // units; the last unit of a range whose length is not a multiple of 16 is copied bytewise.
 __global__ void __launch_bounds__(256) multi_copy_kernel(const CopySegments s) {
+    grid_dependency_wait();
     const unsigned long long total = s.vec_end[s.n - 1];
     const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
     unsigned long long v = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x;
@@ -72,6 +73,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const V* __restrict__ 
                                                           const int32_t* __restrict__ idx,
                                                           long long n, long long n_src_rows,
                                                           long long units, V* __restrict__ dst) {
+    grid_dependency_wait();
     const long long total = n * units;
     const long long stride = (long long)gridDim.x * blockDim.x;
     for (long long v = (long long)blockIdx.x * blockDim.x + threadIdx.x; v < total; v += stride) {
@@ -196,8 +198,7 @@ static int32_t launch_copy(const CopySegments& segs, cudaStream_t stream) {
     const DeviceInfo* di = current_device_info();
     if (!di) return IMPACT_ERR_CUDA;
     const unsigned long long total = segs.vec_end[segs.n - 1];
-    multi_copy_kernel<<<blocks_for(total, 4, di), 256, 0, stream>>>(segs);
-    IMPACT_CUDA_TRY(cudaGetLastError());
+    IMPACT_CUDA_TRY(launch_serialized(multi_copy_kernel, dim3(blocks_for(total, 4, di)), dim3(256), 0, stream, segs));
     return IMPACT_OK;
 }
 
@@ -362,16 +363,16 @@ extern "C" int32_t impact_gather_rows(const void* src, const int32_t* idx, int64
     const uintptr_t both = reinterpret_cast<uintptr_t>(src) | reinterpret_cast<uintptr_t>(dst) | row_bytes;
     if ((both & 15u) == 0) {
         const long long units = (long long)(row_bytes / 16);
-        gather_rows_kernel<uint4><<<blocks_for((unsigned long long)n * units, 4, di), 256, 0, cs>>>(
-            static_cast<const uint4*>(src), idx, n, n_src_rows, units, static_cast<uint4*>(dst));
+        IMPACT_CUDA_TRY(launch_serialized(gather_rows_kernel<uint4>, dim3(blocks_for((unsigned long long)n * units, 4, di)), dim3(256), 0, cs,
+                                          static_cast<const uint4*>(src), idx, (long long)n, (long long)n_src_rows, units, static_cast<uint4*>(dst)));
     } else if ((both & 3u) == 0) {
         const long long units = (long long)(row_bytes / 4);
-        gather_rows_kernel<uint32_t><<<blocks_for((unsigned long long)n * units, 4, di), 256, 0, cs>>>(
-            static_cast<const uint32_t*>(src), idx, n, n_src_rows, units, static_cast<uint32_t*>(dst));
+        IMPACT_CUDA_TRY(launch_serialized(gather_rows_kernel<uint32_t>, dim3(blocks_for((unsigned long long)n * units, 4, di)), dim3(256), 0, cs,
+                                          static_cast<const uint32_t*>(src), idx, (long long)n, (long long)n_src_rows, units, static_cast<uint32_t*>(dst)));
     } else {
         const long long units = (long long)row_bytes;
-        gather_rows_kernel<unsigned char><<<blocks_for((unsigned long long)n * units, 4, di), 256, 0, cs>>>(
-            static_cast<const unsigned char*>(src), idx, n, n_src_rows, units, static_cast<unsigned char*>(dst));
+        IMPACT_CUDA_TRY(launch_serialized(gather_rows_kernel<unsigned char>, dim3(blocks_for((unsigned long long)n * units, 4, di)), dim3(256), 0, cs,
+                                          static_cast<const unsigned char*>(src), idx, (long long)n, (long long)n_src_rows, units, static_cast<unsigned char*>(dst)));
     }
     IMPACT_CUDA_TRY(cudaGetLastError());
     return IMPACT_OK;
