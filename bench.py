@@ -158,6 +158,169 @@ def run_reference(args):
     print(json.dumps(line))
 
 
+def synth_categorical_device(B, T, A, seed, p_done, gamma, dtype):
+    """The categorical generator's recipe, drawn on the device with torch (for the sweep's large points)."""
+    import torch
+    g = torch.Generator(device="cuda").manual_seed(seed)
+    zl = torch.randn(B, T, A, device="cuda", generator=g)
+    zt = zl + 0.1 * torch.randn(B, T, A, device="cuda", generator=g)
+    zw = zl + 0.5 * torch.randn(B, T, A, device="cuda", generator=g)
+    lpw = torch.log_softmax(zw, -1)
+    del zw
+    u = torch.rand(B, T, 1, device="cuda", generator=g)
+    act = (u > lpw.exp().cumsum(-1)).sum(-1).clamp_(max=A - 1)
+    wl = lpw.gather(-1, act.unsqueeze(-1)).squeeze(-1).contiguous()
+    del lpw
+    u = torch.rand(B, T, device="cuda", generator=g)
+    rew = (u < 0.05).float() * torch.where(u < 0.025, -1.0, 1.0)
+    dis = torch.where(torch.rand(B, T, device="cuda", generator=g) < p_done, 0.0, gamma).float()
+    val = torch.randn(B, T, device="cuda", generator=g)
+    boot = torch.randn(B, device="cuda", generator=g)
+    return dict(learner_logits=zl.to(dtype), target_logits=zt.to(dtype), worker_logp=wl,
+                actions=act.to(torch.int32), rewards=rew, discounts=dis, values=val, bootstrap_values=boot)
+
+
+def run_sweep(args):
+    """Throughput sweep: categorical A x B*T x T x dtype, the Gaussian config, and ring (N, K) settings."""
+    import torch
+    import paper_1912_00167_b200 as ip
+    torch.cuda.set_device(0)
+    ip.load_library()
+    peak, peak_kind = peak_hbm_gbs()
+    stream = torch.cuda.current_stream()
+    sid = stream.cuda_stream
+    coef = ip.Coefficients(clip_eps=0.4)
+    rows = []
+
+    def time_calls(calls, n):
+        for c in calls:
+            c.on_stream(sid)
+        torch.cuda.synchronize()
+        best = None
+        for _ in range(3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(n):
+                calls[i % len(calls)].on_stream(sid)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / n
+            best = ms if best is None else min(best, ms)
+        return best
+
+    ws = ip.new_workspace(1, 1)
+    targets = [4096 * 4 ** i for i in range(6)]  # 4,096 ... 4,194,304 timesteps
+    for A in (6, 18, 64):
+        for T in (20, 50, 128):
+            for M_target in targets:
+                B = -(-M_target // T)
+                M = B * T
+                for dtype, name, lb in ((torch.float32, "fp32", 4), (torch.bfloat16, "bf16", 2)):
+                    per_step = algorithmic_bytes_per_step(A, lb, lb)
+                    foot = per_step * M
+                    nsets = int(max(2, min(12, -(-400_000_000 // foot))))
+                    if foot * nsets > 12_000_000_000:
+                        nsets = 2
+                    calls = []
+                    for i in range(nsets):
+                        d = synth_categorical_device(B, T, A, 100 + i, 0.01, 0.99, dtype)
+                        out = dict(loss_terms=torch.zeros(8, device="cuda"),
+                                   dlogits=torch.empty(B, T, A, device="cuda", dtype=dtype),
+                                   dvalues=torch.empty(B, T, device="cuda"))
+                        calls.append(ip.prepare_loss_fwd_bwd(d["learner_logits"], d["target_logits"], d["worker_logp"],
+                                                             d["actions"], d["rewards"], d["discounts"], d["values"],
+                                                             d["bootstrap_values"], coef, workspace=ws, **out))
+                    n = int(max(20, min(400, 20_000_000_000 // max(foot, 1) // 50)))
+                    ms = time_calls(calls, n)
+                    gbs = foot / (ms * 1e-3) / 1e9
+                    rows.append(dict(kind="categorical", A=A, T=T, B=B, timesteps=M, dtype=name,
+                                     us_per_launch=ms * 1e3, timesteps_per_s=M / (ms * 1e-3), gbs=gbs,
+                                     frac_of_peak=gbs / peak))
+                    del calls
+                    torch.cuda.empty_cache()
+    # Gaussian (config 3 shape and two larger batches)
+    cfg3 = ii.CONFIGS[3]
+    for mult in (1, 4, 16):
+        B, T, D = cfg3.B * mult, cfg3.T, cfg3.A
+        calls = []
+        for i in range(6 if mult == 1 else 3):
+            hb = ii.gaussian_batch(cfg3.B, T, D, 300 + i, p_done=cfg3.p_done)
+            d = {k: torch.from_numpy(v).cuda().repeat(*([mult] + [1] * (v.ndim - 1))) for k, v in hb.items()}
+            out = dict(loss_terms=torch.zeros(8, device="cuda"), dmean=torch.empty(B, T, D, device="cuda"),
+                       dlogstd=torch.empty(B, T, D, device="cuda"), dvalues=torch.empty(B, T, device="cuda"))
+            calls.append(ip.prepare_loss_fwd_bwd_gaussian(
+                d["learner_mean"], d["learner_logstd"], d["target_mean"], d["target_logstd"], d["worker_logp"],
+                d["actions"], d["rewards"], d["discounts"], d["values"], d["bootstrap_values"],
+                ip.Coefficients(ent_coef=0.0), workspace=ws, **out))
+        ms = time_calls(calls, 200 if mult == 1 else 50)
+        foot = (4 * (5 * D + 5) + 4 * (2 * D + 1)) * B * T
+        gbs = foot / (ms * 1e-3) / 1e9
+        rows.append(dict(kind="gaussian", A=D, T=T, B=B, timesteps=B * T, dtype="fp32", us_per_launch=ms * 1e3,
+                         timesteps_per_s=B * T / (ms * 1e-3), gbs=gbs, frac_of_peak=gbs / peak))
+        del calls
+        torch.cuda.empty_cache()
+    # ring settings at the config-2 shape: learner iterations per second with push / append / sample
+    cfg = ii.CONFIGS[WORKLOAD_IDX]
+    B, T, A = cfg.B, cfg.T, cfg.A
+    batches = [synth_categorical_device(B, T, A, 500 + i, cfg.p_done, cfg.gamma, torch.float32) for i in range(8)]
+    outs = [dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
+                 dvalues=torch.empty(B, T, device="cuda")) for _ in range(8)]
+    for N in (4, 32):
+        for K in (1, 2, 4, 8):
+            fields = [[b[n] for n in FIELD_NAMES] for b in batches]
+            ring = ip.ImpactBuffer(N, K, [t.numel() * t.element_size() for t in fields[0]], seed=N * 10 + K)
+            calls = []
+            for s_ in range(N):
+                v = [ring.slot_view(s_, f, fields[0][f].dtype, fields[0][f].shape) for f in range(5)]
+                bb = batches[s_ % 8]
+                calls.append(ip.prepare_loss_fwd_bwd(bb["learner_logits"], v[4], v[3], v[0], v[1], v[2], bb["values"],
+                                                     bb["bootstrap_values"], coef, workspace=ws, **outs[s_ % 8]))
+            state = {"pushed": 0}
+            where = [0] * N
+
+            def push():
+                src = list(fields[state["pushed"] % 8])
+                src[4] = None
+                slot = ring.push(src, sid)
+                if slot is not None:
+                    where[slot] = state["pushed"] % 8
+                    state["pushed"] += 1
+                return slot
+
+            def step():
+                slot, k = ring.sample(None, sid)
+                if k == 0:
+                    ring.append(slot, 4, fields[where[slot]][4], sid)
+                calls[slot].on_stream(sid)
+                if k == K - 1:
+                    push()
+            while push() is not None:
+                pass
+            for _ in range(50):
+                step()
+            torch.cuda.synchronize()
+            n = 500
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for _ in range(n):
+                step()
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / n
+            rows.append(dict(kind="ring+loss", A=A, T=T, B=B, timesteps=B * T, dtype="fp32", N=N, K=K,
+                             us_per_launch=ms * 1e3, timesteps_per_s=B * T / (ms * 1e-3)))
+            ring.close()
+    out_path = args.sweep_out
+    with open(out_path, "w") as f:
+        json.dump({"peak_gbs": peak, "peak_kind": peak_kind, "rows": rows}, f, indent=1)
+    print(f"# sweep: us per launch / timesteps per second / algorithmic GB/s / fraction of {peak:.0f} GB/s ({peak_kind})")
+    for r in rows:
+        extra = f" N={r['N']} K={r['K']}" if "N" in r else ""
+        gb = f" {r['gbs']:8.0f} GB/s {r['frac_of_peak']:.3f}" if "gbs" in r else ""
+        print(f"{r['kind']:12s} A={r['A']:3d} T={r['T']:4d} B={r['B']:7d} steps={r['timesteps']:8d} {r['dtype']}{extra}: "
+              f"{r['us_per_launch']:9.2f} us {r['timesteps_per_s'] / 1e9:7.3f} G/s{gb}")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -165,7 +328,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=200)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sweep", action="store_true", help="run the throughput sweep instead of the benchmark line")
+    ap.add_argument("--sweep-out", default="sweep.json")
     args = ap.parse_args()
+    if args.sweep:
+        run_sweep(args)
+        return
     if args.warmup < 3:
         args.warmup = 3
     if args.impl == "reference":
