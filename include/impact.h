@@ -71,8 +71,8 @@ extern "C" {
 #define IMPACT_TERM_POLICY 1     /* -(1/M) sum_t surrogate_t */
 #define IMPACT_TERM_VALUE 2      /* (1/M) sum_t 1/2 (V_t - Vhat_t)^2 */
 #define IMPACT_TERM_ENTROPY 3    /* (1/M) sum_t H(pi_theta(.|s_t)) */
-#define IMPACT_TERM_KL 4         /* (1/M) sum_t KL(pi_target(.|s_t) || pi_theta(.|s_t)); the categorical
-                                    call evaluates it only when kl_coef != 0 and reports 0 otherwise */
+#define IMPACT_TERM_KL 4         /* (1/M) sum_t KL(pi_target(.|s_t) || pi_theta(.|s_t)); evaluated only
+                                    when kl_coef != 0, reported as 0 otherwise */
 #define IMPACT_TERM_CLIP_FRAC 5  /* share of steps whose policy gradient the eps-clip removed */
 #define IMPACT_TERM_RHO_FRAC 6   /* share of steps whose importance weight exceeded rho_bar */
 #define IMPACT_TERM_MEAN_RATIO 7 /* (1/M) sum_t R_t */

@@ -737,10 +737,11 @@ __global__ void __launch_bounds__(NT) impact_loss_gaussian_kernel(const GaussPar
                     lth += (double)(fmaf(-0.5f * z1, z1, -ls) - half_log_2pi);
                     ltg += (double)(fmaf(-0.5f * z2, z2, -lt) - half_log_2pi);
                     ent += ls + (half_log_2pi + 0.5f);
-                    // KL(target || learner), per dimension
-                    const float dm = (r_mt[j] - r_mu[j]) * inv_s;
-                    const float sr = expf(lt - ls);  // sigma_target / sigma_learner
-                    kl += (ls - lt) + 0.5f * fmaf(sr, sr, dm * dm) - 0.5f;
+                    if (k.kl_coef != 0.0f) {  // KL(target || learner), per dimension
+                        const float dm = (r_mt[j] - r_mu[j]) * inv_s;
+                        const float sr = expf(lt - ls);  // sigma_target / sigma_learner
+                        kl += (ls - lt) + 0.5f * fmaf(sr, sr, dm * dm) - 0.5f;
+                    }
                 }
                 // differences against the worker's log-probability are taken in fp64, then
                 // everything continues in fp32 relative to it
@@ -800,6 +801,199 @@ __global__ void __launch_bounds__(NT) impact_loss_gaussian_kernel(const GaussPar
     }
     dev::finish_loss_terms<NT>(acc, p.partials, p.counter, p.loss_terms, k,
                                (double)g.B * (double)g.T);
+}
+
+// ------------------------------------------------------------------------------------------
+// Diagonal-Gaussian policy, action dimension known at compile time
+// ------------------------------------------------------------------------------------------
+// Same structure as the register-resident categorical kernel: the five [tile, D] slabs
+// (learner mean / log-std, target mean / log-std, actions) arrive by bulk copies, a thread
+// walks its row with every loop unrolled, dmean / dlogstd replace the learner slabs in place and
+// leave by two bulk stores.  One stage per block (five slabs are 43 KB at D = 17), four
+// blocks per SM overlap each other's loads and arithmetic.
+template <int D>
+__global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kernel(const GaussParams p) {
+    grid_dependency_wait();
+    constexpr int NT = kRegTileRows;
+    constexpr int kSlab = NT * D * (int)sizeof(float);
+    constexpr float kLog2e = 1.4426950408889634f;
+    constexpr float kHalfLog2Pi = 0.91893853320467274178f;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    float* const s_mu = reinterpret_cast<float*>(smem_raw);              // learner mean -> dmean
+    float* const s_ls = reinterpret_cast<float*>(smem_raw + kSlab);      // learner log-std -> dlogstd
+    const float* const s_mt = reinterpret_cast<const float*>(smem_raw + 2 * kSlab);
+    const float* const s_lt = reinterpret_cast<const float*>(smem_raw + 3 * kSlab);
+    const float* const s_ac = reinterpret_cast<const float*>(smem_raw + 4 * kSlab);
+    __shared__ __align__(8) uint64_t bar;
+    __shared__ float2 warp_agg[NT / 32];
+    __shared__ float red[NT / 32][8];
+    __shared__ float carry_s;
+    __shared__ int is_last_s;
+
+    const int tid = threadIdx.x;
+    const LossScalars k = p.k;
+    const TileGeometry g = p.geo;
+    const bool want_kl = (k.kl_coef != 0.0f);
+    const float* const src[5] = {p.learner_mean, p.learner_logstd, p.target_mean, p.target_logstd, p.actions};
+
+    if (tid == 0) {
+        dev::mbarrier_init(&bar, 1);
+        is_last_s = 0;
+    }
+    __syncthreads();
+    uint32_t parity = 0;
+
+    float acc[dev::kNumSums];
+#pragma unroll
+    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = 0.0f;
+
+    for (long long chunk = blockIdx.x; chunk < g.nchunks; chunk += gridDim.x) {
+        float carry = 0.0f;
+        for (int tile = g.ntiles - 1; tile >= 0; --tile) {
+            const bool final_tile = (tile == 0) && (chunk + gridDim.x >= g.nchunks);
+            const TileRows tr = tile_rows<NT>(g, chunk, tile);
+            const long long base = tr.row0 * D;
+            const uint32_t bytes = (uint32_t)tr.nrows * D * (uint32_t)sizeof(float);
+            uintptr_t align = bytes;
+#pragma unroll
+            for (int q = 0; q < 5; ++q) align |= reinterpret_cast<uintptr_t>(src[q] + base);
+            const bool bulk_in = (align & 15u) == 0;
+            const bool bulk_out = (((reinterpret_cast<uintptr_t>(p.dmean + base) |
+                                     reinterpret_cast<uintptr_t>(p.dlogstd + base) | bytes) & 15u) == 0);
+            if (bulk_in) {
+                if (tid == 0) {
+                    dev::mbarrier_expect_tx(&bar, 5 * bytes);
+#pragma unroll
+                    for (int q = 0; q < 5; ++q) dev::bulk_load(smem_raw + q * kSlab, src[q] + base, bytes, &bar);
+                }
+            } else {
+                const int nelem = tr.nrows * D;
+#pragma unroll
+                for (int q = 0; q < 5; ++q)
+                    for (int e = tid; e < nelem; e += NT) reinterpret_cast<float*>(smem_raw + q * kSlab)[e] = src[q][base + e];
+            }
+
+            const bool active = tid < tr.nrows;
+            const long long row = tr.row0 + tid;
+            dev::StepIn s;
+            float lw = 0.0f;
+            if (active) {
+                long long b, t;
+                if (g.ntiles > 1) { b = chunk; t = (long long)tile * NT + tid; }
+                else if (g.G == 1) { b = chunk; t = tid; }
+                else { const int q = tid / (int)g.T; b = chunk * g.G + q; t = tid - q * (int)g.T; }
+                lw = p.worker_logp[row];
+                s.reward = p.rewards[row];
+                s.discount = p.discounts[row];
+                s.value = p.values[row];
+                s.last_step = (t == g.T - 1);
+                s.value_next = s.last_step ? p.bootstrap[b] : p.values[row + 1];
+            }
+            if (bulk_in) {
+                if (tid < 32) {
+                    if (!dev::mbarrier_wait(&bar, parity)) atomicExch(p.counter + 1, 1u);
+                }
+                parity ^= 1u;
+            }
+            __syncthreads();
+
+            float* const r_mu = s_mu + tid * D;
+            float* const r_ls = s_ls + tid * D;
+            const float* const r_mt = s_mt + tid * D;
+            const float* const r_lt = s_lt + tid * D;
+            const float* const r_ac = s_ac + tid * D;
+            float fa = 1.0f, fb = 0.0f, ent = 0.0f, kl = 0.0f;
+            bool truncated = false;
+            if (active) {
+                // log-probabilities: D-term sums of magnitude tens that end up in exponents, so they
+                // are accumulated in fp64 (half-rate here, a few percent of the pipe)
+                double lth = 0.0, ltg = 0.0;
+                float ls_sum = 0.0f;
+#pragma unroll
+                for (int j = 0; j < D; ++j) {
+                    const float ls = r_ls[j], lt = r_lt[j], ac = r_ac[j], mu = r_mu[j], mt = r_mt[j];
+                    const float inv_s = dev::exp2_fast(-ls * kLog2e), inv_st = dev::exp2_fast(-lt * kLog2e);
+                    const float z1 = (ac - mu) * inv_s;
+                    const float z2 = (ac - mt) * inv_st;
+                    lth += (double)fmaf(-0.5f * z1, z1, -ls);
+                    ltg += (double)fmaf(-0.5f * z2, z2, -lt);
+                    ls_sum += ls;
+                    if (want_kl) {  // KL(target || learner), per dimension
+                        const float dm = (mt - mu) * inv_s;
+                        const float sr = dev::exp2_fast((lt - ls) * kLog2e);  // sigma_target / sigma_learner
+                        kl += (ls - lt) + 0.5f * fmaf(sr, sr, dm * dm) - 0.5f;
+                    }
+                }
+                ent = ls_sum + (float)D * (kHalfLog2Pi + 0.5f);
+                const double shift = (double)lw + (double)D * (double)kHalfLog2Pi;
+                // everything downstream works on log-probabilities relative to the worker's
+                s.l_theta = (float)(lth - shift);
+                s.l_target = (float)(ltg - shift);
+                s.l_worker = 0.0f;
+                truncated = dev::recursion_map(s, k, fa, fb);
+            }
+            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
+            if (tid == 0) carry_s = adv;
+
+            float surr = 0.0f, ratio = 0.0f, wpg = 0.0f;
+            bool clipped = false;
+            if (active) wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
+            {
+                const float sums5[5] = {surr, active ? 0.5f * adv * adv : 0.0f, ent, kl, ratio};
+                dev::block_sums_stage1_flags<NT>(sums5, clipped, truncated, red);
+            }
+            __syncthreads();
+            unsigned int ticket = 0;
+            if (tid == 0) {
+                dev::block_sums_stage2<NT>(acc, red);
+                if (final_tile) ticket = dev::publish_block_sums(acc, p.partials, p.counter);
+            }
+            if (active) {
+                const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = k.kl_coef * k.inv_M;
+#pragma unroll
+                for (int j = 0; j < D; ++j) {
+                    const float ls = r_ls[j], mu = r_mu[j];
+                    const float inv_s = dev::exp2_fast(-ls * kLog2e);
+                    const float z = (r_ac[j] - mu) * inv_s;  // (a - mu) / sigma
+                    // d log pi / d mu = z / sigma ;  d log pi / d logstd = z^2 - 1 ;  d H / d logstd = 1
+                    float gm = -w1 * z;
+                    float gs = -w1 * fmaf(z, z, -1.0f) - ce;
+                    if (want_kl) {
+                        // d KL / d mu = (mu - mu_t) / sigma^2 ; d KL / d logstd = 1 - (sigma_t^2 + (mu_t - mu)^2) / sigma^2
+                        const float dm = (mu - r_mt[j]) * inv_s;
+                        const float sr = dev::exp2_fast((r_lt[j] - ls) * kLog2e);
+                        gm = fmaf(ck, dm, gm);
+                        gs = fmaf(ck, 1.0f - fmaf(sr, sr, dm * dm), gs);
+                    }
+                    r_mu[j] = gm * inv_s;
+                    r_ls[j] = gs;
+                }
+                p.dvalues[row] = -k.vf_coef * k.inv_M * adv;
+                if (p.vtarget) p.vtarget[row] = s.value + adv;
+                if (p.advantage) p.advantage[row] = adv;
+            }
+            if (bulk_out) dev::fence_async_shared();
+            if (tid == 0 && final_tile) is_last_s = (ticket == gridDim.x - 1) ? 1 : 0;
+            __syncthreads();
+            carry = carry_s;
+            if (bulk_out) {
+                if (tid == 0) {
+                    dev::bulk_store(p.dmean + base, s_mu, bytes);
+                    dev::bulk_store(p.dlogstd + base, s_ls, bytes);
+                    if (!final_tile) dev::bulk_store_wait_read();
+                }
+            } else {
+                const int nelem = tr.nrows * D;
+                for (int i = tid; i < nelem; i += NT) {
+                    p.dmean[base + i] = s_mu[i];
+                    p.dlogstd[base + i] = s_ls[i];
+                }
+            }
+            if (!final_tile) __syncthreads();
+        }
+    }
+    if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k, (double)g.B * (double)g.T);
+    if (tid == 0) dev::bulk_store_wait_read();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -961,6 +1155,20 @@ int32_t launch_gaussian(const GaussParams& p, const DeviceInfo* di, cudaStream_t
     return IMPACT_OK;
 }
 
+template <int D>
+int32_t launch_gaussian_reg(const GaussParams& p, const DeviceInfo* di, cudaStream_t stream) {
+    auto kernel = impact_loss_gaussian_reg_kernel<D>;
+    const size_t smem = (size_t)5 * kRegTileRows * D * sizeof(float);
+    int grid = 0;
+    int32_t st = grid_for(kernel, kRegTileRows, smem, p.geo.nchunks, di, &grid);
+    if (st != IMPACT_OK) return st;
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3(grid), dim3(kRegTileRows), smem, stream, p));
+    return IMPACT_OK;
+}
+
+// Action dimensions with a compiled register-resident kernel (the MuJoCo tasks of Section 4.3).
+constexpr bool has_gaussian_reg_kernel(int D) { return D == 3 || D == 6 || D == 17; }
+
 }  // namespace
 }  // namespace impact
 
@@ -1087,6 +1295,16 @@ extern "C" int32_t impact_loss_fwd_bwd_gaussian(
     p.counter = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) +
                                                 (size_t)kMaxGridBlocks * 8 * sizeof(float));
     p.D = D;
+    if (has_gaussian_reg_kernel(D)) {
+        p.Ds = D;
+        p.geo = make_geometry(B, T, kRegTileRows);
+        cudaStream_t rs = static_cast<cudaStream_t>(stream);
+        switch (D) {
+            case 3: return launch_gaussian_reg<3>(p, di, rs);
+            case 6: return launch_gaussian_reg<6>(p, di, rs);
+            default: return launch_gaussian_reg<17>(p, di, rs);
+        }
+    }
     p.Ds = pad_odd(D);
     const int nt = pick_nt(p.Ds, 5, 100 * 1024);
     p.geo = make_geometry(B, T, nt);

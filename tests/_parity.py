@@ -190,4 +190,4 @@ def check_gaussian(oracle, batch, h, **tol):
     sens = _policy_sensitivity(oracle.loss_gaussian, batch, h, ["dmean", "dlogstd"], M,
                                near.astype(np.int8) if near.any() else None)
     return compare(gpu, ref, ref_flipped, near, M, ["dmean", "dlogstd"], h.kl_coef, sens, h.vf_coef,
-                   scale_l=logp_scale(batch), kl_always=True, **tol)
+                   scale_l=logp_scale(batch), **tol)
