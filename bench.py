@@ -129,6 +129,18 @@ def time_oracle(batch, hyper, min_seconds: float, max_reps: int):
     return reps * M / el, reps, el
 
 
+def aggregate_over_ranks(times_ms, steps, timesteps_per_step, world, dist=None, device="cpu"):
+    """Whole-job numbers from per-rank times: the slowest rank sets each time (MAX over ranks) and every
+    rank contributes the same number of timesteps (replicas of one workload: weak scaling)."""
+    import torch
+    vals = torch.tensor(list(times_ms), dtype=torch.float64, device=device)
+    if dist is not None and world > 1:
+        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
+    times = [float(x) for x in vals.cpu()]
+    value = world * steps * timesteps_per_step / (times[0] * 1e-3)
+    return times, value
+
+
 def run_reference(args):
     """The reference arm: the CPU oracle on the same workload, metric and unit."""
     rank = int(os.environ.get("RANK", "0"))
@@ -557,11 +569,8 @@ def main():
     e2e_s = time.perf_counter() - t0
 
     # ---- reduce over ranks: the slowest rank sets the time ---------------------------------------------------
-    vals = torch.tensor([ms_total, e2e_s, loop_ms, dense_ms, overlap_ms], device="cuda", dtype=torch.float64)
-    if dist is not None:
-        dist.all_reduce(vals, op=dist.ReduceOp.MAX)
-    ms_total, e2e_s, loop_ms, dense_ms, overlap_ms = [float(x) for x in vals.cpu()]
-    value = world * args.steps * M / (ms_total * 1e-3)
+    (ms_total, e2e_s, loop_ms, dense_ms, overlap_ms), value = aggregate_over_ranks(
+        [ms_total, e2e_s, loop_ms, dense_ms, overlap_ms], args.steps, M, world, dist, "cuda")
     e2e_value = world * e2e_steps * M / e2e_s
 
     peak, peak_kind = peak_hbm_gbs()

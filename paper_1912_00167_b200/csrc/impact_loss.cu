@@ -478,9 +478,9 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
         return r;
     };
 
-    float acc[dev::kNumSums];
+    float acc[dev::kNumSums], tsum[dev::kNumSums];
 #pragma unroll
-    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = 0.0f;
+    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = tsum[j] = 0.0f;
 
     Tile cur_tile = tile_of(0);
     fill_stage(cur_tile, 0);
@@ -595,16 +595,26 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
             float surr = 0.0f, ratio = 0.0f, wpg = 0.0f;
             bool clipped = false;
             if (active) wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
-            {
-                const float sums5[5] = {surr, active ? 0.5f * adv * adv : 0.0f, ent, kl, ratio};
-                dev::block_sums_stage1_flags<NT>(sums5, clipped, truncated, red);
+            // each thread keeps its own running sums over the block's tiles; they are added across
+            // the block once, in the last tile, and published right away so that the round trip
+            // hides behind the epilogue
+            if (active) {
+                tsum[0] += surr;
+                tsum[1] = fmaf(0.5f * adv, adv, tsum[1]);
+                tsum[2] += ent;
+                tsum[3] += kl;
+                tsum[4] += clipped ? 1.0f : 0.0f;
+                tsum[5] += truncated ? 1.0f : 0.0f;
+                tsum[6] += ratio;
             }
-            __syncthreads();
             unsigned int ticket = 0;
-            if (tid == 0) {
-                dev::block_sums_stage2<NT>(acc, red);
-                // sums of the block's last tile: publish now, the round trip hides behind the epilogue
-                if (final_tile) ticket = dev::publish_block_sums(acc, p.partials, p.counter);
+            if (final_tile) {
+                dev::block_sums_stage1<NT>(tsum, red);
+                __syncthreads();
+                if (tid == 0) {
+                    dev::block_sums_stage2<NT>(acc, red);
+                    ticket = dev::publish_block_sums(acc, p.partials, p.counter);
+                }
             }
 
             if (active) {
@@ -843,9 +853,9 @@ __global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kern
     __syncthreads();
     uint32_t parity = 0;
 
-    float acc[dev::kNumSums];
+    float acc[dev::kNumSums], tsum[dev::kNumSums];
 #pragma unroll
-    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = 0.0f;
+    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = tsum[j] = 0.0f;
 
     for (long long chunk = blockIdx.x; chunk < g.nchunks; chunk += gridDim.x) {
         float carry = 0.0f;
@@ -938,15 +948,26 @@ __global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kern
             float surr = 0.0f, ratio = 0.0f, wpg = 0.0f;
             bool clipped = false;
             if (active) wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
-            {
-                const float sums5[5] = {surr, active ? 0.5f * adv * adv : 0.0f, ent, kl, ratio};
-                dev::block_sums_stage1_flags<NT>(sums5, clipped, truncated, red);
+            // each thread keeps its own running sums over the block's tiles; they are added across
+            // the block once, in the last tile, and published right away so that the round trip
+            // hides behind the epilogue
+            if (active) {
+                tsum[0] += surr;
+                tsum[1] = fmaf(0.5f * adv, adv, tsum[1]);
+                tsum[2] += ent;
+                tsum[3] += kl;
+                tsum[4] += clipped ? 1.0f : 0.0f;
+                tsum[5] += truncated ? 1.0f : 0.0f;
+                tsum[6] += ratio;
             }
-            __syncthreads();
             unsigned int ticket = 0;
-            if (tid == 0) {
-                dev::block_sums_stage2<NT>(acc, red);
-                if (final_tile) ticket = dev::publish_block_sums(acc, p.partials, p.counter);
+            if (final_tile) {
+                dev::block_sums_stage1<NT>(tsum, red);
+                __syncthreads();
+                if (tid == 0) {
+                    dev::block_sums_stage2<NT>(acc, red);
+                    ticket = dev::publish_block_sums(acc, p.partials, p.counter);
+                }
             }
             if (active) {
                 const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = k.kl_coef * k.inv_M;
