@@ -183,3 +183,39 @@ def test_bad_arguments_are_rejected_before_launch():
     assert e.value.status == bd.ERR_INVALID_ARG
     call(ip.Coefficients())  # and the good call still works afterwards
     torch.cuda.synchronize()
+
+
+@pytest.mark.parametrize("B,T,A,dtype", [(8192, 128, 18, torch.float32), (20972, 50, 18, torch.float32),
+                                         (4096, 128, 18, torch.bfloat16), (512, 1000, 6, torch.float32)])
+def test_sampled_trajectories_at_sweep_sizes(oracle, B, T, A, dtype):
+    """Sizes far beyond what the oracle runs in full: trajectories are independent except for the 1/M
+    normaliser, so a sample of them is recomputed by the oracle alone and compared after rescaling."""
+    import paper_1912_00167_b200 as ip
+    batch = ii.categorical_batch(B, T, A, seed=4242 + B, p_done=0.01)
+    if dtype == torch.bfloat16:
+        batch["learner_logits"] = ii.round_to_bf16(batch["learner_logits"])
+        batch["target_logits"] = ii.round_to_bf16(batch["target_logits"])
+    h = P.f32_hyper(LossHyper(clip_eps=0.4, rho_tw=2.0, lam=0.995))
+    gpu = P.run_gpu_categorical(batch, h, dtype, torch.float32)
+    M = B * T
+    rng = np.random.default_rng(7)
+    pick = np.sort(rng.choice(B, size=24, replace=False))
+    pick[0], pick[-1] = 0, B - 1  # first and last tile
+    sub = {k: np.ascontiguousarray(v[pick]) for k, v in batch.items()}
+    ref = oracle.loss_categorical(sub, h)
+    Ms = len(pick) * T
+    near = P.near_clip_bound(ref, h)
+    tol = 1e-5 * np.abs(ref["dlogits"] * Ms) + 1e-6 + 4e-6 * (ref["adv_cond"] * ref["ratio"])[..., None]
+    err = np.abs(gpu["dlogits"][pick] * M - ref["dlogits"] * Ms)
+    assert (err <= tol)[~near].all(), float((err - tol)[~near].max())
+    np.testing.assert_array_less(np.abs(gpu["advantage"][pick] - ref["advantage"]),
+                                 1e-5 * np.abs(ref["advantage"]) + 1e-6 + 4e-6 * ref["adv_cond"])
+    np.testing.assert_array_less(np.abs(gpu["dvalues"][pick] * M - ref["dvalues"] * Ms),
+                                 1e-5 * np.abs(ref["dvalues"] * Ms) + 1e-6 + 4e-6 * ref["adv_cond"])
+    # properties that hold at any size
+    rows = gpu["dlogits"].sum(-1) * M
+    assert (np.abs(rows) <= 1e-5 * (1.0 + np.abs(gpu["dlogits"]).sum(-1) * M)).all()
+    lt = gpu["loss_terms"]
+    assert lt[0] == pytest.approx(lt[1] + h.vf_coef * lt[2] - h.ent_coef * lt[3] + h.kl_coef * lt[4], rel=1e-5, abs=1e-6)
+    assert lt[2] == pytest.approx(0.5 * np.mean(gpu["advantage"] ** 2), rel=1e-4)
+    assert 0.0 < lt[3] <= np.log(A) + 1e-5 and 0.0 <= lt[5] <= 1.0 and 0.0 <= lt[6] <= 1.0
