@@ -116,6 +116,16 @@ size_t impact_loss_workspace_bytes(int64_t B, int64_t T);
 int32_t impact_loss_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Reads a workspace's error word into *flag_out (HOST): 0 = no loss call that used this
+ * workspace ever gave up waiting for one of its own asynchronous copies; non-zero = at least
+ * one did (the wait inside the kernels is bounded, so a copy that never lands becomes this
+ * flag instead of a hang, and that call's outputs are not to be trusted).  The word is
+ * cleared by impact_loss_workspace_init only.  Synchronises `stream` before reading.
+ */
+int32_t impact_loss_workspace_status(const void* workspace, size_t workspace_bytes, int32_t* flag_out,
+                                     void* stream);
+
+/*
  * IMPACT loss and gradients for a discrete-action policy (Algorithm 1, "Compute policy
  * and value network gradients"), in one fused pass.  With M = B*T, per step t of a
  * trajectory (a = actions[b,t], gamma_t = discounts[b,t]):
@@ -230,7 +240,8 @@ int32_t impact_loss_fwd_bwd_gaussian(
  *
  * Limits: A <= 64, and the batch must split into at most 1024 tiles of 128 steps:
  * ceil(B / floor(128 / T)) <= 1024 when T <= 128, else B <= 1024.  (B=1024, T=128 is the
- * largest batch of full-length trajectories.)  Larger batches return
+ * largest batch of full-length trajectories.  One combination works on tiles of 64 steps and
+ * so fits half as much: 32 < A <= 64 with fp32 logits and bf16 gradients.)  Larger batches return
  * IMPACT_ERR_WORKSPACE_TOO_SMALL, A > 64 returns IMPACT_ERR_UNSUPPORTED; use
  * impact_loss_fwd_bwd with a workspace for those.
  *

@@ -32,7 +32,7 @@ EXPORTS = (
     "impact_buffer_destroy", "impact_buffer_push", "impact_buffer_sample", "impact_buffer_append",
     "impact_buffer_slot_ptr", "impact_buffer_live", "impact_buffer_state_bytes",
     "impact_buffer_export_state", "impact_buffer_import_state", "impact_gather_rows",
-    "impact_loss_fwd_bwd_static_scratch", "impact_loss_fwd_bwd_call",
+    "impact_loss_fwd_bwd_static_scratch", "impact_loss_fwd_bwd_call", "impact_loss_workspace_status",
 )
 
 
@@ -83,6 +83,8 @@ def load_library() -> ctypes.CDLL:
     lib.impact_loss_fwd_bwd.restype = _i32
     lib.impact_loss_fwd_bwd.argtypes = [_vp] * 8 + [_f32] * 3 + [ctypes.POINTER(impact_coefficients), _i64, _i64,
                                                                _i32, _i32] + [_vp] * 6 + [_sz, _vp]
+    lib.impact_loss_workspace_status.restype = _i32
+    lib.impact_loss_workspace_status.argtypes = [_vp, _sz, ctypes.POINTER(_i32), _vp]
     lib.impact_loss_fwd_bwd_call.restype = _i32
     lib.impact_loss_fwd_bwd_call.argtypes = [ctypes.POINTER(impact_loss_call), _vp]
     lib.impact_loss_fwd_bwd_static_scratch.restype = _i32
@@ -184,6 +186,15 @@ def impact_loss_workspace_bytes(B: int, T: int) -> int:
 def impact_loss_workspace_init(workspace: torch.Tensor, stream=None) -> None:
     _check(load_library().impact_loss_workspace_init(workspace.data_ptr(), workspace.numel() * workspace.element_size(),
                                                      _stream(stream)), "impact_loss_workspace_init")
+
+
+def impact_loss_workspace_status(workspace: torch.Tensor, stream=None) -> int:
+    """The workspace's error word (0 = every bounded wait of the loss kernels completed); synchronises."""
+    flag = _i32(-1)
+    _check(load_library().impact_loss_workspace_status(workspace.data_ptr(), workspace.numel() * workspace.element_size(),
+                                                       ctypes.byref(flag), _stream(stream)),
+           "impact_loss_workspace_status")
+    return flag.value
 
 
 def new_workspace(B: int, T: int, device="cuda") -> torch.Tensor:

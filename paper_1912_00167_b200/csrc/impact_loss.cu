@@ -99,133 +99,230 @@ __device__ __forceinline__ TileRows tile_rows(const TileGeometry& g, long long c
 // ------------------------------------------------------------------------------------------
 // Categorical policy
 // ------------------------------------------------------------------------------------------
+// Element access for slabs that keep their storage type in shared memory.
+template <typename ST> struct Elem;
+template <> struct Elem<float> {
+    static constexpr int kPerWord = 1;
+    static __device__ __forceinline__ float ld(const unsigned char* slab, int i) { return reinterpret_cast<const float*>(slab)[i]; }
+    static __device__ __forceinline__ void st(unsigned char* slab, int i, float x) { reinterpret_cast<float*>(slab)[i] = x; }
+};
+template <> struct Elem<__nv_bfloat16> {
+    static constexpr int kPerWord = 2;
+    static __device__ __forceinline__ float ld(const unsigned char* slab, int i) {
+        return __uint_as_float((uint32_t)reinterpret_cast<const unsigned short*>(slab)[i] << 16);
+    }
+    static __device__ __forceinline__ void st(unsigned char* slab, int i, float x) {
+        reinterpret_cast<__nv_bfloat16*>(slab)[i] = __float2bfloat16_rn(x);
+    }
+};
+
+// Any action count (runtime A): the same tile protocol as the compile-time kernel below --
+// bulk copies in, one thread per step, bulk copy out -- but rows stay in shared memory and
+// are walked element by element in three passes.  The slabs keep their dense layout, so for
+// row pitches that are a multiple of the bank width every thread would hit the same bank;
+// instead thread r starts its walk at column (r * step) mod A and wraps, which spreads a
+// warp's accesses over all banks without padding (order is irrelevant to max and sum).
 template <typename LT, typename GT, int NT>
 __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatParams p) {
     grid_dependency_wait();
-    extern __shared__ __align__(16) float smem[];
-    float* const sl = smem;                          // learner rows, then gradient rows
-    float* const st = smem + (size_t)NT * p.As;      // target rows
+    constexpr float kLog2e = 1.4426950408889634f;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const int A = p.A;
+    const int in_row = A * (int)sizeof(LT), out_row = A * (int)sizeof(GT);
+    unsigned char* const s0 = smem_raw;                // learner logits
+    unsigned char* const s1 = smem_raw + NT * in_row;  // target logits
+    unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : smem_raw + 2 * NT * in_row;  // gradients
+    __shared__ __align__(8) uint64_t bar;
     __shared__ float2 warp_agg[NT / 32];
     __shared__ float red[NT / 32][8];
     __shared__ float carry_s;
+    __shared__ int is_last_s;
 
     const int tid = threadIdx.x;
-    const int A = p.A, As = p.As;
     const LossScalars k = p.k;
     const TileGeometry g = p.geo;
     const LT* const zl = static_cast<const LT*>(p.learner_logits);
     const LT* const zt = static_cast<const LT*>(p.target_logits);
     GT* const dz = static_cast<GT*>(p.dlogits);
     const bool want_kl = (k.kl_coef != 0.0f);
+    // first column of this thread's walk (see above): one storage word per row of skew when the
+    // row pitch in words is even
+    const int words = (A * (int)sizeof(LT)) / 4;
+    const int rot = ((A * (int)sizeof(LT)) % 4 == 0 && words % 2 == 0) ? (tid * Elem<LT>::kPerWord) % A : 0;
 
-    float acc[dev::kNumSums];
+    if (tid == 0) {
+        dev::mbarrier_init(&bar, 1);
+        is_last_s = 0;
+    }
+    __syncthreads();
+    uint32_t parity = 0;
+
+    float acc[dev::kNumSums], tsum[dev::kNumSums];
 #pragma unroll
-    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = 0.0f;
+    for (int j = 0; j < dev::kNumSums; ++j) acc[j] = tsum[j] = 0.0f;
 
     for (long long chunk = blockIdx.x; chunk < g.nchunks; chunk += gridDim.x) {
         float carry = 0.0f;
         for (int tile = g.ntiles - 1; tile >= 0; --tile) {
+            const bool final_tile = (tile == 0) && (chunk + gridDim.x >= g.nchunks);
             const TileRows tr = tile_rows<NT>(g, chunk, tile);
             const long long base = tr.row0 * A;
-            const int nelem = tr.nrows * A;
-            __syncthreads();  // the previous tile's rows, sums and carry have been consumed
-            dev::stage_slab<LT, NT>(sl, zl, base, nelem, A, As);
-            dev::stage_slab<LT, NT>(st, zt, base, nelem, A, As);
-            __syncthreads();
+            const LT* const gl = zl + base;
+            const LT* const gt = zt + base;
+            GT* const gd = dz + base;
+            const uint32_t in_bytes = (uint32_t)(tr.nrows * in_row), out_bytes = (uint32_t)(tr.nrows * out_row);
+            const bool bulk_in = (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | in_bytes) & 15u) == 0);
+            const bool bulk_out = (((reinterpret_cast<uintptr_t>(gd) | out_bytes) & 15u) == 0);
+            if (bulk_in) {
+                if (tid == 0) {
+                    dev::mbarrier_expect_tx(&bar, 2 * in_bytes);
+                    dev::bulk_load(s0, gl, in_bytes, &bar);
+                    dev::bulk_load(s1, gt, in_bytes, &bar);
+                }
+            } else {  // ragged or unaligned slab: plain element copies
+                const int nelem = tr.nrows * A;
+                for (int e = tid; e < nelem; e += NT) {
+                    reinterpret_cast<LT*>(s0)[e] = gl[e];
+                    reinterpret_cast<LT*>(s1)[e] = gt[e];
+                }
+            }
 
             const bool active = tid < tr.nrows;
             const long long row = tr.row0 + tid;
-            float* const rl = sl + tid * As;
-            const float* const rt = st + tid * As;
             dev::StepIn s;
-            float fa = 1.0f, fb = 0.0f;  // identity map for idle threads
-            float lse_l = 0.0f, lse_t = 0.0f, ent = 0.0f, kl = 0.0f;
             int a = 0;
-            bool truncated = false;
             if (active) {
                 long long b, t;
                 if (g.ntiles > 1) { b = chunk; t = (long long)tile * NT + tid; }
+                else if (g.G == 1) { b = chunk; t = tid; }
                 else { const int q = tid / (int)g.T; b = chunk * g.G + q; t = tid - q * (int)g.T; }
                 a = p.actions[row];
                 a = a < 0 ? 0 : (a >= A ? A - 1 : a);
-                // log-softmax of the target row
-                float m = rt[0];
-                for (int j = 1; j < A; ++j) m = fmaxf(m, rt[j]);
-                float sum = 0.0f;
-                for (int j = 0; j < A; ++j) sum += expf(rt[j] - m);
-                lse_t = m + logf(sum);
-                s.l_target = rt[a] - lse_t;
-                // log-softmax and entropy of the learner row: H = ln S - sum e_j (z_j - m) / S
-                m = rl[0];
-                for (int j = 1; j < A; ++j) m = fmaxf(m, rl[j]);
-                sum = 0.0f;
-                float sez = 0.0f;
-                for (int j = 0; j < A; ++j) {
-                    const float d = rl[j] - m;
-                    const float e = expf(d);
-                    sum += e;
-                    sez = fmaf(e, d, sez);
-                }
-                const float ls = logf(sum);
-                lse_l = m + ls;
-                ent = ls - sez / sum;
-                s.l_theta = rl[a] - lse_l;
-                if (want_kl) {
-                    for (int j = 0; j < A; ++j) {
-                        const float lpt = rt[j] - lse_t;
-                        kl = fmaf(expf(lpt), lpt - (rl[j] - lse_l), kl);
-                    }
-                }
                 s.l_worker = p.worker_logp[row];
                 s.reward = p.rewards[row];
                 s.discount = p.discounts[row];
                 s.value = p.values[row];
                 s.last_step = (t == g.T - 1);
                 s.value_next = s.last_step ? p.bootstrap[b] : p.values[row + 1];
-                asm volatile("" ::: "memory");
+            }
+            if (bulk_in) {
+                if (tid < 32) {
+                    if (!dev::mbarrier_wait(&bar, parity)) atomicExch(p.counter + 1, 1u);
+                }
+                parity ^= 1u;
+            }
+            __syncthreads();
+
+            const int r0 = tid * A;  // first element of this thread's row
+            float fa = 1.0f, fb = 0.0f;
+            float m2_l = 0.0f, ln_s = 0.0f, inv_s = 0.0f, lse_t = 0.0f, ent = 0.0f, kl = 0.0f;
+            bool truncated = false;
+            if (active) {
+                // target row: log-sum-exp
+                float m = Elem<LT>::ld(s1, r0 + rot);
+                for (int j = 1, c = rot; j < A; ++j) {
+                    if (++c == A) c = 0;
+                    m = fmaxf(m, Elem<LT>::ld(s1, r0 + c));
+                }
+                float sum = 0.0f;
+                const float nm2 = -m * kLog2e;
+                for (int j = 0, c = rot; j < A; ++j) {
+                    sum += dev::exp2_fast(fmaf(Elem<LT>::ld(s1, r0 + c), kLog2e, nm2));
+                    if (++c == A) c = 0;
+                }
+                lse_t = m + __logf(sum);
+                s.l_target = Elem<LT>::ld(s1, r0 + a) - lse_t;
+                // learner row: log-sum-exp and entropy, H = (m + ln S) - sum_j e_j z_j / S
+                m = Elem<LT>::ld(s0, r0 + rot);
+                for (int j = 1, c = rot; j < A; ++j) {
+                    if (++c == A) c = 0;
+                    m = fmaxf(m, Elem<LT>::ld(s0, r0 + c));
+                }
+                m2_l = m * kLog2e;
+                sum = 0.0f;
+                float sez = 0.0f;
+                for (int j = 0, c = rot; j < A; ++j) {
+                    const float z = Elem<LT>::ld(s0, r0 + c);
+                    const float e = dev::exp2_fast(fmaf(z, kLog2e, -m2_l));
+                    sum += e;
+                    sez = fmaf(e, z, sez);
+                    if (++c == A) c = 0;
+                }
+                ln_s = __logf(sum);
+                inv_s = __frcp_rn(sum);
+                ent = (m + ln_s) - sez * inv_s;
+                s.l_theta = (Elem<LT>::ld(s0, r0 + a) - m) - ln_s;
+                if (want_kl) {
+                    const float lse_l = m + ln_s;
+                    for (int j = 0, c = rot; j < A; ++j) {
+                        const float lpt = Elem<LT>::ld(s1, r0 + c) - lse_t;
+                        kl = fmaf(dev::exp2_fast(lpt * kLog2e), lpt - (Elem<LT>::ld(s0, r0 + c) - lse_l), kl);
+                        if (++c == A) c = 0;
+                    }
+                }
                 truncated = dev::recursion_map(s, k, fa, fb);
             }
             const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
             if (tid == 0) carry_s = adv;
 
-            float sums[dev::kNumSums];
-#pragma unroll
-            for (int j = 0; j < dev::kNumSums; ++j) sums[j] = 0.0f;
+            float surr = 0.0f, ratio = 0.0f, wpg = 0.0f;
+            bool clipped = false;
             if (active) {
-                float surr, ratio;
-                bool clipped;
-                const float wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
+                wpg = dev::surrogate(s, k, adv, surr, ratio, clipped);
+                tsum[0] += surr;
+                tsum[1] = fmaf(0.5f * adv, adv, tsum[1]);
+                tsum[2] += ent;
+                tsum[3] += kl;
+                tsum[4] += clipped ? 1.0f : 0.0f;
+                tsum[5] += truncated ? 1.0f : 0.0f;
+                tsum[6] += ratio;
+            }
+            unsigned int ticket = 0;
+            if (final_tile) {
+                dev::block_sums_stage1<NT>(tsum, red);
+                __syncthreads();
+                if (tid == 0) {
+                    dev::block_sums_stage2<NT>(acc, red);
+                    ticket = dev::publish_block_sums(acc, p.partials, p.counter);
+                }
+            }
+            if (active) {
                 // d total / d logit_j = [ wpg (pi_j - 1[j=a]) + ent_coef pi_j (lp_j + H)
                 //                         + kl_coef (pi_j - pi_target_j) ] / M
                 const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = k.kl_coef * k.inv_M;
-                for (int j = 0; j < A; ++j) {
-                    const float lp = rl[j] - lse_l;
-                    const float pi = expf(lp);
-                    float gj = pi * fmaf(ce, lp + ent, w1);
-                    if (want_kl) gj = fmaf(ck, pi - expf(rt[j] - lse_t), gj);
-                    rl[j] = gj;
+                const float h_off = ent - (m2_l * 0.6931471805599453f + ln_s);
+                const float nlt2 = -lse_t * kLog2e;
+                for (int j = 0, c = rot; j < A; ++j) {
+                    const float z = Elem<LT>::ld(s0, r0 + c);
+                    const float pi = dev::exp2_fast(fmaf(z, kLog2e, -m2_l)) * inv_s;
+                    float gj = pi * fmaf(ce, z + h_off, w1);
+                    if (want_kl) gj = fmaf(ck, pi - dev::exp2_fast(fmaf(Elem<LT>::ld(s1, r0 + c), kLog2e, nlt2)), gj);
+                    if (c == a) gj -= w1;
+                    Elem<GT>::st(so, r0 + c, gj);
+                    if (++c == A) c = 0;
                 }
-                rl[a] -= w1;
                 p.dvalues[row] = -k.vf_coef * k.inv_M * adv;  // V - Vhat = -A
                 if (p.vtarget) p.vtarget[row] = s.value + adv;
                 if (p.advantage) p.advantage[row] = adv;
-                sums[0] = surr;
-                sums[1] = 0.5f * adv * adv;
-                sums[2] = ent;
-                sums[3] = kl;
-                sums[4] = clipped ? 1.0f : 0.0f;
-                sums[5] = truncated ? 1.0f : 0.0f;
-                sums[6] = ratio;
             }
-            dev::block_sums_stage1<NT>(sums, red);
+            if (bulk_out) dev::fence_async_shared();
+            if (tid == 0 && final_tile) is_last_s = (ticket == gridDim.x - 1) ? 1 : 0;
             __syncthreads();
             carry = carry_s;
-            dev::unstage_slab<GT, NT>(dz, sl, base, nelem, A, As);
-            dev::block_sums_stage2<NT>(acc, red);
+            if (bulk_out) {
+                if (tid == 0) {
+                    dev::bulk_store(gd, so, out_bytes);
+                    if (!final_tile) dev::bulk_store_wait_read();
+                }
+            } else {
+                const int nelem = tr.nrows * A;
+                for (int i = tid; i < nelem; i += NT) gd[i] = reinterpret_cast<const GT*>(so)[i];
+            }
+            if (!final_tile) __syncthreads();
         }
     }
-    dev::finish_loss_terms<NT>(acc, p.partials, p.counter, p.loss_terms, k,
-                               (double)g.B * (double)g.T);
+    if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k, (double)g.B * (double)g.T);
+    if (tid == 0) dev::bulk_store_wait_read();
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1025,6 +1122,17 @@ constexpr size_t kCounterBytes = 256; // counter lives in its own 256-byte line 
 
 int pad_odd(int w) { return (w & 1) ? w : w + 1; }
 
+// Shared memory of the runtime-width categorical kernel: two input slabs, and a gradient slab
+// of its own when gradients and logits differ in element size.
+size_t generic_categorical_smem(int nt, int A, size_t in_elem, size_t out_elem) {
+    return (size_t)nt * A * (2 * in_elem + (in_elem == out_elem ? 0 : out_elem));
+}
+int pick_nt_categorical(int A, size_t in_elem, size_t out_elem, size_t budget) {
+    for (int nt : {128, 64})
+        if (generic_categorical_smem(nt, A, in_elem, out_elem) <= budget) return nt;
+    return 32;
+}
+
 // Threads per block = rows per tile: as many as keep a tile's staged slabs within
 // `budget` bytes of shared memory, so that several blocks stay resident per SM.
 int pick_nt(int width_padded, int n_slabs, size_t budget) {
@@ -1103,7 +1211,7 @@ int32_t grid_for(Kernel kernel, int nt, size_t smem, long long nchunks, const De
 template <typename LT, typename GT, int NT>
 int32_t launch_categorical(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
     auto kernel = impact_loss_categorical_kernel<LT, GT, NT>;
-    const size_t smem = (size_t)2 * NT * p.As * sizeof(float);
+    const size_t smem = generic_categorical_smem(NT, p.A, sizeof(LT), sizeof(GT));
     int grid = 0;
     int32_t st = grid_for(kernel, NT, smem, p.geo.nchunks, di, &grid);
     if (st != IMPACT_OK) return st;
@@ -1144,6 +1252,12 @@ int32_t dispatch_reg(const CatParams& p, const DeviceInfo* di, cudaStream_t stre
     }
 }
 
+// Steps per tile of the kernel that run_categorical picks for this call.
+int categorical_tile_rows(int A, bool logits_bf16, bool grads_bf16) {
+    if (has_reg_kernel(A)) return kRegTileRows;
+    return pick_nt_categorical(A, logits_bf16 ? 2 : 4, grads_bf16 ? 2 : 4, 72 * 1024);
+}
+
 // Picks the kernel for a categorical call: the register-resident one where it exists, else
 // the generic one.  `p` arrives complete except for As and geo.
 int32_t run_categorical(CatParams& p, int64_t B, int64_t T, bool logits_bf16, bool grads_bf16,
@@ -1156,8 +1270,8 @@ int32_t run_categorical(CatParams& p, int64_t B, int64_t T, bool logits_bf16, bo
         if (logits_bf16 && !grads_bf16) return dispatch_reg<__nv_bfloat16, float>(p, di, s);
         return dispatch_reg<__nv_bfloat16, __nv_bfloat16>(p, di, s);
     }
-    p.As = pad_odd(p.A);
-    const int nt = pick_nt(p.As, 2, 72 * 1024);
+    p.As = p.A;
+    const int nt = categorical_tile_rows(p.A, logits_bf16, grads_bf16);
     p.geo = make_geometry(B, T, nt);
     if (!logits_bf16 && !grads_bf16) return dispatch_nt<float, float>(p, nt, di, s);
     if (!logits_bf16 && grads_bf16) return dispatch_nt<float, __nv_bfloat16>(p, nt, di, s);
@@ -1203,6 +1317,19 @@ extern "C" size_t impact_loss_workspace_bytes(int64_t B, int64_t T) {
 extern "C" int32_t impact_loss_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
     if (!workspace || !aligned16(workspace) || workspace_bytes == 0) return IMPACT_ERR_INVALID_ARG;
     IMPACT_CUDA_TRY(cudaMemsetAsync(workspace, 0, workspace_bytes, static_cast<cudaStream_t>(stream)));
+    return IMPACT_OK;
+}
+
+extern "C" int32_t impact_loss_workspace_status(const void* workspace, size_t workspace_bytes, int32_t* flag_out,
+                                                void* stream) {
+    if (!workspace || !flag_out || !aligned16(workspace)) return IMPACT_ERR_INVALID_ARG;
+    if (workspace_bytes < impact_loss_workspace_bytes(1, 1)) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const char* word = static_cast<const char*>(workspace) + (size_t)kMaxGridBlocks * 8 * sizeof(float) + sizeof(unsigned int);
+    unsigned int flag = 0;
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(&flag, word, sizeof(flag), cudaMemcpyDeviceToHost, s));
+    IMPACT_CUDA_TRY(cudaStreamSynchronize(s));
+    *flag_out = (int32_t)flag;
     return IMPACT_OK;
 }
 
@@ -1392,8 +1519,9 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     if (st != IMPACT_OK) return st;
     p.A = A;
     // one block's sums per tile at most: more tiles than the built-in scratch holds are refused
-    // (every kernel serving A <= 64 works on tiles of 128 steps)
-    if (make_geometry(B, T, 128).nchunks > kStaticMaxBlocks) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
+    const bool logits_bf16 = logits_dtype == IMPACT_DTYPE_BF16, grads_bf16 = coef->dlogits_dtype == IMPACT_DTYPE_BF16;
+    const int tile_rows_here = categorical_tile_rows(A, logits_bf16, grads_bf16);
+    if (make_geometry(B, T, tile_rows_here).nchunks > kStaticMaxBlocks) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
 
     const DeviceInfo* di = current_device_info();
     if (!di) return IMPACT_ERR_CUDA;

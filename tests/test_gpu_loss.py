@@ -134,6 +134,7 @@ def test_workspace_is_reusable_across_calls_and_shapes(oracle):
         got = lt.cpu().numpy()
         got[4] = ref["loss_terms"][4]  # KL is not evaluated at kl_coef = 0
         np.testing.assert_allclose(got, ref["loss_terms"], rtol=1e-4, atol=1e-7)
+    assert ip.impact_loss_workspace_status(ws) == 0  # no bounded wait ever ran out
 
 
 def test_rows_of_dlogits_sum_to_zero_at_full_size():
