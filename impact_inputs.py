@@ -38,8 +38,9 @@ class LossHyper:
     kl_coef: float = 0.0
     lam: float = 1.0
     rho_tw: float = 1.0
-    is_source: int = 0  # 0: target/worker (Section 3.1), 1: learner/worker (Section 2.2)
+    is_source: int = 0  # 0: target/worker (Section 3.1), 1: learner/worker (Section 2.2), 2: none (rho = c = 1)
     ratio_mode: int = 0  # 0: R3, 1: R1, 2: R2 (Section 4.1)
+    objective: int = 0  # 0: epsilon-clipped surrogate (Appendix E), 1: IMPALA's V-trace policy gradient (Section 2.2)
 
 
 @dataclass(frozen=True)

@@ -33,7 +33,7 @@ class _Coef(ctypes.Structure):
     _fields_ = [("vf_coef", ctypes.c_double), ("ent_coef", ctypes.c_double),
                 ("kl_coef", ctypes.c_double), ("lam", ctypes.c_double),
                 ("rho_tw", ctypes.c_double), ("is_source", ctypes.c_int32),
-                ("ratio_mode", ctypes.c_int32)]
+                ("ratio_mode", ctypes.c_int32), ("objective", ctypes.c_int32)]
 
 
 def _load():
@@ -62,7 +62,7 @@ def _ptr(a):
 
 def _coef(h) -> _Coef:
     return _Coef(float(h.vf_coef), float(h.ent_coef), float(h.kl_coef), float(h.lam),
-                 float(h.rho_tw), int(h.is_source), int(h.ratio_mode))
+                 float(h.rho_tw), int(h.is_source), int(h.ratio_mode), int(getattr(h, "objective", 0)))
 
 
 def loss_categorical(batch: dict, hyper, flip=None) -> dict:

@@ -22,8 +22,11 @@ typedef struct {
     double kl_coef;    /* eta of Algorithm 1's KL term */
     double lambda;     /* lambda of V-trace GAE-lambda (Section 3.1) */
     double rho_tw;     /* rho of the target-worker clipping (Section 3.1), beta = 1/rho */
-    int32_t is_source; /* 0: pi_target/pi_worker (Section 3.1); 1: pi_theta/pi_worker (Section 2.2) */
+    int32_t is_source; /* 0: pi_target/pi_worker (Section 3.1); 1: pi_theta/pi_worker (Section 2.2);
+                          2: no importance weights, rho = c = 1 (GAE-lambda as PPO uses it, Section 2.1) */
     int32_t ratio_mode;/* 0: R3, 1: R1, 2: R2 (Section 4.1) */
+    int32_t objective; /* 0: epsilon-clipped surrogate (Appendix E); 1: IMPALA's importance-weighted
+                          policy gradient with V-trace targets (Section 2.2, Appendix D) */
 } oracle_coef;
 
 /* log-softmax of one row: log pi(k|s) = z_k - log sum_j exp(z_j), max-shifted. */
@@ -62,12 +65,12 @@ static void trajectory_terms(const double* lth, const double* ltg, const float* 
                              double bootstrap, double rho_bar, double c_bar, double clip_eps,
                              const oracle_coef* cf, int64_t T, const int8_t* flip,
                              double* adv, double* vtarget, double* ratio, double* surr,
-                             double* pass, double* rho_trunc, double* adv_cond) {
+                             double* pass, double* rho_trunc, double* adv_cond, double* pgw) {
     double next_adv = 0.0, next_cond = 0.0;
     for (int64_t t = T - 1; t >= 0; --t) {
         double lw = (double)worker_logp[t];
         double x = (cf->is_source == 1 ? lth[t] : ltg[t]) - lw;
-        double w = exp(x);
+        double w = (cf->is_source == 2) ? 1.0 : exp(x);
         double rho = w < rho_bar ? w : rho_bar;
         double c = w < c_bar ? w : c_bar;
         double v = (double)values[t];
@@ -84,6 +87,22 @@ static void trajectory_terms(const double* lth, const double* ltg, const float* 
                     fabs(cf->lambda * g * c) * next_cond;
         adv_cond[t] = next_cond;
         next_adv = a;
+        pgw[t] = rho; /* kept for the policy-gradient objective below */
+    }
+    if (cf->objective == 1) {
+        /* IMPALA's actor update (Section 2.2; Appendix D calls it an importance-sampled vanilla
+         * policy gradient): ascend rho_t (r_t + gamma_t v_{t+1} - V(s_t)) grad log pi_theta(a_t|s_t),
+         * v the V-trace target (the bootstrap value after the last stored step).  The weight is a
+         * constant for the gradient; the reported objective is weight * log pi_theta. */
+        for (int64_t t = 0; t < T; ++t) {
+            double v_next = (t == T - 1) ? bootstrap : vtarget[t + 1];
+            double wgt = pgw[t] * ((double)rewards[t] + (double)discounts[t] * v_next - (double)values[t]);
+            ratio[t] = pgw[t];
+            pgw[t] = wgt;
+            surr[t] = wgt * lth[t];
+            pass[t] = 1.0;
+        }
+        return;
     }
     for (int64_t t = 0; t < T; ++t) {
         double lw = (double)worker_logp[t];
@@ -103,6 +122,7 @@ static void trajectory_terms(const double* lth, const double* ltg, const float* 
         if (flip && flip[t]) clipped = !clipped;
         pass[t] = clipped ? 0.0 : 1.0;
         ratio[t] = R;
+        pgw[t] = pass[t] * adv[t] * R;
     }
 }
 
@@ -134,11 +154,11 @@ int oracle_impact_loss_categorical(
     const double M = (double)B * (double)T;
     double* lp_th = (double*)malloc(sizeof(double) * (size_t)(T * A));
     double* lp_tg = (double*)malloc(sizeof(double) * (size_t)(T * A));
-    double* buf = (double*)malloc(sizeof(double) * (size_t)(T * 9));
+    double* buf = (double*)malloc(sizeof(double) * (size_t)(T * 10));
     if (!lp_th || !lp_tg || !buf) { free(lp_th); free(lp_tg); free(buf); return -1; }
     double *lth = buf, *ltg = buf + T, *adv = buf + 2 * T, *vt = buf + 3 * T,
            *ratio = buf + 4 * T, *surr = buf + 5 * T, *pass = buf + 6 * T, *rtr = buf + 7 * T,
-           *cond = buf + 8 * T;
+           *cond = buf + 8 * T, *pgw = buf + 9 * T;
     double s_surr = 0, s_val = 0, s_ent = 0, s_kl = 0, s_clip = 0, s_trunc = 0, s_ratio = 0;
 
     for (int64_t b = 0; b < B; ++b) {
@@ -155,7 +175,7 @@ int oracle_impact_loss_categorical(
         }
         trajectory_terms(lth, ltg, worker_logp + b * T, rewards + b * T, discounts + b * T,
                          values + b * T, (double)bootstrap_values[b], rho_bar, c_bar, clip_eps,
-                         cf, T, flip ? flip + b * T : NULL, adv, vt, ratio, surr, pass, rtr, cond);
+                         cf, T, flip ? flip + b * T : NULL, adv, vt, ratio, surr, pass, rtr, cond, pgw);
         for (int64_t t = 0; t < T; ++t) {
             const double* lpl = lp_th + t * A;
             const double* lpt = lp_tg + t * A;
@@ -175,7 +195,7 @@ int oracle_impact_loss_categorical(
             s_ratio += ratio[t];
             if (dlogits) {
                 double* g = dlogits + (b * T + t) * A;
-                double w = pass[t] * adv[t] * ratio[t];
+                double w = pgw[t];
                 for (int64_t k = 0; k < A; ++k) {
                     double pi = exp(lpl[k]);
                     double onehot = (k == act[t]) ? 1.0 : 0.0;
@@ -225,11 +245,11 @@ int oracle_impact_loss_gaussian(
     if (B <= 0 || T <= 0 || D <= 0 || !cf) return -1;
     const double M = (double)B * (double)T;
     const double half_log_2pi = 0.5 * log(2.0 * 3.14159265358979323846);
-    double* buf = (double*)malloc(sizeof(double) * (size_t)(T * 9));
+    double* buf = (double*)malloc(sizeof(double) * (size_t)(T * 10));
     if (!buf) return -1;
     double *lth = buf, *ltg = buf + T, *adv = buf + 2 * T, *vt = buf + 3 * T,
            *ratio = buf + 4 * T, *surr = buf + 5 * T, *pass = buf + 6 * T, *rtr = buf + 7 * T,
-           *cond = buf + 8 * T;
+           *cond = buf + 8 * T, *pgw = buf + 9 * T;
     double s_surr = 0, s_val = 0, s_ent = 0, s_kl = 0, s_clip = 0, s_trunc = 0, s_ratio = 0;
 
     for (int64_t b = 0; b < B; ++b) {
@@ -248,11 +268,11 @@ int oracle_impact_loss_gaussian(
         }
         trajectory_terms(lth, ltg, worker_logp + b * T, rewards + b * T, discounts + b * T,
                          values + b * T, (double)bootstrap_values[b], rho_bar, c_bar, clip_eps,
-                         cf, T, flip ? flip + b * T : NULL, adv, vt, ratio, surr, pass, rtr, cond);
+                         cf, T, flip ? flip + b * T : NULL, adv, vt, ratio, surr, pass, rtr, cond, pgw);
         for (int64_t t = 0; t < T; ++t) {
             int64_t o = (b * T + t) * D;
             double H = 0.0, KL = 0.0;
-            double w = pass[t] * adv[t] * ratio[t];
+            double w = pgw[t];
             for (int64_t d = 0; d < D; ++d) {
                 double mu = (double)learner_mean[o + d], ls = (double)learner_logstd[o + d];
                 double mut = (double)target_mean[o + d], lst = (double)target_logstd[o + d];

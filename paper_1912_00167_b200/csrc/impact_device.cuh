@@ -1,6 +1,6 @@
 // Device building blocks of the fused IMPACT loss kernels (sm_100a).
 //
-// Work decomposition shared by the categorical and the Gaussian kernel:
+// Work decomposition shared by all loss kernels:
 //   * one thread per time step ("row"); a block of NT threads owns a tile of up to NT
 //     consecutive rows of the row-major [B*T, width] tensors, which is one contiguous slab
 //     of global memory;
@@ -8,9 +8,11 @@
 //     long ones (T > NT) are swept tile by tile from their END backwards, because the
 //     advantage recursion runs backward in time -- one scalar carry links the tiles, so
 //     every byte is still read once;
-//   * slabs are staged into shared memory with 16-byte streaming loads and re-laid out
-//     with an odd row stride, so that thread-per-row reads are bank-conflict free;
-//   * gradients overwrite the staged rows in place and leave with 16-byte streaming stores.
+//   * slabs reach shared memory by bulk asynchronous copies (one instruction per slab) and
+//     keep their dense layout; the runtime-width Gaussian fallback instead stages them with
+//     16-byte streaming loads into rows of odd stride;
+//   * gradients overwrite the staged rows in place and leave by bulk stores;
+//   * per-block sums are published early and added by the last block to arrive.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -457,26 +459,6 @@ __device__ __noinline__ void reduce_published_sums(const float* partials, unsign
         loss_terms[6] = (float)t[5];
         loss_terms[7] = (float)t[6];
         *counter = 0u;
-    }
-}
-
-// Block sums when two of the seven are counts of a per-thread flag: five float sums by
-// shuffles, the two counts by one ballot each.
-template <int NT>
-__device__ __forceinline__ void block_sums_stage1_flags(const float (&v)[5], bool f0, bool f1, float (*red)[8]) {
-    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
-    float x[5];
-#pragma unroll
-    for (int j = 0; j < 5; ++j) x[j] = v[j];
-#pragma unroll
-    for (int off = 16; off > 0; off >>= 1) {
-#pragma unroll
-        for (int j = 0; j < 5; ++j) x[j] += __shfl_xor_sync(0xffffffffu, x[j], off);
-    }
-    const unsigned int b0 = __ballot_sync(0xffffffffu, f0), b1 = __ballot_sync(0xffffffffu, f1);
-    if (lane == 0) {
-        red[warp][0] = x[0]; red[warp][1] = x[1]; red[warp][2] = x[2]; red[warp][3] = x[3];
-        red[warp][4] = (float)__popc(b0); red[warp][5] = (float)__popc(b1); red[warp][6] = x[4];
     }
 }
 
