@@ -49,6 +49,17 @@ extern "C" {
  * uses pi_theta / pi_worker.  Either way the weights are constants for the gradient. */
 #define IMPACT_IS_TARGET_OVER_WORKER 0
 #define IMPACT_IS_LEARNER_OVER_WORKER 1
+#define IMPACT_IS_NONE 2 /* rho_t = c_t = 1 before truncation: plain GAE-lambda, as PPO uses it (Section 2.1) */
+
+/* What the policy is trained on:
+ *   CLIPPED_SURROGATE  min(R A, clip(R, 1-eps, 1+eps) A) with the ratio of `ratio_mode` (IMPACT, Section 3.1 and
+ *                      Appendix E; PPO is R2 with IMPACT_IS_NONE, Section 2.1);
+ *   VTRACE_PG          IMPALA's importance-weighted policy gradient (Section 2.2, Appendix D): the weight
+ *                      rho_t (r_t + gamma_t v_{t+1} - V_t), v the V-trace target, multiplies grad log pi_theta;
+ *                      the policy term reported is -mean(weight * log pi_theta), nothing is clipped
+ *                      (clip_eps, rho_tw and ratio_mode are ignored; IMPACT_TERM_MEAN_RATIO is mean rho_t). */
+#define IMPACT_OBJECTIVE_CLIPPED_SURROGATE 0
+#define IMPACT_OBJECTIVE_VTRACE_PG 1
 
 /* Likelihood ratio of the surrogate (Section 4.1):
  *   R3 = pi_theta / max(pi_target, pi_worker / rho_tw)   (the IMPACT objective, Section 3.1)
@@ -89,7 +100,7 @@ typedef struct impact_coefficients {
     int32_t is_source;     /* IMPACT_IS_* */
     int32_t ratio_mode;    /* IMPACT_RATIO_* */
     int32_t dlogits_dtype; /* IMPACT_DTYPE_*: storage type of the policy-gradient outputs */
-    int32_t reserved;      /* must be 0 */
+    int32_t objective;     /* IMPACT_OBJECTIVE_* */
 } impact_coefficients;
 
 /* ---- housekeeping --------------------------------------------------------------------- */

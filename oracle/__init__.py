@@ -79,14 +79,14 @@ def loss_categorical(batch: dict, hyper, flip=None) -> dict:
     fl = None if flip is None else np.ascontiguousarray(flip, dtype=np.int8)
     out = dict(loss_terms=np.zeros(8), dlogits=np.zeros((B, T, A)), dvalues=np.zeros((B, T)),
                vtarget=np.zeros((B, T)), advantage=np.zeros((B, T)), ratio=np.zeros((B, T)),
-               adv_cond=np.zeros((B, T)))
+               adv_cond=np.zeros((B, T)), pg_weight=np.zeros((B, T)))
     cf = _coef(hyper)
     rc = lib.oracle_impact_loss_categorical(
         _ptr(zl), _ptr(zt), _ptr(wl), _ptr(act), _ptr(rew), _ptr(dis), _ptr(val), _ptr(boot),
         ctypes.c_double(hyper.rho_bar), ctypes.c_double(hyper.c_bar), ctypes.c_double(hyper.clip_eps),
         ctypes.byref(cf), ctypes.c_int64(B), ctypes.c_int64(T), ctypes.c_int64(A), _ptr(fl),
         _ptr(out["loss_terms"]), _ptr(out["dlogits"]), _ptr(out["dvalues"]), _ptr(out["vtarget"]),
-        _ptr(out["advantage"]), _ptr(out["ratio"]), _ptr(out["adv_cond"]))
+        _ptr(out["advantage"]), _ptr(out["ratio"]), _ptr(out["adv_cond"]), _ptr(out["pg_weight"]))
     if rc != 0:
         raise ValueError("oracle rejected its arguments")
     return out
@@ -106,7 +106,7 @@ def loss_gaussian(batch: dict, hyper, flip=None) -> dict:
     fl = None if flip is None else np.ascontiguousarray(flip, dtype=np.int8)
     out = dict(loss_terms=np.zeros(8), dmean=np.zeros((B, T, D)), dlogstd=np.zeros((B, T, D)),
                dvalues=np.zeros((B, T)), vtarget=np.zeros((B, T)), advantage=np.zeros((B, T)),
-               ratio=np.zeros((B, T)), adv_cond=np.zeros((B, T)))
+               ratio=np.zeros((B, T)), adv_cond=np.zeros((B, T)), pg_weight=np.zeros((B, T)))
     cf = _coef(hyper)
     rc = lib.oracle_impact_loss_gaussian(
         _ptr(mu), _ptr(ls), _ptr(mut), _ptr(lst), _ptr(wl), _ptr(act), _ptr(rew), _ptr(dis),
@@ -114,7 +114,7 @@ def loss_gaussian(batch: dict, hyper, flip=None) -> dict:
         ctypes.c_double(hyper.clip_eps), ctypes.byref(cf), ctypes.c_int64(B), ctypes.c_int64(T),
         ctypes.c_int64(D), _ptr(fl), _ptr(out["loss_terms"]), _ptr(out["dmean"]), _ptr(out["dlogstd"]),
         _ptr(out["dvalues"]), _ptr(out["vtarget"]), _ptr(out["advantage"]), _ptr(out["ratio"]),
-        _ptr(out["adv_cond"]))
+        _ptr(out["adv_cond"]), _ptr(out["pg_weight"]))
     if rc != 0:
         raise ValueError("oracle rejected its arguments")
     return out

@@ -149,7 +149,8 @@ int oracle_impact_loss_categorical(
     double rho_bar, double c_bar, double clip_eps, const oracle_coef* cf,
     int64_t B, int64_t T, int64_t A, const int8_t* flip,
     double* loss_terms, double* dlogits, double* dvalues,
-    double* vtarget_out, double* advantage_out, double* ratio_out, double* adv_cond_out) {
+    double* vtarget_out, double* advantage_out, double* ratio_out, double* adv_cond_out,
+    double* pg_weight_out) {
     if (B <= 0 || T <= 0 || A <= 0 || !cf) return -1;
     const double M = (double)B * (double)T;
     double* lp_th = (double*)malloc(sizeof(double) * (size_t)(T * A));
@@ -208,6 +209,7 @@ int oracle_impact_loss_categorical(
             if (advantage_out) advantage_out[b * T + t] = adv[t];
             if (ratio_out) ratio_out[b * T + t] = ratio[t];
             if (adv_cond_out) adv_cond_out[b * T + t] = cond[t];
+            if (pg_weight_out) pg_weight_out[b * T + t] = pgw[t];
         }
     }
     if (loss_terms) {
@@ -241,7 +243,8 @@ int oracle_impact_loss_gaussian(
     const float* bootstrap_values, double rho_bar, double c_bar, double clip_eps,
     const oracle_coef* cf, int64_t B, int64_t T, int64_t D, const int8_t* flip,
     double* loss_terms, double* dmean, double* dlogstd, double* dvalues,
-    double* vtarget_out, double* advantage_out, double* ratio_out, double* adv_cond_out) {
+    double* vtarget_out, double* advantage_out, double* ratio_out, double* adv_cond_out,
+    double* pg_weight_out) {
     if (B <= 0 || T <= 0 || D <= 0 || !cf) return -1;
     const double M = (double)B * (double)T;
     const double half_log_2pi = 0.5 * log(2.0 * 3.14159265358979323846);
@@ -307,6 +310,7 @@ int oracle_impact_loss_gaussian(
             if (advantage_out) advantage_out[b * T + t] = adv[t];
             if (ratio_out) ratio_out[b * T + t] = ratio[t];
             if (adv_cond_out) adv_cond_out[b * T + t] = cond[t];
+            if (pg_weight_out) pg_weight_out[b * T + t] = pgw[t];
         }
     }
     if (loss_terms) {

@@ -18,7 +18,8 @@ LIB_PATH = os.path.join(_PKG, "libimpact.so")
 OK = 0
 ERR_INVALID_ARG, ERR_UNSUPPORTED, ERR_WORKSPACE_TOO_SMALL, ERR_EMPTY, ERR_FULL, ERR_CUDA = -1, -2, -3, -4, -5, -6
 DTYPE_F32, DTYPE_BF16 = 0, 1
-IS_TARGET_OVER_WORKER, IS_LEARNER_OVER_WORKER = 0, 1
+IS_TARGET_OVER_WORKER, IS_LEARNER_OVER_WORKER, IS_NONE = 0, 1, 2
+OBJECTIVE_CLIPPED_SURROGATE, OBJECTIVE_VTRACE_PG = 0, 1
 RATIO_R3, RATIO_R1, RATIO_R2 = 0, 1, 2
 SAMPLE_UNIFORM, SAMPLE_ROUND_ROBIN = 0, 1
 SRC_DEVICE, SRC_HOST = 0, 1
@@ -46,7 +47,7 @@ class impact_coefficients(ctypes.Structure):
     _fields_ = [("vf_coef", ctypes.c_float), ("ent_coef", ctypes.c_float), ("kl_coef", ctypes.c_float),
                 ("lambda_", ctypes.c_float), ("rho_tw", ctypes.c_float), ("is_source", ctypes.c_int32),
                 ("ratio_mode", ctypes.c_int32), ("dlogits_dtype", ctypes.c_int32),
-                ("reserved", ctypes.c_int32)]
+                ("objective", ctypes.c_int32)]
 
 
 class impact_loss_call(ctypes.Structure):
@@ -173,10 +174,11 @@ class Coefficients:
     rho_tw: float = 1.0
     is_source: int = IS_TARGET_OVER_WORKER
     ratio_mode: int = RATIO_R3
+    objective: int = OBJECTIVE_CLIPPED_SURROGATE
 
     def c_struct(self, dlogits_dtype: int) -> impact_coefficients:
         return impact_coefficients(self.vf_coef, self.ent_coef, self.kl_coef, self.lam, self.rho_tw,
-                                   int(self.is_source), int(self.ratio_mode), int(dlogits_dtype), 0)
+                                   int(self.is_source), int(self.ratio_mode), int(dlogits_dtype), int(self.objective))
 
 
 def impact_loss_workspace_bytes(B: int, T: int) -> int:

@@ -230,8 +230,9 @@ __device__ __forceinline__ void unstage_slab(ST* __restrict__ dst, const float* 
 // (A_i = delta_i + (lambda gamma_i c_i) A_{i+1}).  Returns A_i = f_i(f_{i+1}(... f_{NT-1}(carry))).
 // Affine maps compose associatively, so the recursion is a scan: shuffles inside a warp,
 // one shared-memory hop across warps.  Contains one __syncthreads().
+// `next` receives A_{i+1}, the value the thread's own map was applied to (the carry for the last row).
 template <int NT>
-__device__ __forceinline__ float suffix_affine_scan(float a, float b, float carry, float2* warp_agg) {
+__device__ __forceinline__ float suffix_affine_scan(float a, float b, float carry, float2* warp_agg, float& next) {
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
 #pragma unroll
     for (int off = 1; off < 32; off <<= 1) {
@@ -250,7 +251,10 @@ __device__ __forceinline__ float suffix_affine_scan(float a, float b, float carr
         const float2 g = warp_agg[w];
         x = fmaf(g.x, x, g.y);
     }
-    return fmaf(a, x, b);
+    const float result = fmaf(a, x, b);
+    const float below = __shfl_down_sync(0xffffffffu, result, 1);
+    next = (lane == 31) ? x : below;
+    return result;
 }
 
 // Scalars of the loss that the kernels need; filled on the host.
@@ -258,14 +262,17 @@ struct LossScalars {
     float rho_bar, c_bar, clip_lo, clip_hi;
     float vf_coef, ent_coef, kl_coef, lambda_, log_rho_tw;
     float inv_M;
-    int is_source, ratio_mode;
+    int is_source, ratio_mode, objective;
 };
 
 // Per-step quantities once the three log-probabilities are known.
 struct StepIn {
-    float l_theta, l_target, l_worker;
+    float l_theta, l_target, l_worker;  // may all be shifted by one common amount ...
+    float l_shift = 0.0f;               // ... which is this: l_theta + l_shift is the true log-probability
     float reward, discount, value, value_next;
     bool last_step;  // t == T-1: the trace stops, V_{t+1} is the bootstrap value
+    float rho = 0.0f;       // truncated importance weight of the step (set by recursion_map)
+    float adv_next = 0.0f;  // A_{t+1} (set from the scan)
 };
 
 // Truncated importance weights and the affine map of the advantage recursion
@@ -274,10 +281,11 @@ struct StepIn {
 // multiply-then-exp2 form stays within ~3e-7 relative of the correctly rounded result.
 __device__ __forceinline__ float exp_of_logratio(float x) { return exp2_fast(x * 1.4426950408889634f); }
 
-__device__ __forceinline__ bool recursion_map(const StepIn& s, const LossScalars& k, float& a, float& b) {
-    const float x = (k.is_source ? s.l_theta : s.l_target) - s.l_worker;
-    const float w = exp_of_logratio(x);
+__device__ __forceinline__ bool recursion_map(StepIn& s, const LossScalars& k, float& a, float& b) {
+    const float x = (k.is_source == 1 ? s.l_theta : s.l_target) - s.l_worker;
+    const float w = (k.is_source == 2) ? 1.0f : exp_of_logratio(x);  // 2: plain GAE, no importance weights
     const float rho = fminf(k.rho_bar, w);
+    s.rho = rho;
     const float c = fminf(k.c_bar, w);
     b = rho * (s.reward + s.discount * s.value_next - s.value);
     a = s.last_step ? 0.0f : k.lambda_ * s.discount * c;
@@ -288,6 +296,16 @@ __device__ __forceinline__ bool recursion_map(const StepIn& s, const LossScalars
 // adv * R of the policy-gradient term (0 where the clip removes it).
 __device__ __forceinline__ float surrogate(const StepIn& s, const LossScalars& k, float adv,
                                            float& surr, float& ratio, bool& clipped) {
+    if (k.objective == 1) {
+        // IMPALA's actor update (Section 2.2): weight rho_t (r_t + gamma_t v_{t+1} - V_t) on
+        // grad log pi_theta, v the V-trace target V + A (the bootstrap value after the last step)
+        const float v_next = s.value_next + (s.last_step ? 0.0f : s.adv_next);
+        const float w = s.rho * (s.reward + s.discount * v_next - s.value);
+        surr = w * (s.l_theta + s.l_shift);
+        ratio = s.rho;
+        clipped = false;
+        return w;
+    }
     float d;
     if (k.ratio_mode == 1) d = s.l_target;
     else if (k.ratio_mode == 2) d = s.l_worker;

@@ -262,7 +262,7 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
                 }
                 truncated = dev::recursion_map(s, k, fa, fb);
             }
-            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
+            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg, s.adv_next);
             if (tid == 0) carry_s = adv;
 
             float surr = 0.0f, ratio = 0.0f, wpg = 0.0f;
@@ -686,7 +686,7 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
                 asm volatile("" ::: "memory");
                 truncated = dev::recursion_map(s, k, fa, fb);
             }
-            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
+            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg, s.adv_next);
             if (tid == 0) carry_s = adv;
 
             float surr = 0.0f, ratio = 0.0f, wpg = 0.0f;
@@ -856,6 +856,7 @@ __global__ void __launch_bounds__(NT) impact_loss_gaussian_kernel(const GaussPar
                 s.l_theta = (float)(lth - (double)lw);
                 s.l_target = (float)(ltg - (double)lw);
                 s.l_worker = 0.0f;
+                s.l_shift = lw;
                 s.reward = p.rewards[row];
                 s.discount = p.discounts[row];
                 s.value = p.values[row];
@@ -864,7 +865,7 @@ __global__ void __launch_bounds__(NT) impact_loss_gaussian_kernel(const GaussPar
                 asm volatile("" ::: "memory");
                 truncated = dev::recursion_map(s, k, fa, fb);
             }
-            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
+            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg, s.adv_next);
             if (tid == 0) carry_s = adv;
 
             float sums[dev::kNumSums];
@@ -1037,9 +1038,10 @@ __global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kern
                 s.l_theta = (float)(lth - shift);
                 s.l_target = (float)(ltg - shift);
                 s.l_worker = 0.0f;
+                s.l_shift = lw;
                 truncated = dev::recursion_map(s, k, fa, fb);
             }
-            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg);
+            const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg, s.adv_next);
             if (tid == 0) carry_s = adv;
 
             float surr = 0.0f, ratio = 0.0f, wpg = 0.0f;
@@ -1164,9 +1166,10 @@ int32_t fill_scalars(LossScalars& k, float rho_bar, float c_bar, float clip_eps,
                      const impact_coefficients* coef, int64_t B, int64_t T) {
     if (bad_scalar(rho_bar) || bad_scalar(c_bar) || bad_scalar(clip_eps)) return IMPACT_ERR_INVALID_ARG;
     if (!(coef->rho_tw > 0.0f) || !isfinite(coef->vf_coef) || !isfinite(coef->ent_coef) ||
-        !isfinite(coef->kl_coef) || !isfinite(coef->lambda_) || coef->reserved != 0)
+        !isfinite(coef->kl_coef) || !isfinite(coef->lambda_))
         return IMPACT_ERR_INVALID_ARG;
-    if (coef->is_source != IMPACT_IS_TARGET_OVER_WORKER && coef->is_source != IMPACT_IS_LEARNER_OVER_WORKER)
+    if (coef->is_source < IMPACT_IS_TARGET_OVER_WORKER || coef->is_source > IMPACT_IS_NONE) return IMPACT_ERR_INVALID_ARG;
+    if (coef->objective != IMPACT_OBJECTIVE_CLIPPED_SURROGATE && coef->objective != IMPACT_OBJECTIVE_VTRACE_PG)
         return IMPACT_ERR_INVALID_ARG;
     if (coef->ratio_mode < IMPACT_RATIO_R3 || coef->ratio_mode > IMPACT_RATIO_R2) return IMPACT_ERR_INVALID_ARG;
     k.rho_bar = rho_bar;
@@ -1181,6 +1184,7 @@ int32_t fill_scalars(LossScalars& k, float rho_bar, float c_bar, float clip_eps,
     k.inv_M = (float)(1.0 / ((double)B * (double)T));
     k.is_source = coef->is_source;
     k.ratio_mode = coef->ratio_mode;
+    k.objective = coef->objective;
     return IMPACT_OK;
 }
 

@@ -30,7 +30,7 @@ def to_coef(h: ii.LossHyper):
     import paper_1912_00167_b200 as ip
     return ip.Coefficients(rho_bar=h.rho_bar, c_bar=h.c_bar, clip_eps=h.clip_eps, vf_coef=h.vf_coef,
                            ent_coef=h.ent_coef, kl_coef=h.kl_coef, lam=h.lam, rho_tw=h.rho_tw,
-                           is_source=h.is_source, ratio_mode=h.ratio_mode)
+                           is_source=h.is_source, ratio_mode=h.ratio_mode, objective=h.objective)
 
 
 def run_gpu_categorical(batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, extra=True):
@@ -93,7 +93,7 @@ def logp_scale(batch):
 
 def compare(gpu, ref, ref_flipped, near, M, grad_keys, kl_coef, sens, vf_coef, rtol=RTOL_ELEM, atol=ATOL_ELEM,
             rtol_scalar=RTOL_SCALAR, atol_scalar=ATOL_SCALAR, cond=COND_ADV, min_literal=0.995, scale_l=1.0,
-            kl_always=False):
+            kl_always=False, term_tol=None):
     """Element-by-element comparison.
 
     Bar per element: |gpu - oracle| <= rtol |oracle| + atol + s * cond * S_t, where the last
@@ -118,6 +118,8 @@ def compare(gpu, ref, ref_flipped, near, M, grad_keys, kl_coef, sens, vf_coef, r
             extra = abs(vf_coef) * adv_tol
         else:
             extra = adv_tol
+        if term_tol is not None and key in term_tol:
+            extra = extra + term_tol[key]
         err = np.abs(got - want)
         literal = err <= rtol * np.abs(want) + atol
         ok = err <= rtol * np.abs(want) + atol + extra
@@ -163,6 +165,15 @@ def _policy_sensitivity(loss_fn, batch, h, keys, M, flip):
     return out
 
 
+def _vtrace_pg_bounds(ref, sens):
+    """For the V-trace policy-gradient objective the weight of grad log pi is
+    rho_t (r_t + gamma_t (V_{t+1} + A_{t+1}) - V_t): its rounding is bounded through the largest condition sum
+    of the trajectory, and `sens` is |d (M * gradient) / d weight| per element."""
+    ref = dict(ref)
+    ref["adv_cond"] = np.broadcast_to(ref["adv_cond"].max(axis=1, keepdims=True), ref["adv_cond"].shape).copy()
+    return ref, sens
+
+
 def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, **tol):
     h = f32_hyper(h)
     if logits_dtype == torch.bfloat16:
@@ -174,6 +185,18 @@ def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtyp
     ref_flipped = oracle.loss_categorical(batch, h, flip=near.astype(np.int8)) if near.any() else None
     gpu = run_gpu_categorical(batch, h, logits_dtype, dlogits_dtype)
     M = batch["rewards"].size
+    if h.objective == 1:
+        from scipy.special import softmax
+        pi = softmax(batch["learner_logits"].astype(np.float64), axis=-1)
+        onehot = np.eye(pi.shape[-1])[batch["actions"]]
+        gpu_ = gpu  # (unchanged) advantage / vtarget keep their own per-step bound
+        adv_ref = ref
+        ref2, sens = _vtrace_pg_bounds(ref, {"dlogits": np.abs(onehot - pi)})
+        rep = compare({k_: v for k_, v in gpu.items() if k_ in ("dlogits", "loss_terms")}, ref2, None, near & False, M,
+                      ["dlogits"], h.kl_coef, sens, h.vf_coef, scale_l=logp_scale(batch), **tol)
+        compare({k_: v for k_, v in gpu.items() if k_ != "dlogits"}, adv_ref, None, near & False, M, [], h.kl_coef,
+                {}, h.vf_coef, scale_l=logp_scale(batch), **tol)
+        return rep
     sens = _policy_sensitivity(oracle.loss_categorical, batch, h, ["dlogits"], M,
                                near.astype(np.int8) if near.any() else None)
     return compare(gpu, ref, ref_flipped, near, M, ["dlogits"], h.kl_coef, sens, h.vf_coef,
@@ -183,10 +206,25 @@ def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtyp
 def check_gaussian(oracle, batch, h, **tol):
     h = f32_hyper(h)
     ref = oracle.loss_gaussian(batch, h)
+    # d/dlogstd carries weight * (z^2 - 1): where z^2 is near 1 the difference cancels, so its rounding is
+    # bounded relative to weight * (z^2 + 1), a few fp32 roundoffs of the terms themselves
+    a_, mu_ = batch["actions"].astype(np.float64), batch["learner_mean"].astype(np.float64)
+    z2_ = (a_ - mu_) ** 2 / np.exp(2.0 * batch["learner_logstd"].astype(np.float64))
+    tol = dict(tol)
+    tol["term_tol"] = {"dlogstd": 1e-6 * logp_scale(batch) * np.abs(ref["pg_weight"])[..., None] * (z2_ + 1.0)}
     near = near_clip_bound(ref, h)
     ref_flipped = oracle.loss_gaussian(batch, h, flip=near.astype(np.int8)) if near.any() else None
     gpu = run_gpu_gaussian(batch, h)
     M = batch["rewards"].size
+    if h.objective == 1:
+        a, mu = batch["actions"].astype(np.float64), batch["learner_mean"].astype(np.float64)
+        var = np.exp(2.0 * batch["learner_logstd"].astype(np.float64))
+        ref2, sens = _vtrace_pg_bounds(ref, {"dmean": np.abs(a - mu) / var, "dlogstd": np.abs((a - mu) ** 2 / var - 1.0)})
+        rep = compare({k_: v for k_, v in gpu.items() if k_ in ("dmean", "dlogstd", "loss_terms")}, ref2, None,
+                      near & False, M, ["dmean", "dlogstd"], h.kl_coef, sens, h.vf_coef, scale_l=logp_scale(batch), **tol)
+        compare({k_: v for k_, v in gpu.items() if k_ not in ("dmean", "dlogstd")}, ref, None, near & False, M, [],
+                h.kl_coef, {}, h.vf_coef, scale_l=logp_scale(batch), **tol)
+        return rep
     sens = _policy_sensitivity(oracle.loss_gaussian, batch, h, ["dmean", "dlogstd"], M,
                                near.astype(np.int8) if near.any() else None)
     return compare(gpu, ref, ref_flipped, near, M, ["dmean", "dlogstd"], h.kl_coef, sens, h.vf_coef,

@@ -42,7 +42,7 @@ def test_housekeeping_calls(lib):
 def test_struct_layout_matches_header():
     from paper_1912_00167_b200.binding import impact_coefficients
     assert ctypes.sizeof(impact_coefficients) == 36
-    assert impact_coefficients.rho_tw.offset == 16 and impact_coefficients.reserved.offset == 32
+    assert impact_coefficients.rho_tw.offset == 16 and impact_coefficients.objective.offset == 32
 
 
 def test_host_side_validation_needs_no_gpu(lib):

@@ -220,3 +220,28 @@ def test_sampled_trajectories_at_sweep_sizes(oracle, B, T, A, dtype):
     assert lt[0] == pytest.approx(lt[1] + h.vf_coef * lt[2] - h.ent_coef * lt[3] + h.kl_coef * lt[4], rel=1e-5, abs=1e-6)
     assert lt[2] == pytest.approx(0.5 * np.mean(gpu["advantage"] ** 2), rel=1e-4)
     assert 0.0 < lt[3] <= np.log(A) + 1e-5 and 0.0 <= lt[5] <= 1.0 and 0.0 <= lt[6] <= 1.0
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_baseline_objectives_categorical(oracle, idx):
+    """PPO (ratio R2, plain GAE-lambda) and IMPALA (V-trace policy gradient) on the same fused pass."""
+    cfg, batch = ii.make_config(idx)
+    ppo = dataclasses.replace(cfg.hyper, is_source=2, ratio_mode=2, lam=0.95, clip_eps=0.3)
+    P.check_categorical(oracle, batch, ppo)
+    impala = dataclasses.replace(cfg.hyper, objective=1, is_source=1, lam=1.0, kl_coef=0.1)
+    P.check_categorical(oracle, batch, impala)
+
+
+@pytest.mark.parametrize("B,T,A", [(5, 33, 7), (3, 300, 6), (9, 50, 18), (2, 70, 40)])
+def test_vtrace_policy_gradient_ragged(oracle, B, T, A):
+    batch = ii.categorical_batch(B, T, A, seed=5000 + T, p_done=0.05)
+    P.check_categorical(oracle, batch, LossHyper(objective=1, is_source=1, rho_bar=1.3, c_bar=1.1, lam=0.97, ent_coef=0.02))
+    P.check_categorical(oracle, batch, LossHyper(is_source=2, ratio_mode=2, lam=0.9))
+
+
+def test_baseline_objectives_gaussian(oracle):
+    cfg, batch = ii.make_config(3)
+    P.check_gaussian(oracle, batch, dataclasses.replace(cfg.hyper, is_source=2, ratio_mode=2, lam=0.95, clip_eps=0.3))
+    P.check_gaussian(oracle, batch, dataclasses.replace(cfg.hyper, objective=1, is_source=1, lam=1.0))
+    small = ii.gaussian_batch(3, 140, 5, seed=77, p_done=0.05)
+    P.check_gaussian(oracle, small, LossHyper(objective=1, is_source=1, ent_coef=0.01, kl_coef=0.2))
