@@ -336,10 +336,12 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
 //   * the slabs keep their dense global layout in shared memory; a thread reads its row
 //     with the widest vector access the row pitch allows, which is bank-conflict free for
 //     the action counts compiled here (pitch/width odd);
-//   * A is a template parameter, rows live in registers, every loop is unrolled;
+//   * A is a template parameter and every loop is unrolled; rows are streamed pair by pair from
+//     shared memory in each pass, so that few registers are live;
 //   * the softmax runs on exp2 of pre-scaled differences (one multiply + one MUFU each).
-// Five blocks per SM (<= 102 registers, no spills) measured faster than seven at 72 registers
-// with spills, even though a B*T = 131072 batch then runs as two waves of blocks.
+// Five blocks per SM (<= 102 registers, no spills) measured faster than seven at 72 registers,
+// with or without the second stage, even though 740 blocks then walk the 1024 tiles of a
+// B*T = 131072 batch.
 template <typename ST, int W> struct RowIO;
 
 // Rows are handled as NP = ceil(W/2) pairs; for odd W the second lane of the last pair is
@@ -378,6 +380,17 @@ template <int W> struct RowIO<float, W> {
             for (int j = 0; j < W / 2; ++j) { r[2 * j] = v[j].x; r[2 * j + 1] = v[j].y; }
             r[W - 1] = v[NP - 1].x;
         }
+    }
+    // pair j of a row (elements 2j, 2j+1; the second lane of an odd row's last pair is 0)
+    static __device__ __forceinline__ float2 load_pair(const unsigned char* slab, int row, int j) {
+        const float* r = reinterpret_cast<const float*>(slab) + row * W;
+        if constexpr (W % 2 == 0) return reinterpret_cast<const float2*>(r)[j];
+        else return (2 * j + 1 < W) ? make_float2(r[2 * j], r[2 * j + 1]) : make_float2(r[2 * j], 0.0f);
+    }
+    static __device__ __forceinline__ void store_pair(unsigned char* slab, int row, int j, float2 v) {
+        float* r = reinterpret_cast<float*>(slab) + row * W;
+        if constexpr (W % 2 == 0) reinterpret_cast<float2*>(r)[j] = v;
+        else { r[2 * j] = v.x; if (2 * j + 1 < W) r[2 * j + 1] = v.y; }
     }
     static __device__ __forceinline__ float at(const unsigned char* slab, int row, int col) {
         return reinterpret_cast<const float*>(slab)[row * W + col];
@@ -423,6 +436,24 @@ template <int W> struct RowIO<__nv_bfloat16, W> {
             r[W - 1] = __float2bfloat16_rn(v[NP - 1].x);
         }
     }
+    static __device__ __forceinline__ float2 load_pair(const unsigned char* slab, int row, int j) {
+        if constexpr (W % 2 == 0) {
+            const uint32_t w = reinterpret_cast<const uint32_t*>(slab)[row * (W / 2) + j];
+            return make_float2(__uint_as_float(w << 16), __uint_as_float(w & 0xFFFF0000u));
+        } else {
+            const unsigned short* r = reinterpret_cast<const unsigned short*>(slab) + row * W;
+            return (2 * j + 1 < W) ? make_float2(widen(r[2 * j]), widen(r[2 * j + 1])) : make_float2(widen(r[2 * j]), 0.0f);
+        }
+    }
+    static __device__ __forceinline__ void store_pair(unsigned char* slab, int row, int j, float2 v) {
+        if constexpr (W % 2 == 0) {
+            reinterpret_cast<uint32_t*>(slab)[row * (W / 2) + j] = dev::Pack<__nv_bfloat16>::two(v.x, v.y);
+        } else {
+            __nv_bfloat16* r = reinterpret_cast<__nv_bfloat16*>(slab) + row * W;
+            r[2 * j] = __float2bfloat16_rn(v.x);
+            if (2 * j + 1 < W) r[2 * j + 1] = __float2bfloat16_rn(v.y);
+        }
+    }
     static __device__ __forceinline__ float at(const unsigned char* slab, int row, int col) {
         return widen(reinterpret_cast<const unsigned short*>(slab)[row * W + col]);
     }
@@ -448,33 +479,11 @@ constexpr size_t reg_kernel_smem() {
     return 2 * reg_kernel_stage_bytes<LT, GT, A>();  // two stages
 }
 
-// A row of A logits in registers, as pairs: Blackwell's packed fp32 instructions (two lanes
-// per instruction for add, mul and fma) halve the arithmetic issue slots of the row passes.
-// Odd A carries its last element in a pair whose second lane is padding.
-template <int A> struct RowRegs {
-    static constexpr int NP = (A + 1) / 2;
-    float2 v[NP];
-    __device__ __forceinline__ float get(int j) const { return (j & 1) ? v[j >> 1].y : v[j >> 1].x; }
-};
-
-template <typename ST, int A>
-__device__ __forceinline__ void load_row_pairs(const unsigned char* slab, int row, RowRegs<A>& r) {
-    RowIO<ST, A>::load(slab, row, r.v);
-}
-
-template <int A>
-__device__ __forceinline__ float row_max(const RowRegs<A>& r) {
-    float m = r.v[0].x;
-#pragma unroll
-    for (int j = 1; j < A; ++j) m = fmaxf(m, r.get(j));
-    return m;
-}
-
 template <typename LT, typename GT, int A>
 __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_kernel(const CatParams p) {
     grid_dependency_wait();
     constexpr int NT = kRegTileRows;
-    constexpr int NP = RowRegs<A>::NP;
+    constexpr int NP = (A + 1) / 2;  // pairs per row: Blackwell's packed fp32 add / mul / fma work on two lanes at once
     constexpr bool kOdd = (A & 1) != 0;
     constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
     constexpr int kStageBytes = (int)reg_kernel_stage_bytes<LT, GT, A>();
@@ -628,21 +637,28 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
             __syncthreads();
 
             float fa = 1.0f, fb = 0.0f;
-            // Nothing row-sized stays in registers across the scan: the epilogue re-reads the
-            // learner row from shared memory and re-forms its exponentials (18 more MUFU ops are
-            // cheaper than 36 registers held across the barrier).
+            // Rows are streamed pair by pair from shared memory in every pass and nothing row-sized is
+            // held in registers (not within a pass, not across the scan): shared-memory reads are cheap
+            // here, registers are what limits how many rows an SM works on at once.
             float m2_l = 0.0f, ln_s = 0.0f, inv_s = 0.0f, lse_t = 0.0f, ent = 0.0f, kl = 0.0f;
             bool truncated = false;
             if (active) {
                 {   // target row: only its log-sum-exp and the taken action's logit are needed
-                    RowRegs<A> zr;
-                    load_row_pairs<LT, A>(s1, tid, zr);
-                    const float m = row_max<A>(zr);
+                    float2 mx = RowIO<LT, A>::load_pair(s1, tid, 0);
+                    if (kOdd && NP == 1) mx.y = mx.x;
+#pragma unroll
+                    for (int j = 1; j < NP; ++j) {
+                        float2 v = RowIO<LT, A>::load_pair(s1, tid, j);
+                        if (kOdd && j == NP - 1) v.y = v.x;
+                        mx.x = fmaxf(mx.x, v.x);
+                        mx.y = fmaxf(mx.y, v.y);
+                    }
+                    const float m = fmaxf(mx.x, mx.y);
                     const float2 neg_m2 = make_float2(-m * kLog2e, -m * kLog2e);
                     float2 sum2 = make_float2(0.0f, 0.0f);
 #pragma unroll
                     for (int j = 0; j < NP; ++j) {
-                        const float2 t2 = __ffma2_rn(zr.v[j], log2e2, neg_m2);  // (z - m) log2 e
+                        const float2 t2 = __ffma2_rn(RowIO<LT, A>::load_pair(s1, tid, j), log2e2, neg_m2);  // (z - m) log2 e
                         float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
                         if (kOdd && j == NP - 1) ex.y = 0.0f;
                         sum2 = __fadd2_rn(sum2, ex);
@@ -650,22 +666,27 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
                     lse_t = m + __logf(sum2.x + sum2.y);
                     s.l_target = RowIO<LT, A>::at(s1, tid, a) - lse_t;
                 }
-                // keep the compiler from hoisting the next row's loads over this one's arithmetic:
-                // one row in registers at a time
-                asm volatile("" ::: "memory");
-                RowRegs<A> z;
-                load_row_pairs<LT, A>(s0, tid, z);
-                const float m = row_max<A>(z);
+                float2 mx = RowIO<LT, A>::load_pair(s0, tid, 0);
+                if (kOdd && NP == 1) mx.y = mx.x;
+#pragma unroll
+                for (int j = 1; j < NP; ++j) {
+                    float2 v = RowIO<LT, A>::load_pair(s0, tid, j);
+                    if (kOdd && j == NP - 1) v.y = v.x;
+                    mx.x = fmaxf(mx.x, v.x);
+                    mx.y = fmaxf(mx.y, v.y);
+                }
+                const float m = fmaxf(mx.x, mx.y);
                 m2_l = m * kLog2e;
                 const float2 neg_m2 = make_float2(-m2_l, -m2_l);
                 float2 sum2 = make_float2(0.0f, 0.0f), sez2 = make_float2(0.0f, 0.0f);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
-                    const float2 t2 = __ffma2_rn(z.v[j], log2e2, neg_m2);
+                    const float2 z = RowIO<LT, A>::load_pair(s0, tid, j);
+                    const float2 t2 = __ffma2_rn(z, log2e2, neg_m2);
                     float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
                     if (kOdd && j == NP - 1) ex.y = 0.0f;
                     sum2 = __fadd2_rn(sum2, ex);
-                    sez2 = __ffma2_rn(ex, z.v[j], sez2);
+                    sez2 = __ffma2_rn(ex, z, sez2);
                 }
                 const float sum = sum2.x + sum2.y;
                 ln_s = __logf(sum);
@@ -674,16 +695,13 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
                 ent = (m + ln_s) - (sez2.x + sez2.y) * inv_s;
                 s.l_theta = (RowIO<LT, A>::at(s0, tid, a) - m) - ln_s;
                 if (want_kl) {
-                    RowRegs<A> zr;
-                    load_row_pairs<LT, A>(s1, tid, zr);
                     const float lse_l = m + ln_s;
 #pragma unroll
                     for (int j = 0; j < A; ++j) {
-                        const float lpt = zr.get(j) - lse_t;
-                        kl = fmaf(dev::exp2_fast(lpt * kLog2e), lpt - (z.get(j) - lse_l), kl);
+                        const float lpt = RowIO<LT, A>::at(s1, tid, j) - lse_t;
+                        kl = fmaf(dev::exp2_fast(lpt * kLog2e), lpt - (RowIO<LT, A>::at(s0, tid, j) - lse_l), kl);
                     }
                 }
-                asm volatile("" ::: "memory");
                 truncated = dev::recursion_map(s, k, fa, fb);
             }
             const float adv = dev::suffix_affine_scan<NT>(fa, fb, carry, warp_agg, s.adv_next);
@@ -723,35 +741,28 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
                 const float2 inv_s2 = make_float2(inv_s, inv_s), hoff2 = make_float2(h_off, h_off);
                 const float2 ce2 = make_float2(ce, ce), w12 = make_float2(w1, w1);
                 const float2 neg_m2 = make_float2(-m2_l, -m2_l);
-                RowRegs<A> z, gr;
-                load_row_pairs<LT, A>(s0, tid, z);
+                const float2 ck2 = make_float2(ck, ck);
+                const float2 neg_lse_t2 = make_float2(-lse_t * kLog2e, -lse_t * kLog2e);
 #pragma unroll
                 for (int j = 0; j < NP; ++j) {
-                    const float2 t2 = __ffma2_rn(z.v[j], log2e2, neg_m2);
+                    const float2 z = RowIO<LT, A>::load_pair(s0, tid, j);
+                    const float2 t2 = __ffma2_rn(z, log2e2, neg_m2);
                     const float2 pi2 = __fmul2_rn(make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y)), inv_s2);
-                    gr.v[j] = __fmul2_rn(pi2, __ffma2_rn(ce2, __fadd2_rn(z.v[j], hoff2), w12));
-                    if (want_kl) z.v[j] = pi2;  // keep pi_j for the KL term below
+                    float2 g2 = __fmul2_rn(pi2, __ffma2_rn(ce2, __fadd2_rn(z, hoff2), w12));
+                    if (want_kl) {
+                        const float2 tt = __ffma2_rn(RowIO<LT, A>::load_pair(s1, tid, j), log2e2, neg_lse_t2);
+                        const float2 npt = make_float2(-dev::exp2_fast(tt.x), -dev::exp2_fast(tt.y));
+                        g2 = __ffma2_rn(ck2, __fadd2_rn(pi2, npt), g2);
+                    }
+                    RowIO<GT, A>::store_pair(so, tid, j, g2);
                 }
                 // the taken action's entry, from its own log-probability
                 const float pi_a = dev::exp2_fast(s.l_theta * kLog2e);
                 float g_a = fmaf(pi_a, fmaf(ce, s.l_theta + ent, w1), -w1);
-                if (want_kl) {
-                    RowRegs<A> zr;
-                    load_row_pairs<LT, A>(s1, tid, zr);
-                    const float2 ck2 = make_float2(ck, ck);
-                    const float2 neg_lse_t2 = make_float2(-lse_t * kLog2e, -lse_t * kLog2e);
-#pragma unroll
-                    for (int j = 0; j < NP; ++j) {
-                        const float2 tt = __ffma2_rn(zr.v[j], log2e2, neg_lse_t2);
-                        const float2 npt = make_float2(-dev::exp2_fast(tt.x), -dev::exp2_fast(tt.y));
-                        gr.v[j] = __ffma2_rn(ck2, __fadd2_rn(z.v[j], npt), gr.v[j]);
-                    }
-                    g_a = fmaf(ck, pi_a - dev::exp2_fast(s.l_target * kLog2e), g_a);
-                }
+                if (want_kl) g_a = fmaf(ck, pi_a - dev::exp2_fast(s.l_target * kLog2e), g_a);
                 p.dvalues[row] = -k.vf_coef * k.inv_M * adv;  // V - Vhat = -A
                 if (p.vtarget) p.vtarget[row] = s.value + adv;
                 if (p.advantage) p.advantage[row] = adv;
-                RowIO<GT, A>::store(so, tid, gr.v);
                 RowIO<GT, A>::put(so, tid, a, g_a);
             }
             if (bulk_out) dev::fence_async_shared();
