@@ -412,9 +412,11 @@ __device__ __forceinline__ unsigned int publish_block_sums(const float (&acc)[kN
     float4* row = reinterpret_cast<float4*>(partials + (size_t)blockIdx.x * 8);
     row[0] = make_float4(acc[0], acc[1], acc[2], acc[3]);
     row[1] = make_float4(acc[4], acc[5], acc[6], 0.0f);
-    // release the row, then draw the ticket (acq_rel: the last drawer also acquires all rows)
-    asm volatile("fence.acq_rel.gpu;" ::: "memory");
-    return atomicAdd(counter, 1u);
+    // one acq_rel atomic: releases this block's row and, for the block that draws the last ticket,
+    // acquires every other block's (their atomics on the counter form the release sequence)
+    unsigned int ticket;
+    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(ticket) : "l"(counter) : "memory");
+    return ticket;
 }
 
 // Run by every thread of the block that drew the last ticket: add all blocks' sums in index
@@ -423,7 +425,8 @@ template <int NT>
 __device__ __noinline__ void reduce_published_sums(const float* partials, unsigned int* counter,
                                                       float* loss_terms, const LossScalars& k, double M) {
     __shared__ double dred[NT / 32][kNumSums];
-    asm volatile("fence.acq_rel.gpu;" ::: "memory");
+    // thread 0 acquired the rows with its ticket and a block barrier lies between that and here;
+    // the loads below go to L2 (ld.cg), so no further fence is needed
     double s[kNumSums];
 #pragma unroll
     for (int j = 0; j < kNumSums; ++j) s[j] = 0.0;
