@@ -90,7 +90,9 @@ __device__ __forceinline__ void mbarrier_expect_tx(uint64_t* bar, uint32_t bytes
 // bytes never arrive the caller gets `false` instead of a hang.
 __device__ __forceinline__ bool mbarrier_wait(uint64_t* bar, uint32_t parity) {
     const uint32_t addr = smem_addr(bar);
-    constexpr uint32_t kSuspendHintNs = 100000;  // each try may sleep this long: few tries, no busy spinning
+    // each try may sleep up to the hint and a failed try backs off 64 ns: the wait gives up after
+    // somewhere between ~0.07 s and ~1.1 s, far beyond any copy's latency, far short of a hang
+    constexpr uint32_t kSuspendHintNs = 1000;
     for (uint32_t tries = 0; tries < (1u << 20); ++tries) {
         uint32_t done;
         asm volatile(

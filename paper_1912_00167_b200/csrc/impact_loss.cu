@@ -525,7 +525,8 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
     };
     auto tile_of = [&](long long it) {
         Tile t;
-        const long long ci = it / g.ntiles;
+        // (no 64-bit division on the common path: one tile per trajectory)
+        const long long ci = (g.ntiles == 1) ? it : (long long)((unsigned long long)it / (unsigned int)g.ntiles);
         t.chunk = blockIdx.x + ci * gridDim.x;
         t.tile = g.ntiles - 1 - (int)(it - ci * g.ntiles);
         const TileRows tr = tile_rows<NT>(g, t.chunk, t.tile);
