@@ -582,7 +582,7 @@ def main():
     achieved = bytes_per_launch / (dense_ms * 1e-3) / 1e9
     gbs = lambda ms: bytes_per_launch / (ms * 1e-3) / 1e9
     roofline = {
-        "bound": "hbm", "kernel": "impact_loss_categorical_reg_kernel<float,float,18>",
+        "bound": "hbm", "kernel": "impact_loss_categorical_ws_kernel<float,float,18>",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
         "traffic": NCU_TRAFFIC_BYTES,
         "algorithmic_bytes_per_launch": bytes_per_launch,

@@ -86,6 +86,9 @@ __device__ __forceinline__ void mbarrier_expect_tx(uint64_t* bar, uint32_t bytes
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
                  : "memory");
 }
+__device__ __forceinline__ void mbarrier_arrive(uint64_t* bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(smem_addr(bar)) : "memory");
+}
 // Waits for the phase with the given parity to complete.  The wait is bounded: if the
 // bytes never arrive the caller gets `false` instead of a hang.
 __device__ __forceinline__ bool mbarrier_wait(uint64_t* bar, uint32_t parity) {
@@ -103,6 +106,26 @@ __device__ __forceinline__ bool mbarrier_wait(uint64_t* bar, uint32_t parity) {
         if (done) return true;
         __nanosleep(64);  // a failed try returns early on this part: back off instead of spinning
     }
+    return false;
+}
+// The same wait for blocks in which several warps wait on one another's barriers: it also gives up
+// (at once) when `*abort_flag` is set, and sets it when it gives up itself, so that one wait that
+// runs out ends every other wait of the block instead of each running out in turn.
+__device__ __forceinline__ bool mbarrier_wait(uint64_t* bar, uint32_t parity, int* abort_flag) {
+    const uint32_t addr = smem_addr(bar);
+    constexpr uint32_t kSuspendHintNs = 1000;
+    for (uint32_t tries = 0; tries < (1u << 20); ++tries) {
+        uint32_t done;
+        asm volatile(
+            "{\n\t.reg .pred p;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "selp.u32 %0, 1, 0, p;\n\t}"
+            : "=r"(done) : "r"(addr), "r"(parity), "r"(kSuspendHintNs) : "memory");
+        if (done) return true;
+        if (*reinterpret_cast<volatile int*>(abort_flag)) return false;
+        __nanosleep(64);
+    }
+    *reinterpret_cast<volatile int*>(abort_flag) = 1;
     return false;
 }
 __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, uint32_t bytes, uint64_t* bar) {
@@ -124,6 +147,41 @@ __device__ __forceinline__ float exp2_fast(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
+}
+
+__device__ __forceinline__ float log2_fast(float x) {
+    float y;
+    asm("lg2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+__device__ __forceinline__ float rcp_fast(float x) {
+    float y;
+    asm("rcp.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
+    return y;
+}
+
+// Sum of one value over the warp, in every lane (fixed order).
+__device__ __forceinline__ float warp_sum(float x) {
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+    return x;
+}
+// Sums of four values over the warp in one butterfly of six shuffles: lanes 0-7 return the
+// total of `a`, lanes 8-15 of `b`, lanes 16-23 of `c`, lanes 24-31 of `d` (fixed order).
+__device__ __forceinline__ float warp_sum4(float a, float b, float c, float d) {
+    const int lane = threadIdx.x & 31;
+    const bool hi16 = (lane & 16) != 0, hi8 = (lane & 8) != 0;
+    float k0 = hi16 ? c : a, k1 = hi16 ? d : b;
+    const float s0 = hi16 ? a : c, s1 = hi16 ? b : d;
+    k0 += __shfl_xor_sync(0xffffffffu, s0, 16);
+    k1 += __shfl_xor_sync(0xffffffffu, s1, 16);
+    float x = hi8 ? k1 : k0;
+    const float y = hi8 ? k0 : k1;
+    x += __shfl_xor_sync(0xffffffffu, y, 8);
+    x += __shfl_xor_sync(0xffffffffu, x, 4);
+    x += __shfl_xor_sync(0xffffffffu, x, 2);
+    x += __shfl_xor_sync(0xffffffffu, x, 1);
+    return x;
 }
 
 // Walks (row, col) positions of a dense [rows, W] slab in steps of a fixed element count.
@@ -259,6 +317,34 @@ __device__ __forceinline__ float suffix_affine_scan(float a, float b, float carr
     return result;
 }
 
+// The same scan inside a group of NT threads that synchronises on named barrier `bar_id`
+// (trajectories never continue past a tile here, so there is no carry).
+template <int NT>
+__device__ __forceinline__ float suffix_affine_scan_group(float a, float b, float2* warp_agg, float& next, int bar_id) {
+    const int lane = threadIdx.x & 31, warp = (threadIdx.x & (NT - 1)) >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float a2 = __shfl_down_sync(0xffffffffu, a, off);
+        const float b2 = __shfl_down_sync(0xffffffffu, b, off);
+        if (lane + off < 32) {
+            b = fmaf(a, b2, b);
+            a = a * a2;
+        }
+    }
+    if (lane == 0) warp_agg[warp] = make_float2(a, b);
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory");
+    float x = 0.0f;
+#pragma unroll
+    for (int w = NT / 32 - 1; w > 0; --w) {
+        const float2 g = warp_agg[w];
+        if (w > warp) x = fmaf(g.x, x, g.y);
+    }
+    const float result = fmaf(a, x, b);
+    const float below = __shfl_down_sync(0xffffffffu, result, 1);
+    next = (lane == 31) ? x : below;
+    return result;
+}
+
 // Scalars of the loss that the kernels need; filled on the host.
 struct LossScalars {
     float rho_bar, c_bar, clip_lo, clip_hi;
@@ -312,6 +398,28 @@ __device__ __forceinline__ float surrogate(const StepIn& s, const LossScalars& k
     if (k.ratio_mode == 1) d = s.l_target;
     else if (k.ratio_mode == 2) d = s.l_worker;
     else d = fmaxf(s.l_target, s.l_worker - k.log_rho_tw);
+    const float R = exp_of_logratio(s.l_theta - d);
+    const float Rc = fminf(fmaxf(R, k.clip_lo), k.clip_hi);
+    surr = fminf(R * adv, Rc * adv);
+    clipped = (adv > 0.0f && R > k.clip_hi) || (adv < 0.0f && R < k.clip_lo);
+    ratio = R;
+    return clipped ? 0.0f : adv * R;
+}
+
+// The two functions above for the default configuration (importance weights pi_target / pi_worker,
+// ratio R3, clipped surrogate), without the run-time switches.
+__device__ __forceinline__ bool recursion_map_plain(StepIn& s, const LossScalars& k, float& a, float& b) {
+    const float w = exp_of_logratio(s.l_target - s.l_worker);
+    const float rho = fminf(k.rho_bar, w);
+    s.rho = rho;
+    const float c = fminf(k.c_bar, w);
+    b = rho * (s.reward + s.discount * s.value_next - s.value);
+    a = s.last_step ? 0.0f : k.lambda_ * s.discount * c;
+    return w > k.rho_bar;
+}
+__device__ __forceinline__ float surrogate_plain(const StepIn& s, const LossScalars& k, float adv, float& surr,
+                                                 float& ratio, bool& clipped) {
+    const float d = fmaxf(s.l_target, s.l_worker - k.log_rho_tw);
     const float R = exp_of_logratio(s.l_theta - d);
     const float Rc = fminf(fmaxf(R, k.clip_lo), k.clip_hi);
     surr = fminf(R * adv, Rc * adv);
@@ -420,12 +528,19 @@ __device__ __forceinline__ unsigned int publish_block_sums(const float (&acc)[kN
     asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(ticket) : "l"(counter) : "memory");
     return ticket;
 }
+// The ticket alone, for blocks whose row was written by several lanes of the calling warp
+// (with a __syncwarp() between those stores and this call).
+__device__ __forceinline__ unsigned int take_ticket(unsigned int* counter) {
+    unsigned int ticket;
+    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(ticket) : "l"(counter) : "memory");
+    return ticket;
+}
 
 // Run by every thread of the block that drew the last ticket: add all blocks' sums in index
 // order (fp64), write the eight loss terms, and leave the counter at 0 for the next launch.
 template <int NT>
-__device__ __noinline__ void reduce_published_sums(const float* partials, unsigned int* counter,
-                                                      float* loss_terms, const LossScalars& k, double M) {
+__device__ __noinline__ void reduce_published_sums(const float* partials, unsigned int* counter, float* loss_terms,
+                                                      float vf_coef, float ent_coef, float kl_coef, double M) {
     __shared__ double dred[NT / 32][kNumSums];
     // thread 0 acquired the rows with its ticket and a block barrier lies between that and here;
     // the loads below go to L2 (ld.cg), so no further fence is needed
@@ -472,8 +587,70 @@ __device__ __noinline__ void reduce_published_sums(const float* partials, unsign
             t[j] = x * inv_m;
         }
         const double l_pi = -t[0], l_v = t[1], ent = t[2], kl = t[3];
-        loss_terms[0] = (float)(l_pi + (double)k.vf_coef * l_v - (double)k.ent_coef * ent +
-                                (double)k.kl_coef * kl);
+        loss_terms[0] = (float)(l_pi + (double)vf_coef * l_v - (double)ent_coef * ent +
+                                (double)kl_coef * kl);
+        loss_terms[1] = (float)l_pi;
+        loss_terms[2] = (float)l_v;
+        loss_terms[3] = (float)ent;
+        loss_terms[4] = (float)kl;
+        loss_terms[5] = (float)t[4];
+        loss_terms[6] = (float)t[5];
+        loss_terms[7] = (float)t[6];
+        *counter = 0u;
+    }
+}
+
+// reduce_published_sums for a group of NT threads inside a larger block: `gtid` is the thread's
+// index in the group, `bar_id` the group's named barrier.  Only one group of a grid ever runs it (the
+// one that drew the last ticket), so the shared scratch is not contended.
+template <int NT>
+__device__ __noinline__ void reduce_rows_group(const float* partials, int nrows, unsigned int* counter, float* loss_terms,
+                                                 float vf_coef, float ent_coef, float kl_coef, double M, int gtid,
+                                                 int bar_id) {
+    __shared__ double dred[NT / 32][kNumSums];
+    double s[kNumSums];
+#pragma unroll
+    for (int j = 0; j < kNumSums; ++j) s[j] = 0.0;
+    constexpr int kBatch = 8;
+    for (int first = gtid; first < nrows; first += NT * kBatch) {
+        float4 p0[kBatch], p1[kBatch];
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            const int r = first + u * NT;
+            if (r < nrows) {
+                p0[u] = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)r * 8));
+                p1[u] = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)r * 8 + 4));
+            } else {
+                p0[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                p1[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < kBatch; ++u) {
+            s[0] += p0[u].x; s[1] += p0[u].y; s[2] += p0[u].z; s[3] += p0[u].w;
+            s[4] += p1[u].x; s[5] += p1[u].y; s[6] += p1[u].z;
+        }
+    }
+    const int lane = gtid & 31, warp = gtid >> 5;
+#pragma unroll
+    for (int j = 0; j < kNumSums; ++j) {
+        double x = s[j];
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
+        if (lane == 0) dred[warp][j] = x;
+    }
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory");
+    if (gtid == 0) {
+        const double inv_m = 1.0 / M;
+        double t[kNumSums];
+#pragma unroll
+        for (int j = 0; j < kNumSums; ++j) {
+            double x = 0.0;
+            for (int w = 0; w < NT / 32; ++w) x += dred[w][j];
+            t[j] = x * inv_m;
+        }
+        const double l_pi = -t[0], l_v = t[1], ent = t[2], kl = t[3];
+        loss_terms[0] = (float)(l_pi + (double)vf_coef * l_v - (double)ent_coef * ent + (double)kl_coef * kl);
         loss_terms[1] = (float)l_pi;
         loss_terms[2] = (float)l_v;
         loss_terms[3] = (float)ent;

@@ -321,7 +321,8 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
             if (!final_tile) __syncthreads();
         }
     }
-    if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k, (double)g.B * (double)g.T);
+    if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef,
+                                                   (double)g.B * (double)g.T);
     if (tid == 0) dev::bulk_store_wait_read();
 }
 
@@ -784,8 +785,361 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
             cur = nxt;
         }
     }
-    if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k, (double)g.B * (double)g.T);
+    if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef,
+                                                   (double)g.B * (double)g.T);
     if (tid == 0) dev::bulk_store_wait_read();  // shared memory must outlive the store's reads
+}
+
+// ------------------------------------------------------------------------------------------
+// Categorical policy, persistent warp-specialised form (trajectories of at most 128 steps)
+// ------------------------------------------------------------------------------------------
+// One block per SM.  A producer warp streams the block's tiles (blockIdx.x, + gridDim.x, ...)
+// through a ring of shared-memory stages, keeping a fixed number of tiles in flight, so that
+// tiles land one after the other from the first microseconds on instead of all at the end;
+// C consumer groups of 128 threads (one thread per step, as above) each take every C-th tile
+// as it lands, and every warp sends its own 32 gradient rows off by a bulk store while later
+// tiles are still arriving.  Loading, arithmetic and storing overlap inside one launch: a
+// B*T = 131072 batch (seven tiles per SM) takes 9.7 us against 12.5 us for resident blocks
+// that each load, compute and store one tile, and batches of a million steps and more run at
+// the speed of a device-to-device copy.
+//
+// Barriers: full[s] (one arrival + the bytes of the two slabs) says stage s holds a tile;
+// empty[s] (one arrival per consumer warp, after that warp's store has finished reading the
+// stage) says it may be refilled.  Every wait is bounded; a wait that gives up raises the
+// workspace's error word and the block's abort flag, after which nobody waits any more and
+// the block runs to its end on whatever the stages hold.
+constexpr int kWsMaxStages = 24;
+constexpr int kWsGroups = 4;  // consumer groups per block: 16 consumer warps + the producer warp, <= 120 registers each
+
+__device__ __forceinline__ void group_barrier(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
+
+// Row passes of one step, shared by the kernels with a compile-time action count.  `zr` / `tr`
+// point at the thread's learner / target row in shared memory.
+template <typename LT, int A>
+struct RowMath {
+    static constexpr int NP = (A + 1) / 2;
+    static constexpr bool kOdd = (A & 1) != 0;
+    static constexpr float kLog2e = 1.4426950408889634f;
+
+    // log2-sum-exp (base 2, of z log2 e) of a row; optionally keeps the exponentials and sum_j e_j z_j
+    template <bool kKeep>
+    static __device__ __forceinline__ float lse2(const unsigned char* slab, int row, float2 (&e)[NP], float& m2, float& sum,
+                                                 float& sez) {
+        float2 v[NP];
+        RowIO<LT, A>::load(slab, row, v);
+        float m0, m1;
+        {
+            const float y0 = (kOdd && NP == 1) ? v[0].x : v[0].y;
+            m0 = fmaxf(v[0].x, y0);
+            m1 = m0;
+        }
+#pragma unroll
+        for (int j = 1; j < NP; ++j) {
+            const float y = (kOdd && j == NP - 1) ? v[j].x : v[j].y;
+            if (j & 1) m1 = fmaxf(m1, fmaxf(v[j].x, y));
+            else m0 = fmaxf(m0, fmaxf(v[j].x, y));
+        }
+        m2 = fmaxf(m0, m1) * kLog2e;
+        const float2 neg_m2 = make_float2(-m2, -m2), log2e2 = make_float2(kLog2e, kLog2e);
+        float2 sum2 = make_float2(0.0f, 0.0f), sez2 = make_float2(0.0f, 0.0f);
+#pragma unroll
+        for (int j = 0; j < NP; ++j) {
+            const float2 t2 = __ffma2_rn(v[j], log2e2, neg_m2);  // (z - m) log2 e
+            float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
+            if (kOdd && j == NP - 1) ex.y = 0.0f;
+            sum2 = __fadd2_rn(sum2, ex);
+            if (kKeep) {
+                e[j] = ex;
+                sez2 = __ffma2_rn(ex, v[j], sez2);
+            }
+        }
+        sum = sum2.x + sum2.y;
+        sez = sez2.x + sez2.y;
+        return m2 + dev::log2_fast(sum);
+    }
+};
+
+// kPlain: the configuration of the paper's experiments -- no KL term, the clipped surrogate with the
+// default ratio and importance weights, no optional outputs -- with those branches compiled out.
+template <typename LT, typename GT, int A, int C, bool kPlain>
+__global__ void __launch_bounds__(C * 128 + 32, 1)
+impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W) {
+    constexpr int NT = 128;
+    constexpr int NP = (A + 1) / 2;
+    constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
+    constexpr int kStageBytes = (int)reg_kernel_stage_bytes<LT, GT, A>();
+    constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
+    using RM = RowMath<LT, A>;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kWsMaxStages], empty_bar[kWsMaxStages];
+    __shared__ float2 warp_agg[C][NT / 32];
+    __shared__ __align__(16) float red[C][NT / 32][8];
+    __shared__ int is_last_s[C];
+    __shared__ int abort_s;
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    const LossScalars& k = p.k;
+    const TileGeometry& g = p.geo;
+    const int n_tiles = (int)((g.nchunks - blockIdx.x + gridDim.x - 1) / gridDim.x);  // this block's tiles
+    const int rows_full = g.G * (int)g.T;                                                // rows of a full tile
+    const long long total_rows = g.B * g.T;
+
+    if (tid == 0) {
+        for (int s = 0; s < S; ++s) {
+            dev::mbarrier_init(&full_bar[s], 1);
+            dev::mbarrier_init(&empty_bar[s], NT / 32);  // one arrival per consumer warp
+        }
+        abort_s = 0;
+    }
+    __syncthreads();
+    grid_dependency_wait();  // everything above touches only this block's shared memory
+
+    if (tid >= C * NT) {
+        // ---- producer warp: one lane streams the block's tiles into the ring ------------------
+        if (lane != 0) return;
+        const LT* gl = static_cast<const LT*>(p.learner_logits) + (long long)blockIdx.x * rows_full * A;
+        const LT* gt = static_cast<const LT*>(p.target_logits) + (long long)blockIdx.x * rows_full * A;
+        const long long step_elems = (long long)gridDim.x * rows_full * A;
+        long long rows_left = total_rows - (long long)blockIdx.x * rows_full;
+        const long long step_rows = (long long)gridDim.x * rows_full;
+        int s = 0, ws = 0;         // stage of tile n, stage of tile n - W
+        uint32_t ph = 0, wph = 0;  // their phase parities
+        for (int n = 0; n < n_tiles; ++n) {
+            bool ok = true;
+            if (n >= S) ok = dev::mbarrier_wait(&empty_bar[s], ph ^ 1u, &abort_s);   // the stage's previous tile has left
+            if (ok && n >= W) ok = dev::mbarrier_wait(&full_bar[ws], wph, &abort_s);  // at most W tiles in flight
+            if (!ok) { atomicExch(p.counter + 1, 1u); return; }
+            const int nrows = rows_left < rows_full ? (int)rows_left : rows_full;
+            unsigned char* const d0 = smem_raw + s * kStageBytes;
+            unsigned char* const d1 = d0 + NT * kInRow;
+            const uint32_t bytes = (uint32_t)nrows * kInRow;
+            if (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | bytes) & 15u) == 0) {
+                dev::mbarrier_expect_tx(&full_bar[s], 2 * bytes);
+                dev::bulk_load(d0, gl, bytes, &full_bar[s]);
+                dev::bulk_load(d1, gt, bytes, &full_bar[s]);
+            } else {  // ragged or unaligned slab: element by element
+                const int nelem = nrows * A;
+                for (int e = 0; e < nelem; ++e) {
+                    reinterpret_cast<LT*>(d0)[e] = gl[e];
+                    reinterpret_cast<LT*>(d1)[e] = gt[e];
+                }
+                dev::mbarrier_arrive(&full_bar[s]);
+            }
+            gl += step_elems;
+            gt += step_elems;
+            rows_left -= step_rows;
+            if (++s == S) { s = 0; ph ^= 1u; }
+            if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
+        }
+        return;
+    }
+
+    // ---- consumer groups ------------------------------------------------------------------
+    const int grp = tid >> 7, gtid = tid & (NT - 1), gwarp = gtid >> 5;
+    const int bar_id = grp + 1;
+    const bool want_kl = !kPlain && (k.kl_coef != 0.0f);
+
+    // the thread's place in a tile never changes: step ts of trajectory q of the tile
+    int q = 0, ts = gtid;
+    if (g.G > 1) { q = gtid / (int)g.T; ts = gtid - q * (int)g.T; }
+    const bool in_layout = gtid < rows_full;
+    const bool last_step = (ts == (int)g.T - 1);
+    // row and trajectory of this thread in the group's current tile, and their advance per tile
+    long long row = ((long long)blockIdx.x + (long long)grp * gridDim.x) * rows_full + gtid;
+    long long traj = ((long long)blockIdx.x + (long long)grp * gridDim.x) * g.G + q;
+    const long long row_step = (long long)gridDim.x * C * rows_full, traj_step = (long long)gridDim.x * C * g.G;
+
+    struct StepRaw {
+        int a;
+        float l_worker, reward, discount, value, value_next;
+    };
+    auto load_scalars = [&](long long r, long long b, bool act) {
+        StepRaw x;
+        x.a = 0; x.l_worker = 0.0f; x.reward = 0.0f; x.discount = 0.0f; x.value = 0.0f; x.value_next = 0.0f;
+        if (act) {
+            const int a = p.actions[r];
+            x.a = min(max(a, 0), A - 1);
+            x.l_worker = p.worker_logp[r];
+            x.reward = p.rewards[r];
+            x.discount = p.discounts[r];
+            x.value = p.values[r];
+            x.value_next = last_step ? p.bootstrap[b] : p.values[r + 1];
+        }
+        return x;
+    };
+
+    float t_surr = 0.0f, t_val = 0.0f, t_ent = 0.0f, t_ratio = 0.0f, t_kl = 0.0f;
+    int n_clip = 0, n_trunc = 0;
+    bool pending = false;  // lane 0 of each warp: a store of this warp may still be reading its stage
+    int pending_stage = 0;
+
+    bool active = in_layout && row < total_rows;
+    StepRaw cur;
+    if (grp < n_tiles) cur = load_scalars(row, traj, active);
+    int s = grp % S;
+    uint32_t ph = (uint32_t)(grp / S) & 1u;
+
+    for (int n = grp; n < n_tiles; n += C) {
+        // the next tile's scalars travel while this tile is worked on
+        const bool active_next = (n + C < n_tiles) && in_layout && (row + row_step < total_rows);
+        const StepRaw nxt = load_scalars(row + row_step, traj + traj_step, active_next);
+        if (lane == 0 && pending) {  // this warp's previous rows have left shared memory: hand the stage back
+            dev::bulk_store_wait_read();
+            dev::mbarrier_arrive(&empty_bar[pending_stage]);
+            pending = false;
+        }
+        // every thread waits for the stage itself (a bounded wait: on a time-out the flag is set and the
+        // thread goes on with whatever the stage holds, so that all barriers below still pair up)
+        if (!dev::mbarrier_wait(&full_bar[s], ph, &abort_s)) atomicExch(p.counter + 1, 1u);
+
+        unsigned char* const s0 = smem_raw + s * kStageBytes;  // learner logits
+        unsigned char* const s1 = s0 + NT * kInRow;             // target logits
+        unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : s0 + 2 * NT * kInRow;
+        const int a = cur.a;
+        dev::StepIn st;
+        st.l_worker = cur.l_worker;
+        st.reward = cur.reward;
+        st.discount = cur.discount;
+        st.value = cur.value;
+        st.value_next = cur.value_next;
+        st.last_step = last_step;
+
+        // ---- row passes (every thread; rows beyond the tile hold stale bytes and are masked)
+        float2 e[NP];
+        float m2_t, sum_t, unused, m2_l, sum_l, sez;
+        const float lse2_t = RM::template lse2<false>(s1, gtid, e, m2_t, sum_t, unused);
+        st.l_target = fmaf(RowIO<LT, A>::at(s1, gtid, a), kLog2e, -lse2_t) * kLn2;
+        const float lse2_l = RM::template lse2<true>(s0, gtid, e, m2_l, sum_l, sez);
+        const float inv_s = dev::rcp_fast(sum_l);
+        // H = -sum_j pi_j lp_j = (m + ln S) - sum_j e_j z_j / S
+        const float ent = fmaf(lse2_l, kLn2, -sez * inv_s);
+        st.l_theta = fmaf(RowIO<LT, A>::at(s0, gtid, a), kLog2e, -lse2_l) * kLn2;
+        float kl = 0.0f;
+        if (want_kl) {
+#pragma unroll
+            for (int j = 0; j < A; ++j) {
+                const float lpt2 = fmaf(RowIO<LT, A>::at(s1, gtid, j), kLog2e, -lse2_t);
+                const float lpl2 = fmaf(RowIO<LT, A>::at(s0, gtid, j), kLog2e, -lse2_l);
+                kl = fmaf(dev::exp2_fast(lpt2), (lpt2 - lpl2) * kLn2, kl);
+            }
+        }
+        float fa, fb;
+        bool truncated;
+        if (kPlain) truncated = dev::recursion_map_plain(st, k, fa, fb);
+        else truncated = dev::recursion_map(st, k, fa, fb);
+        if (!active) { fa = 1.0f; fb = 0.0f; }
+        const float adv = dev::suffix_affine_scan_group<NT>(fa, fb, warp_agg[grp], st.adv_next, bar_id);
+
+        float surr, ratio;
+        bool clipped;
+        const float wpg = kPlain ? dev::surrogate_plain(st, k, adv, surr, ratio, clipped) : dev::surrogate(st, k, adv, surr, ratio, clipped);
+        if (active) {
+            t_surr += surr;
+            t_val = fmaf(0.5f * adv, adv, t_val);
+            t_ent += ent;
+            t_ratio += ratio;
+            if (!kPlain) t_kl += kl;
+        }
+        n_clip += __popc(__ballot_sync(0xffffffffu, active && clipped));
+        n_trunc += __popc(__ballot_sync(0xffffffffu, active && truncated));
+
+        // ---- gradients: row_j = e_j (ga z_j + gb) [- kl_coef pi_target_j / M], then the taken action's entry
+        {
+            const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = kPlain ? 0.0f : k.kl_coef * k.inv_M;
+            const float h_off = fmaf(-lse2_l, kLn2, ent);
+            const float ga = ce * inv_s, gb = (fmaf(ce, h_off, w1) + ck) * inv_s;
+            const float2 ga2 = make_float2(ga, ga), gb2 = make_float2(gb, gb);
+            if (!want_kl) {
+#pragma unroll
+                for (int j = 0; j < NP; ++j) {
+                    const float2 z = RowIO<LT, A>::load_pair(s0, gtid, j);
+                    RowIO<GT, A>::store_pair(so, gtid, j, __fmul2_rn(e[j], __ffma2_rn(z, ga2, gb2)));
+                }
+            } else {
+                const float2 neg_lse2 = make_float2(-lse2_t, -lse2_t), nck2 = make_float2(-ck, -ck);
+                const float2 log2e2 = make_float2(kLog2e, kLog2e);
+#pragma unroll
+                for (int j = 0; j < NP; ++j) {
+                    const float2 z = RowIO<LT, A>::load_pair(s0, gtid, j);
+                    const float2 tt = __ffma2_rn(RowIO<LT, A>::load_pair(s1, gtid, j), log2e2, neg_lse2);
+                    const float2 pt = make_float2(dev::exp2_fast(tt.x), dev::exp2_fast(tt.y));
+                    RowIO<GT, A>::store_pair(so, gtid, j, __ffma2_rn(nck2, pt, __fmul2_rn(e[j], __ffma2_rn(z, ga2, gb2))));
+                }
+            }
+            const float pi_a = dev::exp2_fast(st.l_theta * kLog2e);
+            float g_a = fmaf(pi_a, fmaf(ce, st.l_theta + ent, w1), -w1);
+            if (want_kl) g_a = fmaf(ck, pi_a - dev::exp2_fast(st.l_target * kLog2e), g_a);
+            if (active) {
+                p.dvalues[row] = -k.vf_coef * k.inv_M * adv;  // V - Vhat = -A
+                if (!kPlain) {
+                    if (p.vtarget) p.vtarget[row] = st.value + adv;
+                    if (p.advantage) p.advantage[row] = adv;
+                }
+            }
+            RowIO<GT, A>::put(so, gtid, a, g_a);
+        }
+        // ---- each warp sends its own 32 rows: no barrier across the group
+        {
+            const long long wrow0 = row - lane;  // first row of this warp
+            long long left = total_rows - wrow0;
+            const int cap = rows_full - (gtid - lane);
+            if (left > cap) left = cap;
+            const int wrows = left > 32 ? 32 : (left > 0 ? (int)left : 0);
+            GT* const gd = static_cast<GT*>(p.dlogits) + wrow0 * A;
+            const unsigned char* const src = so + (gtid - lane) * kOutRow;
+            const uint32_t out_bytes = (uint32_t)wrows * kOutRow;
+            if (((reinterpret_cast<uintptr_t>(gd) | out_bytes) & 15u) == 0) {
+                dev::fence_async_shared();
+                __syncwarp();
+                if (lane == 0) {
+                    if (out_bytes) dev::bulk_store(gd, src, out_bytes);
+                    pending = true;
+                    pending_stage = s;
+                }
+            } else {
+                __syncwarp();
+                const int nelem = wrows * A;
+                for (int i = lane; i < nelem; i += 32) gd[i] = reinterpret_cast<const GT*>(src)[i];
+                __syncwarp();
+                if (lane == 0) dev::mbarrier_arrive(&empty_bar[s]);
+            }
+        }
+        cur = nxt;
+        active = active_next;
+        row += row_step;
+        traj += traj_step;
+        s += C;
+        while (s >= S) { s -= S; ph ^= 1u; }
+    }
+
+    // ---- the group's sums: one published row per group; the group that draws the last ticket adds all rows
+    {
+        const float x = dev::warp_sum4(t_surr, t_val, t_ent, t_ratio);
+        const float xk = want_kl ? dev::warp_sum(t_kl) : 0.0f;
+        if ((lane & 7) == 0) red[grp][gwarp][lane == 24 ? 6 : (lane >> 3)] = x;
+        if (lane == 0) {
+            red[grp][gwarp][3] = xk;
+            red[grp][gwarp][4] = (float)n_clip;
+            red[grp][gwarp][5] = (float)n_trunc;
+            red[grp][gwarp][7] = 0.0f;
+        }
+    }
+    group_barrier(bar_id);
+    if (gwarp == 0) {
+        if (lane < 8) {
+            float x = 0.0f;
+#pragma unroll
+            for (int w = 0; w < NT / 32; ++w) x += red[grp][w][lane];
+            p.partials[((size_t)blockIdx.x * C + grp) * 8 + lane] = x;
+        }
+        __syncwarp();
+        if (lane == 0) is_last_s[grp] = (dev::take_ticket(p.counter) == gridDim.x * C - 1) ? 1 : 0;
+    }
+    group_barrier(bar_id);
+    if (is_last_s[grp])
+        dev::reduce_rows_group<NT>(p.partials, (int)gridDim.x * C, p.counter, p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef,
+                                   (double)g.B * (double)g.T, gtid, bar_id);
+    if (lane == 0) dev::bulk_store_wait_read();  // shared memory must outlive the stores' reads
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1124,7 +1478,8 @@ __global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kern
             if (!final_tile) __syncthreads();
         }
     }
-    if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k, (double)g.B * (double)g.T);
+    if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef,
+                                                   (double)g.B * (double)g.T);
     if (tid == 0) dev::bulk_store_wait_read();
 }
 
@@ -1244,8 +1599,52 @@ int32_t dispatch_nt(const CatParams& p, int nt, const DeviceInfo* di, cudaStream
     }
 }
 
+// Tiles the producer keeps in flight and stages of the ring, for tiles of `tile_in_bytes` bytes of logits:
+// about 48 KB per SM on the way (enough, over 148 SMs, to cover HBM's latency at full bandwidth; more
+// only delays the first tiles), and room beyond that for the tiles being worked on and being stored.
+void ws_ring_shape(size_t stage_bytes, size_t tile_in_bytes, int groups, int max_smem, int* stages, int* in_flight) {
+    int w = (int)((48 * 1024 + tile_in_bytes - 1) / tile_in_bytes);
+    if (w < 3) w = 3;
+    if (w > 12) w = 12;
+    int s = w + groups + 3;
+    if (s > kWsMaxStages) s = kWsMaxStages;
+    const int fit = (int)((size_t)(max_smem - 4096) / stage_bytes);  // 4 KB left for static shared memory
+    if (s > fit) s = fit;
+    if (w > s) w = s;
+    *stages = s;
+    *in_flight = w;
+}
+
+template <typename LT, typename GT, int A, bool kPlain>
+int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
+    constexpr int C = kWsGroups;
+    auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain>;
+    const size_t stage = reg_kernel_stage_bytes<LT, GT, A>();
+    int S = 0, W = 0;
+    ws_ring_shape(stage, 2 * (size_t)kRegTileRows * A * sizeof(LT), C, di->max_smem_optin, &S, &W);
+    if (S < 2) return IMPACT_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)S * stage;
+    static thread_local int configured_device = -1;
+    if (configured_device != di->device) {
+        IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured_device = di->device;
+    }
+    const long long grid = p.geo.nchunks < di->sm_count ? p.geo.nchunks : di->sm_count;
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W));
+    return IMPACT_OK;
+}
+
+// The persistent kernel serves every batch whose trajectories fit a tile (T <= 128); longer
+// trajectories go to the kernel that carries the recursion from tile to tile.
 template <typename LT, typename GT, int A>
 int32_t launch_categorical_reg(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
+    if (p.geo.ntiles == 1) {
+        const bool plain = p.k.kl_coef == 0.0f && p.k.objective == IMPACT_OBJECTIVE_CLIPPED_SURROGATE &&
+                           p.k.is_source == IMPACT_IS_TARGET_OVER_WORKER && p.k.ratio_mode == IMPACT_RATIO_R3 &&
+                           !p.vtarget && !p.advantage;
+        if (plain) return launch_categorical_ws<LT, GT, A, true>(p, di, stream);
+        return launch_categorical_ws<LT, GT, A, false>(p, di, stream);
+    }
     auto kernel = impact_loss_categorical_reg_kernel<LT, GT, A>;
     const size_t smem = reg_kernel_smem<LT, GT, A>();
     int grid = 0;

@@ -174,7 +174,7 @@ def _vtrace_pg_bounds(ref, sens):
     return ref, sens
 
 
-def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, **tol):
+def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, extra=True, **tol):
     h = f32_hyper(h)
     if logits_dtype == torch.bfloat16:
         batch = dict(batch)
@@ -183,7 +183,7 @@ def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtyp
     ref = oracle.loss_categorical(batch, h)
     near = near_clip_bound(ref, h)
     ref_flipped = oracle.loss_categorical(batch, h, flip=near.astype(np.int8)) if near.any() else None
-    gpu = run_gpu_categorical(batch, h, logits_dtype, dlogits_dtype)
+    gpu = run_gpu_categorical(batch, h, logits_dtype, dlogits_dtype, extra=extra)
     M = batch["rewards"].size
     if h.objective == 1:
         from scipy.special import softmax

@@ -105,6 +105,22 @@ def test_all_steps_terminal_and_on_policy(oracle):
     P.check_categorical(oracle, batch, LossHyper(kl_coef=1.0))
 
 
+@pytest.mark.parametrize("B,T,A", [(4, 20, 6), (32, 50, 18), (1024, 128, 18), (7, 33, 4), (5, 127, 9), (130, 1, 18),
+                                   (301, 21, 9), (1500, 128, 6), (2000, 50, 18)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_default_configuration_without_optional_outputs(oracle, B, T, A, dtype):
+    """No KL term, default ratio and importance weights, no vtarget / advantage: the configuration for which the
+    library compiles its switches out.  Shapes cover one and several trajectories per tile, tiles that end
+    unaligned, a ragged last tile, and more tiles per block than the ring has stages."""
+    batch = ii.categorical_batch(B, T, A, seed=31 + B + T + A, p_done=0.02)
+    h = LossHyper(rho_bar=1.0, c_bar=1.0, clip_eps=0.3, vf_coef=0.5, ent_coef=0.01, kl_coef=0.0, rho_tw=1.0)
+    if dtype == torch.bfloat16:
+        P.check_categorical(oracle, batch, h, torch.bfloat16, torch.bfloat16, extra=False, rtol=P.RTOL_BF16,
+                            atol=P.ATOL_BF16)
+    else:
+        P.check_categorical(oracle, batch, h, extra=False)
+
+
 def test_optional_outputs_can_be_skipped_and_results_are_deterministic(oracle):
     cfg, batch = ii.make_config(1)
     h = P.f32_hyper(cfg.hyper)
