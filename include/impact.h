@@ -244,7 +244,7 @@ int32_t impact_loss_fwd_bwd_gaussian(
  * control loop that may not block on the driver's allocator; a process that was handed
  * fixed buffers by its parent and nothing else.  Such a caller has no workspace to pass.
  * This entry point therefore takes none: the per-block sums and the completion counter
- * live in a 33,024-byte array that is part of the library image (one copy on every GPU that
+ * live in a 98,560-byte array that is part of the library image (one copy on every GPU that
  * loads the library, held until the process exits).  Inputs, outputs, arithmetic and
  * results are those of impact_loss_fwd_bwd; nothing is allocated or freed, here or in
  * anything this call uses.

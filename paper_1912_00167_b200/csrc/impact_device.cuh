@@ -82,6 +82,12 @@ __device__ __forceinline__ void mbarrier_init(uint64_t* bar, uint32_t arrivals) 
     asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
     asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
 }
+// Initialisation of many barriers: each without a fence, then one fence_mbarrier_init() by every
+// initialising thread before the block-wide barrier that precedes their first use.
+__device__ __forceinline__ void mbarrier_init_nofence(uint64_t* bar, uint32_t arrivals) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+}
+__device__ __forceinline__ void fence_mbarrier_init() { asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory"); }
 __device__ __forceinline__ void mbarrier_expect_tx(uint64_t* bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes)
                  : "memory");
@@ -107,6 +113,16 @@ __device__ __forceinline__ bool mbarrier_wait(uint64_t* bar, uint32_t parity) {
         __nanosleep(64);  // a failed try returns early on this part: back off instead of spinning
     }
     return false;
+}
+// One look at the barrier, without waiting: has the phase with the given parity completed?
+__device__ __forceinline__ bool mbarrier_test(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.test_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return done != 0;
 }
 // The same wait for blocks in which several warps wait on one another's barriers: it also gives up
 // (at once) when `*abort_flag` is set, and sets it when it gives up itself, so that one wait that
@@ -143,6 +159,11 @@ __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy
 // All bulk stores of this thread have finished READING shared memory (it may be reused).
 __device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
+__device__ __forceinline__ unsigned long long global_timer_ns() {
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
 __device__ __forceinline__ float exp2_fast(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -600,54 +621,77 @@ __device__ __noinline__ void reduce_published_sums(const float* partials, unsign
     }
 }
 
-// reduce_published_sums for a group of NT threads inside a larger block: `gtid` is the thread's
-// index in the group, `bar_id` the group's named barrier.  Only one group of a grid ever runs it (the
-// one that drew the last ticket), so the shared scratch is not contended.
+// ---- sums published as tagged rows (persistent kernel) --------------------------------------
+// Every launch that uses a workspace has a number, kept in the workspace's third counter word: the
+// launch's tag is that word + 1 (never 0, which is what a cleared workspace holds), and the launch's
+// collecting group stores the tag back as its last act.  A group's row is eight (value, tag) pairs,
+// each written by ONE aligned 8-byte store, which the memory model makes indivisible: a reader that
+// sees this launch's tag in a pair sees this launch's value beside it.  So rows need no fence, no
+// atomic counter and no "last block" -- the collecting group simply reads every row until all its
+// pairs carry the tag (a bounded wait), and adds them in index order.
+__device__ __forceinline__ unsigned int launch_tag(const unsigned int* counter_words) {
+    unsigned int n;
+    asm volatile("ld.relaxed.gpu.global.u32 %0, [%1];" : "=r"(n) : "l"(counter_words + 2) : "memory");
+    return n + 1u == 0u ? 1u : n + 1u;
+}
+__device__ __forceinline__ void publish_tagged(unsigned long long* slot, float value, unsigned int tag) {
+    const unsigned long long v = ((unsigned long long)tag << 32) | (unsigned long long)__float_as_uint(value);
+    asm volatile("st.relaxed.gpu.global.u64 [%0], %1;" ::"l"(slot), "l"(v) : "memory");
+}
+
+// Run by the NT threads of one group (`gtid` in the group, named barrier `bar_id`): waits for `nrows`
+// tagged rows, adds them, writes the eight loss terms and advances the workspace's launch number.
+// Thread t owns column t % 8 of rows t / 8, t / 8 + NT / 8, ...: a row is read by eight neighbouring
+// lanes (64 contiguous bytes) and all of a thread's loads are in flight together, so a grid's worth of rows
+// costs one trip to L2.  The sum is a fixed fp32 tree (each thread its rows in index order, then lanes,
+// then warps) -- the rows are fp32 sums over whole tiles already.  Returns false if a row never showed up.
 template <int NT>
-__device__ __noinline__ void reduce_rows_group(const float* partials, int nrows, unsigned int* counter, float* loss_terms,
-                                                 float vf_coef, float ent_coef, float kl_coef, double M, int gtid,
-                                                 int bar_id) {
-    __shared__ double dred[NT / 32][kNumSums];
-    double s[kNumSums];
+__device__ __noinline__ bool reduce_tagged_rows(const unsigned long long* rows, int nrows, unsigned int tag,
+                                                  unsigned int* counter_words, float* loss_terms, float vf_coef,
+                                                  float ent_coef, float kl_coef, double M, int gtid, int bar_id,
+                                                  int* abort_flag) {
+    __shared__ float fred[NT / 32][8];
+    constexpr int kStride = NT / 8, kU = 10;
+    const int col = gtid & 7, rc = gtid >> 3;
+    float acc = 0.0f;
+    bool missing = false;
+    for (int base = rc; base < nrows && !missing; base += kStride * kU) {
+        unsigned long long v[kU];
+        unsigned int have = 0;
 #pragma unroll
-    for (int j = 0; j < kNumSums; ++j) s[j] = 0.0;
-    constexpr int kBatch = 8;
-    for (int first = gtid; first < nrows; first += NT * kBatch) {
-        float4 p0[kBatch], p1[kBatch];
+        for (int u = 0; u < kU; ++u)
+            if (base + kStride * u >= nrows) have |= 1u << u;  // beyond the last row: nothing to wait for
+        for (int tries = 0; tries < (1 << 22) && have != (1u << kU) - 1u; ++tries) {
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            const int r = first + u * NT;
-            if (r < nrows) {
-                p0[u] = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)r * 8));
-                p1[u] = __ldcg(reinterpret_cast<const float4*>(partials + (size_t)r * 8 + 4));
-            } else {
-                p0[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                p1[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-            }
+            for (int u = 0; u < kU; ++u)
+                if (!(have & (1u << u)))
+                    asm volatile("ld.relaxed.gpu.global.u64 %0, [%1];"
+                                 : "=l"(v[u]) : "l"(rows + (size_t)(base + kStride * u) * 8 + col) : "memory");
+#pragma unroll
+            for (int u = 0; u < kU; ++u)
+                if (!(have & (1u << u)) && (unsigned int)(v[u] >> 32) == tag) have |= 1u << u;
+            if (have != (1u << kU) - 1u && *reinterpret_cast<volatile int*>(abort_flag)) break;
         }
+        if (have != (1u << kU) - 1u) missing = true;
 #pragma unroll
-        for (int u = 0; u < kBatch; ++u) {
-            s[0] += p0[u].x; s[1] += p0[u].y; s[2] += p0[u].z; s[3] += p0[u].w;
-            s[4] += p1[u].x; s[5] += p1[u].y; s[6] += p1[u].z;
-        }
+        for (int u = 0; u < kU; ++u)
+            if (base + kStride * u < nrows) acc += __uint_as_float((unsigned int)v[u]);
     }
+    if (missing) *reinterpret_cast<volatile int*>(abort_flag) = 1;  // read back below, after the group's barrier
     const int lane = gtid & 31, warp = gtid >> 5;
-#pragma unroll
-    for (int j = 0; j < kNumSums; ++j) {
-        double x = s[j];
-#pragma unroll
-        for (int off = 16; off > 0; off >>= 1) x += __shfl_xor_sync(0xffffffffu, x, off);
-        if (lane == 0) dred[warp][j] = x;
-    }
+    acc += __shfl_xor_sync(0xffffffffu, acc, 8);
+    acc += __shfl_xor_sync(0xffffffffu, acc, 16);
+    if (lane < 8) fred[warp][lane] = acc;
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory");
     if (gtid == 0) {
         const double inv_m = 1.0 / M;
         double t[kNumSums];
 #pragma unroll
         for (int j = 0; j < kNumSums; ++j) {
-            double x = 0.0;
-            for (int w = 0; w < NT / 32; ++w) x += dred[w][j];
-            t[j] = x * inv_m;
+            float x = 0.0f;
+#pragma unroll
+            for (int w = 0; w < NT / 32; ++w) x += fred[w][j];
+            t[j] = (double)x * inv_m;
         }
         const double l_pi = -t[0], l_v = t[1], ent = t[2], kl = t[3];
         loss_terms[0] = (float)(l_pi + (double)vf_coef * l_v - (double)ent_coef * ent + (double)kl_coef * kl);
@@ -658,8 +702,9 @@ __device__ __noinline__ void reduce_rows_group(const float* partials, int nrows,
         loss_terms[5] = (float)t[4];
         loss_terms[6] = (float)t[5];
         loss_terms[7] = (float)t[6];
-        *counter = 0u;
+        counter_words[2] = tag;
     }
+    return *reinterpret_cast<volatile int*>(abort_flag) == 0;
 }
 
 }  // namespace dev

@@ -43,6 +43,7 @@ struct CatParams {
     float* advantage;
     float* partials;
     unsigned int* counter;
+    unsigned long long* tagged_rows;  // persistent kernel: rows of (value, launch tag) pairs, see publish_tagged_row
     TileGeometry geo;
     LossScalars k;
     int A, As;
@@ -811,8 +812,6 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
 constexpr int kWsMaxStages = 24;
 constexpr int kWsGroups = 4;  // consumer groups per block: 16 consumer warps + the producer warp, <= 120 registers each
 
-__device__ __forceinline__ void group_barrier(int id) { asm volatile("bar.sync %0, 128;" ::"r"(id) : "memory"); }
-
 // Row passes of one step, shared by the kernels with a compile-time action count.  `zr` / `tr`
 // point at the thread's learner / target row in shared memory.
 template <typename LT, int A>
@@ -863,7 +862,7 @@ struct RowMath {
 // default ratio and importance weights, no optional outputs -- with those branches compiled out.
 template <typename LT, typename GT, int A, int C, bool kPlain>
 __global__ void __launch_bounds__(C * 128 + 32, 1)
-impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W) {
+impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W, const int pace_ns) {
     constexpr int NT = 128;
     constexpr int NP = (A + 1) / 2;
     constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
@@ -872,9 +871,9 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     using RM = RowMath<LT, A>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kWsMaxStages], empty_bar[kWsMaxStages];
+    __shared__ __align__(8) uint64_t sums_bar[C];  // a group's final sums are in `red`
     __shared__ float2 warp_agg[C][NT / 32];
     __shared__ __align__(16) float red[C][NT / 32][8];
-    __shared__ int is_last_s[C];
     __shared__ int abort_s;
 
     const int tid = threadIdx.x, lane = tid & 31;
@@ -884,52 +883,95 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     const int rows_full = g.G * (int)g.T;                                                // rows of a full tile
     const long long total_rows = g.B * g.T;
 
-    if (tid == 0) {
-        for (int s = 0; s < S; ++s) {
-            dev::mbarrier_init(&full_bar[s], 1);
-            dev::mbarrier_init(&empty_bar[s], NT / 32);  // one arrival per consumer warp
-        }
-        abort_s = 0;
+    // one barrier per thread, then a single fence
+    if (tid < S) {
+        dev::mbarrier_init_nofence(&full_bar[tid], 1);
+        dev::mbarrier_init_nofence(&empty_bar[tid], NT / 32);  // one arrival per consumer warp
+    } else if (tid >= 32 && tid < 32 + C) {
+        dev::mbarrier_init_nofence(&sums_bar[tid - 32], NT / 32);
     }
+    if (tid == 0) abort_s = 0;
+    dev::fence_mbarrier_init();
     __syncthreads();
     grid_dependency_wait();  // everything above touches only this block's shared memory
 
     if (tid >= C * NT) {
-        // ---- producer warp: one lane streams the block's tiles into the ring ------------------
-        if (lane != 0) return;
-        const LT* gl = static_cast<const LT*>(p.learner_logits) + (long long)blockIdx.x * rows_full * A;
-        const LT* gt = static_cast<const LT*>(p.target_logits) + (long long)blockIdx.x * rows_full * A;
-        const long long step_elems = (long long)gridDim.x * rows_full * A;
-        long long rows_left = total_rows - (long long)blockIdx.x * rows_full;
-        const long long step_rows = (long long)gridDim.x * rows_full;
-        int s = 0, ws = 0;         // stage of tile n, stage of tile n - W
-        uint32_t ph = 0, wph = 0;  // their phase parities
-        for (int n = 0; n < n_tiles; ++n) {
-            bool ok = true;
-            if (n >= S) ok = dev::mbarrier_wait(&empty_bar[s], ph ^ 1u, &abort_s);   // the stage's previous tile has left
-            if (ok && n >= W) ok = dev::mbarrier_wait(&full_bar[ws], wph, &abort_s);  // at most W tiles in flight
-            if (!ok) { atomicExch(p.counter + 1, 1u); return; }
-            const int nrows = rows_left < rows_full ? (int)rows_left : rows_full;
-            unsigned char* const d0 = smem_raw + s * kStageBytes;
-            unsigned char* const d1 = d0 + NT * kInRow;
-            const uint32_t bytes = (uint32_t)nrows * kInRow;
-            if (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | bytes) & 15u) == 0) {
-                dev::mbarrier_expect_tx(&full_bar[s], 2 * bytes);
-                dev::bulk_load(d0, gl, bytes, &full_bar[s]);
-                dev::bulk_load(d1, gt, bytes, &full_bar[s]);
-            } else {  // ragged or unaligned slab: element by element
-                const int nelem = nrows * A;
-                for (int e = 0; e < nelem; ++e) {
-                    reinterpret_cast<LT*>(d0)[e] = gl[e];
-                    reinterpret_cast<LT*>(d1)[e] = gt[e];
+        // ---- producer warp: lane 0 streams the block's tiles into the ring --------------------
+        if (lane == 0) {
+            const LT* gl = static_cast<const LT*>(p.learner_logits) + (long long)blockIdx.x * rows_full * A;
+            const LT* gt = static_cast<const LT*>(p.target_logits) + (long long)blockIdx.x * rows_full * A;
+            const long long step_elems = (long long)gridDim.x * rows_full * A;
+            long long rows_left = total_rows - (long long)blockIdx.x * rows_full;
+            const long long step_rows = (long long)gridDim.x * rows_full;
+            int s = 0, ws = 0;         // stage of tile n, stage of tile n - W
+            uint32_t ph = 0, wph = 0;  // their phase parities
+            // The first tiles are sent off one by one at the pace at which HBM can deliver them to this SM, not
+            // all at once: requests in flight share the bandwidth, so W tiles asked for together all land late
+            // together, while paced ones land in order and the arithmetic starts a microsecond earlier.
+            const unsigned long long t_begin = dev::global_timer_ns();
+            for (int n = 0; n < n_tiles; ++n) {
+                bool ok = true;
+                if (n >= S) ok = dev::mbarrier_wait(&empty_bar[s], ph ^ 1u, &abort_s);   // the stage's previous tile has left
+                if (ok && n >= W) ok = dev::mbarrier_wait(&full_bar[ws], wph, &abort_s);  // at most W tiles in flight
+                if (!ok) { atomicExch(p.counter + 1, 1u); break; }
+                if (n > 0 && n < 2 * W) {
+                    const unsigned long long due = (unsigned long long)n * (unsigned)pace_ns;
+                    for (int spin = 0; spin < 4096 && dev::global_timer_ns() - t_begin < due; ++spin) {}
                 }
-                dev::mbarrier_arrive(&full_bar[s]);
+                const int nrows = rows_left < rows_full ? (int)rows_left : rows_full;
+                unsigned char* const d0 = smem_raw + s * kStageBytes;
+                unsigned char* const d1 = d0 + NT * kInRow;
+                const uint32_t bytes = (uint32_t)nrows * kInRow;
+                if (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | bytes) & 15u) == 0) {
+                    dev::mbarrier_expect_tx(&full_bar[s], 2 * bytes);
+                    dev::bulk_load(d0, gl, bytes, &full_bar[s]);
+                    dev::bulk_load(d1, gt, bytes, &full_bar[s]);
+                } else {  // ragged or unaligned slab: element by element
+                    const int nelem = nrows * A;
+                    for (int e = 0; e < nelem; ++e) {
+                        reinterpret_cast<LT*>(d0)[e] = gl[e];
+                        reinterpret_cast<LT*>(d1)[e] = gt[e];
+                    }
+                    dev::mbarrier_arrive(&full_bar[s]);
+                }
+                gl += step_elems;
+                gt += step_elems;
+                rows_left -= step_rows;
+                if (++s == S) { s = 0; ph ^= 1u; }
+                if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
             }
-            gl += step_elems;
-            gt += step_elems;
-            rows_left -= step_rows;
-            if (++s == S) { s = 0; ph ^= 1u; }
-            if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
+        }
+        __syncwarp();
+        // ---- then it publishes the block's sums, once every group's are final: one row of (value, tag)
+        // pairs, the tag being this launch's number.  A pair is one 8-byte store, so whoever reads the tag of
+        // this launch reads this launch's value with it: no fence, no atomic, no round trip.  The groups'
+        // barriers are polled without blocking and their sums added in group order, whatever order they
+        // arrive in.
+        const unsigned int tag = dev::launch_tag(p.counter);
+        float yc[C];
+        unsigned int todo = (1u << C) - 1u;
+        for (unsigned int spin = 0; todo != 0u && spin < (1u << 24); ++spin) {
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                if (!(todo & (1u << c))) continue;
+                bool ready = (lane == 0) && dev::mbarrier_test(&sums_bar[c], 0u);
+                ready = __shfl_sync(0xffffffffu, ready, 0);
+                if (!ready) continue;
+                float y = 0.0f;
+#pragma unroll
+                for (int w = 0; w < NT / 32; ++w) y += red[c][w][lane & 7];
+                yc[c] = y;
+                todo &= ~(1u << c);
+            }
+            if (*reinterpret_cast<volatile int*>(&abort_s)) break;
+        }
+        if (todo == 0u) {
+            float y = yc[0];
+#pragma unroll
+            for (int c = 1; c < C; ++c) y += yc[c];
+            if (lane < 8) dev::publish_tagged(p.tagged_rows + (size_t)blockIdx.x * 8 + lane, y, tag);
+        } else if (lane == 0) {
+            atomicExch(p.counter + 1, 1u);  // a group never delivered its sums
         }
         return;
     }
@@ -970,6 +1012,21 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
 
     float t_surr = 0.0f, t_val = 0.0f, t_ent = 0.0f, t_ratio = 0.0f, t_kl = 0.0f;
     int n_clip = 0, n_trunc = 0;
+    // The group's sums, once final: a butterfly per warp into `red`, then one arrival per warp tells the
+    // producer warp that the row can be published (fixed order throughout).
+    auto hand_over_sums = [&]() {
+        const float x = dev::warp_sum4(t_surr, t_val, t_ent, t_ratio);
+        const float xk = want_kl ? dev::warp_sum(t_kl) : 0.0f;
+        if ((lane & 7) == 0) red[grp][gwarp][lane == 24 ? 6 : (lane >> 3)] = x;
+        if (lane == 0) {
+            red[grp][gwarp][3] = xk;
+            red[grp][gwarp][4] = (float)n_clip;
+            red[grp][gwarp][5] = (float)n_trunc;
+            red[grp][gwarp][7] = 0.0f;
+        }
+        __syncwarp();
+        if (lane == 0) dev::mbarrier_arrive(&sums_bar[grp]);
+    };
     bool pending = false;  // lane 0 of each warp: a store of this warp may still be reading its stage
     int pending_stage = 0;
 
@@ -1042,6 +1099,9 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         }
         n_clip += __popc(__ballot_sync(0xffffffffu, active && clipped));
         n_trunc += __popc(__ballot_sync(0xffffffffu, active && truncated));
+        // the group's sums are final after its last tile's scan: handed over here, they are published while
+        // that tile's gradient pass runs
+        if (n + C >= n_tiles) hand_over_sums();
 
         // ---- gradients: row_j = e_j (ga z_j + gb) [- kl_coef pi_target_j / M], then the taken action's entry
         {
@@ -1112,33 +1172,16 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         while (s >= S) { s -= S; ph ^= 1u; }
     }
 
-    // ---- the group's sums: one published row per group; the group that draws the last ticket adds all rows
-    {
-        const float x = dev::warp_sum4(t_surr, t_val, t_ent, t_ratio);
-        const float xk = want_kl ? dev::warp_sum(t_kl) : 0.0f;
-        if ((lane & 7) == 0) red[grp][gwarp][lane == 24 ? 6 : (lane >> 3)] = x;
-        if (lane == 0) {
-            red[grp][gwarp][3] = xk;
-            red[grp][gwarp][4] = (float)n_clip;
-            red[grp][gwarp][5] = (float)n_trunc;
-            red[grp][gwarp][7] = 0.0f;
-        }
+    // a group without tiles still hands over its (zero) sums, so that every row of the grid is defined
+    if (grp >= n_tiles) hand_over_sums();
+    // ---- one group of the grid (block 0's, the one with that block's last tile) collects every block's row
+    // as it appears and writes the loss terms
+    if (blockIdx.x == 0 && grp == (n_tiles - 1) % C) {
+        if (!dev::reduce_tagged_rows<NT>(p.tagged_rows, (int)gridDim.x, dev::launch_tag(p.counter), p.counter,
+                                         p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, (double)g.B * (double)g.T,
+                                         gtid, bar_id, &abort_s))
+            if (gtid == 0) atomicExch(p.counter + 1, 1u);
     }
-    group_barrier(bar_id);
-    if (gwarp == 0) {
-        if (lane < 8) {
-            float x = 0.0f;
-#pragma unroll
-            for (int w = 0; w < NT / 32; ++w) x += red[grp][w][lane];
-            p.partials[((size_t)blockIdx.x * C + grp) * 8 + lane] = x;
-        }
-        __syncwarp();
-        if (lane == 0) is_last_s[grp] = (dev::take_ticket(p.counter) == gridDim.x * C - 1) ? 1 : 0;
-    }
-    group_barrier(bar_id);
-    if (is_last_s[grp])
-        dev::reduce_rows_group<NT>(p.partials, (int)gridDim.x * C, p.counter, p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef,
-                                   (double)g.B * (double)g.T, gtid, bar_id);
     if (lane == 0) dev::bulk_store_wait_read();  // shared memory must outlive the stores' reads
 }
 
@@ -1487,7 +1530,8 @@ __global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kern
 // Host side
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxGridBlocks = 4096;  // upper bound on blocks of a loss launch (sizes the workspace)
-constexpr size_t kCounterBytes = 256; // counter lives in its own 256-byte line after the partials
+constexpr size_t kCounterBytes = 256; // words after the partials: [0] completion counter, [1] error flag, [2] launch number
+constexpr int kMaxTaggedRows = 1024;  // rows of eight (value, tag) pairs after the counter words: one per block of the persistent kernel
 
 int pad_odd(int w) { return (w & 1) ? w : w + 1; }
 
@@ -1630,7 +1674,9 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
         configured_device = di->device;
     }
     const long long grid = p.geo.nchunks < di->sm_count ? p.geo.nchunks : di->sm_count;
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W));
+    // time in which HBM delivers one tile's logits to one SM at the device's nominal bandwidth
+    const int pace_ns = (int)((double)(2 * (size_t)kRegTileRows * A * sizeof(LT)) / di->hbm_bytes_per_ns_per_sm);
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W, pace_ns));
     return IMPACT_OK;
 }
 
@@ -1726,7 +1772,7 @@ using namespace impact;
 
 extern "C" size_t impact_loss_workspace_bytes(int64_t B, int64_t T) {
     if (B <= 0 || T <= 0) return 0;
-    return (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes;
+    return (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes + (size_t)kMaxTaggedRows * 8 * sizeof(unsigned long long);
 }
 
 extern "C" int32_t impact_loss_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
@@ -1794,6 +1840,8 @@ extern "C" int32_t impact_loss_fwd_bwd(
     p.partials = static_cast<float*>(workspace);
     p.counter = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) +
                                                 (size_t)kMaxGridBlocks * 8 * sizeof(float));
+    p.tagged_rows = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) +
+                                                          (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes);
     p.A = A;
     return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
                            di, static_cast<cudaStream_t>(stream));
@@ -1886,10 +1934,12 @@ namespace impact {
 namespace {
 
 constexpr int kStaticMaxBlocks = 1024;  // tiles (= blocks) the built-in scratch has room for
-constexpr size_t kStaticScratchBytes = (size_t)kStaticMaxBlocks * 8 * sizeof(float) + kCounterBytes;
+constexpr size_t kStaticScratchBytes = (size_t)kStaticMaxBlocks * 8 * sizeof(float) + kCounterBytes +
+                                       (size_t)kMaxTaggedRows * 8 * sizeof(unsigned long long);
 
-// Scratch that lives in the library image: per-block sums first, the completion counter in
-// the last 256 bytes.  Every device that loads the library carries its own copy.
+// Scratch that lives in the library image, laid out like a workspace: per-block sums, 256 bytes of
+// counter words, the tagged rows of the persistent kernel.  Every device that loads the library
+// carries its own copy.
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
 // Device address of g_static_scratch on the current device.  In host code the symbol's name
@@ -1944,9 +1994,11 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     st = static_scratch_address(di, &scratch);
     if (st != IMPACT_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // the scratch keeps whatever the previous call left; the counter is what has to start at zero
+    // the scratch keeps whatever the previous call left; the completion counter and the error word are
+    // what has to start at zero (the launch number next to them must live on: it is what tells this call's
+    // rows from the previous call's)
     unsigned char* counter = scratch + (size_t)kStaticMaxBlocks * 8 * sizeof(float);
-    IMPACT_CUDA_TRY(cudaMemsetAsync(counter, 0, kCounterBytes, s));
+    IMPACT_CUDA_TRY(cudaMemsetAsync(counter, 0, 2 * sizeof(unsigned int), s));
 
     p.learner_logits = learner_logits;
     p.target_logits = target_logits;
@@ -1963,6 +2015,7 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     p.advantage = advantage;
     p.partials = reinterpret_cast<float*>(scratch);
     p.counter = reinterpret_cast<unsigned int*>(counter);
+    p.tagged_rows = reinterpret_cast<unsigned long long*>(counter + kCounterBytes);
     // the same kernels, chosen the same way, as impact_loss_fwd_bwd
     return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
                            di, s);
