@@ -149,6 +149,10 @@ __device__ __forceinline__ void bulk_load(void* smem_dst, const void* gmem_src, 
                  ::"r"(smem_addr(smem_dst)), "l"(__cvta_generic_to_global(gmem_src)), "r"(bytes),
                  "r"(smem_addr(bar)) : "memory");
 }
+// Asks L2 to fetch a contiguous range (16-byte aligned, a multiple of 16 bytes); nothing waits for it.
+__device__ __forceinline__ void bulk_prefetch_l2(const void* gmem_src, uint32_t bytes) {
+    asm volatile("cp.async.bulk.prefetch.L2.global [%0], %1;" ::"l"(__cvta_generic_to_global(gmem_src)), "r"(bytes) : "memory");
+}
 __device__ __forceinline__ void bulk_store(void* gmem_dst, const void* smem_src, uint32_t bytes) {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
                  ::"l"(__cvta_generic_to_global(gmem_dst)), "r"(smem_addr(smem_src)), "r"(bytes) : "memory");

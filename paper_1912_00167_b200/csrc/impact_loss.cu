@@ -883,62 +883,85 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     const int rows_full = g.G * (int)g.T;                                                // rows of a full tile
     const long long total_rows = g.B * g.T;
 
-    // one barrier per thread, then a single fence
-    if (tid < S) {
-        dev::mbarrier_init_nofence(&full_bar[tid], 1);
-        dev::mbarrier_init_nofence(&empty_bar[tid], NT / 32);  // one arrival per consumer warp
-    } else if (tid >= 32 && tid < 32 + C) {
-        dev::mbarrier_init_nofence(&sums_bar[tid - 32], NT / 32);
-    }
-    if (tid == 0) abort_s = 0;
-    dev::fence_mbarrier_init();
-    __syncthreads();
-    grid_dependency_wait();  // everything above touches only this block's shared memory
-
     if (tid >= C * NT) {
-        // ---- producer warp: lane 0 streams the block's tiles into the ring --------------------
+        // ---- producer warp: sets up the barriers, then lane 0 streams the block's tiles into the ring --------
+        if (lane < S) {
+            dev::mbarrier_init_nofence(&full_bar[lane], 1);
+            dev::mbarrier_init_nofence(&empty_bar[lane], NT / 32);  // one arrival per consumer warp
+        }
+        if (lane < C) dev::mbarrier_init_nofence(&sums_bar[lane], NT / 32);
+        if (lane == 0) abort_s = 0;
+        dev::fence_mbarrier_init();
+        __syncwarp();
+
+        const LT* gl = static_cast<const LT*>(p.learner_logits) + (long long)blockIdx.x * rows_full * A;
+        const LT* gt = static_cast<const LT*>(p.target_logits) + (long long)blockIdx.x * rows_full * A;
+        const long long step_elems = (long long)gridDim.x * rows_full * A;
+        long long rows_left = total_rows - (long long)blockIdx.x * rows_full;
+        const long long step_rows = (long long)gridDim.x * rows_full;
+        const int n_first = n_tiles < W ? n_tiles : W;
+        // While the kernel before this one on the stream is still finishing, ask L2 for the first tiles: a
+        // prefetch changes nothing that a program can observe (L2 is where the device's writes meet, so later
+        // writes to these addresses are not lost), but the pages are mapped and the bytes on their way
+        // when the dependency resolves.
         if (lane == 0) {
-            const LT* gl = static_cast<const LT*>(p.learner_logits) + (long long)blockIdx.x * rows_full * A;
-            const LT* gt = static_cast<const LT*>(p.target_logits) + (long long)blockIdx.x * rows_full * A;
-            const long long step_elems = (long long)gridDim.x * rows_full * A;
-            long long rows_left = total_rows - (long long)blockIdx.x * rows_full;
-            const long long step_rows = (long long)gridDim.x * rows_full;
-            int s = 0, ws = 0;         // stage of tile n, stage of tile n - W
-            uint32_t ph = 0, wph = 0;  // their phase parities
-            // The first tiles are sent off one by one at the pace at which HBM can deliver them to this SM, not
-            // all at once: requests in flight share the bandwidth, so W tiles asked for together all land late
-            // together, while paced ones land in order and the arithmetic starts a microsecond earlier.
-            const unsigned long long t_begin = dev::global_timer_ns();
-            for (int n = 0; n < n_tiles; ++n) {
+            const LT *pl = gl, *pt = gt;
+            long long left = rows_left;
+            for (int n = 0; n < n_first; ++n) {
+                const uint32_t bytes = (uint32_t)(left < rows_full ? left : rows_full) * kInRow;
+                if (((reinterpret_cast<uintptr_t>(pl) | reinterpret_cast<uintptr_t>(pt) | bytes) & 15u) == 0) {
+                    dev::bulk_prefetch_l2(pl, bytes);
+                    dev::bulk_prefetch_l2(pt, bytes);
+                }
+                pl += step_elems; pt += step_elems; left -= step_rows;
+            }
+        }
+        grid_dependency_wait();
+
+        int s = 0, ws = 0;         // stage of tile n, stage of tile n - W
+        uint32_t ph = 0, wph = 0;  // their phase parities
+        // The first tiles are sent off one by one at the pace at which HBM can deliver them to this SM, not
+        // all at once: requests in flight share the bandwidth, so W tiles asked for together all land late
+        // together, while paced ones land in order.
+        const unsigned long long t_begin = dev::global_timer_ns();
+        auto send_tile = [&](int n) {
+            if (n > 0 && n < 2 * W) {
+                const unsigned long long due = (unsigned long long)n * (unsigned)pace_ns;
+                for (int spin = 0; spin < 4096 && dev::global_timer_ns() - t_begin < due; ++spin) {}
+            }
+            const int nrows = rows_left < rows_full ? (int)rows_left : rows_full;
+            unsigned char* const d0 = smem_raw + s * kStageBytes;
+            unsigned char* const d1 = d0 + NT * kInRow;
+            const uint32_t bytes = (uint32_t)nrows * kInRow;
+            if (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | bytes) & 15u) == 0) {
+                dev::mbarrier_expect_tx(&full_bar[s], 2 * bytes);
+                dev::bulk_load(d0, gl, bytes, &full_bar[s]);
+                dev::bulk_load(d1, gt, bytes, &full_bar[s]);
+            } else {  // ragged or unaligned slab: element by element
+                const int nelem = nrows * A;
+                for (int e = 0; e < nelem; ++e) {
+                    reinterpret_cast<LT*>(d0)[e] = gl[e];
+                    reinterpret_cast<LT*>(d1)[e] = gt[e];
+                }
+                dev::mbarrier_arrive(&full_bar[s]);
+            }
+            gl += step_elems;
+            gt += step_elems;
+            rows_left -= step_rows;
+            if (++s == S) { s = 0; ph ^= 1u; }
+            if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
+        };
+        // the first W tiles need no wait, and leave before the rest of the block has even started
+        if (lane == 0)
+            for (int n = 0; n < n_first; ++n) send_tile(n);
+        __syncthreads();  // the barriers are set up: the consumer warps may use them
+        if (lane == 0) {
+            for (int n = n_first; n < n_tiles; ++n) {
                 bool ok = true;
                 if (n >= S) ok = dev::mbarrier_wait(&empty_bar[s], ph ^ 1u, &abort_s);   // the stage's previous tile has left
                 if (ok && n >= W) ok = dev::mbarrier_wait(&full_bar[ws], wph, &abort_s);  // at most W tiles in flight
                 if (!ok) { atomicExch(p.counter + 1, 1u); break; }
-                if (n > 0 && n < 2 * W) {
-                    const unsigned long long due = (unsigned long long)n * (unsigned)pace_ns;
-                    for (int spin = 0; spin < 4096 && dev::global_timer_ns() - t_begin < due; ++spin) {}
-                }
-                const int nrows = rows_left < rows_full ? (int)rows_left : rows_full;
-                unsigned char* const d0 = smem_raw + s * kStageBytes;
-                unsigned char* const d1 = d0 + NT * kInRow;
-                const uint32_t bytes = (uint32_t)nrows * kInRow;
-                if (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | bytes) & 15u) == 0) {
-                    dev::mbarrier_expect_tx(&full_bar[s], 2 * bytes);
-                    dev::bulk_load(d0, gl, bytes, &full_bar[s]);
-                    dev::bulk_load(d1, gt, bytes, &full_bar[s]);
-                } else {  // ragged or unaligned slab: element by element
-                    const int nelem = nrows * A;
-                    for (int e = 0; e < nelem; ++e) {
-                        reinterpret_cast<LT*>(d0)[e] = gl[e];
-                        reinterpret_cast<LT*>(d1)[e] = gt[e];
-                    }
-                    dev::mbarrier_arrive(&full_bar[s]);
-                }
-                gl += step_elems;
-                gt += step_elems;
-                rows_left -= step_rows;
-                if (++s == S) { s = 0; ph ^= 1u; }
-                if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
+                send_tile(n);
             }
         }
         __syncwarp();
@@ -1030,9 +1053,11 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     bool pending = false;  // lane 0 of each warp: a store of this warp may still be reading its stage
     int pending_stage = 0;
 
+    grid_dependency_wait();
     bool active = in_layout && row < total_rows;
     StepRaw cur;
     if (grp < n_tiles) cur = load_scalars(row, traj, active);
+    __syncthreads();  // the producer warp has set up the barriers
     int s = grp % S;
     uint32_t ph = (uint32_t)(grp / S) & 1u;
 
