@@ -121,8 +121,9 @@ size_t impact_loss_workspace_bytes(int64_t B, int64_t T);
 
 /*
  * Clears a workspace (enqueues a memset on `stream`).  A workspace must be cleared once
- * before its first use; every loss call leaves it cleared again, so one buffer serves any
- * number of calls on ONE stream.  Calls that may overlap on the GPU need a workspace each.
+ * before its first use; every loss call leaves it ready for the next (it also keeps a count
+ * of the launches that used it, which tells one launch's partial sums from the previous
+ * one's), so one buffer serves any number of calls on ONE stream.  Calls that may overlap on the GPU need a workspace each.
  */
 int32_t impact_loss_workspace_init(void* workspace, size_t workspace_bytes, void* stream);
 
