@@ -28,13 +28,7 @@ const DeviceInfo* current_device_info() {
         e = cudaDeviceGetAttribute(&di.sm_count, cudaDevAttrMultiProcessorCount, dev);
         if (e == cudaSuccess)
             e = cudaDeviceGetAttribute(&di.max_smem_optin, cudaDevAttrMaxSharedMemoryPerBlockOptin, dev);
-        int mem_khz = 0, bus_bits = 0;
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&mem_khz, cudaDevAttrMemoryClockRate, dev);
-        if (e == cudaSuccess) e = cudaDeviceGetAttribute(&bus_bits, cudaDevAttrGlobalMemoryBusWidth, dev);
         if (e != cudaSuccess) { record_cuda_error(e); return nullptr; }
-        // bytes per ns = 2 transfers per clock x clock in GHz x bus bytes; 8 TB/s / 148 SMs = 55 B/ns on B200
-        di.hbm_bytes_per_ns_per_sm = 2.0 * (mem_khz * 1e-6) * (bus_bits / 8.0) / (di.sm_count > 0 ? di.sm_count : 1);
-        if (!(di.hbm_bytes_per_ns_per_sm > 1.0)) di.hbm_bytes_per_ns_per_sm = 55.0;
         infos[dev] = di;
         ready[dev] = true;
     }

@@ -18,7 +18,6 @@ struct DeviceInfo {
     int device = -1;
     int sm_count = 0;
     int max_smem_optin = 0;
-    double hbm_bytes_per_ns_per_sm = 0.0;  // nominal memory bandwidth (clock x bus width, double data rate) / SMs
 };
 // Returns nullptr (and records the error) when no CUDA device is usable.
 const DeviceInfo* current_device_info();

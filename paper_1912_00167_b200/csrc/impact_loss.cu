@@ -862,7 +862,7 @@ struct RowMath {
 // default ratio and importance weights, no optional outputs -- with those branches compiled out.
 template <typename LT, typename GT, int A, int C, bool kPlain>
 __global__ void __launch_bounds__(C * 128 + 32, 1)
-impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W, const int pace_ns) {
+impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W) {
     constexpr int NT = 128;
     constexpr int NP = (A + 1) / 2;
     constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
@@ -884,7 +884,33 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     const long long total_rows = g.B * g.T;
 
     if (tid >= C * NT) {
-        // ---- producer warp: sets up the barriers, then lane 0 streams the block's tiles into the ring --------
+        // ---- producer warp ----------------------------------------------------------------------------------
+        const long long step_elems = (long long)gridDim.x * rows_full * A;
+        const long long step_rows = (long long)gridDim.x * rows_full;
+        const int n_first = n_tiles < W ? n_tiles : W;
+        // First of all, while the kernel before this one on the stream is still finishing, lane n asks L2 for
+        // the block's n-th tile (logits and per-step scalars): a prefetch changes nothing that a program can
+        // observe (L2 is where the device's writes meet, so later writes to these addresses are not lost), but
+        // the pages are mapped and the bytes on their way when the dependency resolves.
+        if (lane < n_first) {
+            const long long row0 = (long long)blockIdx.x * rows_full + lane * step_rows;
+            const long long left = total_rows - row0;
+            const uint32_t nrows = (uint32_t)(left < rows_full ? left : rows_full);
+            const LT* const pl = static_cast<const LT*>(p.learner_logits) + row0 * A;
+            const LT* const pt = static_cast<const LT*>(p.target_logits) + row0 * A;
+            if (((reinterpret_cast<uintptr_t>(pl) | reinterpret_cast<uintptr_t>(pt) | (nrows * kInRow)) & 15u) == 0) {
+                dev::bulk_prefetch_l2(pl, nrows * kInRow);
+                dev::bulk_prefetch_l2(pt, nrows * kInRow);
+            }
+            if (((row0 | nrows) & 3) == 0) {  // 4-byte scalars: 16-byte granules
+                dev::bulk_prefetch_l2(p.actions + row0, nrows * 4u);
+                dev::bulk_prefetch_l2(p.worker_logp + row0, nrows * 4u);
+                dev::bulk_prefetch_l2(p.rewards + row0, nrows * 4u);
+                dev::bulk_prefetch_l2(p.discounts + row0, nrows * 4u);
+                dev::bulk_prefetch_l2(p.values + row0, nrows * 4u);
+            }
+        }
+        // then the barriers
         if (lane < S) {
             dev::mbarrier_init_nofence(&full_bar[lane], 1);
             dev::mbarrier_init_nofence(&empty_bar[lane], NT / 32);  // one arrival per consumer warp
@@ -894,41 +920,15 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         dev::fence_mbarrier_init();
         __syncwarp();
 
+        // lane 0 streams the block's tiles into the ring
         const LT* gl = static_cast<const LT*>(p.learner_logits) + (long long)blockIdx.x * rows_full * A;
         const LT* gt = static_cast<const LT*>(p.target_logits) + (long long)blockIdx.x * rows_full * A;
-        const long long step_elems = (long long)gridDim.x * rows_full * A;
         long long rows_left = total_rows - (long long)blockIdx.x * rows_full;
-        const long long step_rows = (long long)gridDim.x * rows_full;
-        const int n_first = n_tiles < W ? n_tiles : W;
-        // While the kernel before this one on the stream is still finishing, ask L2 for the first tiles: a
-        // prefetch changes nothing that a program can observe (L2 is where the device's writes meet, so later
-        // writes to these addresses are not lost), but the pages are mapped and the bytes on their way
-        // when the dependency resolves.
-        if (lane == 0) {
-            const LT *pl = gl, *pt = gt;
-            long long left = rows_left;
-            for (int n = 0; n < n_first; ++n) {
-                const uint32_t bytes = (uint32_t)(left < rows_full ? left : rows_full) * kInRow;
-                if (((reinterpret_cast<uintptr_t>(pl) | reinterpret_cast<uintptr_t>(pt) | bytes) & 15u) == 0) {
-                    dev::bulk_prefetch_l2(pl, bytes);
-                    dev::bulk_prefetch_l2(pt, bytes);
-                }
-                pl += step_elems; pt += step_elems; left -= step_rows;
-            }
-        }
         grid_dependency_wait();
 
         int s = 0, ws = 0;         // stage of tile n, stage of tile n - W
         uint32_t ph = 0, wph = 0;  // their phase parities
-        // The first tiles are sent off one by one at the pace at which HBM can deliver them to this SM, not
-        // all at once: requests in flight share the bandwidth, so W tiles asked for together all land late
-        // together, while paced ones land in order.
-        const unsigned long long t_begin = dev::global_timer_ns();
         auto send_tile = [&](int n) {
-            if (n > 0 && n < 2 * W) {
-                const unsigned long long due = (unsigned long long)n * (unsigned)pace_ns;
-                for (int spin = 0; spin < 4096 && dev::global_timer_ns() - t_begin < due; ++spin) {}
-            }
             const int nrows = rows_left < rows_full ? (int)rows_left : rows_full;
             unsigned char* const d0 = smem_raw + s * kStageBytes;
             unsigned char* const d1 = d0 + NT * kInRow;
@@ -1699,9 +1699,7 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
         configured_device = di->device;
     }
     const long long grid = p.geo.nchunks < di->sm_count ? p.geo.nchunks : di->sm_count;
-    // time in which HBM delivers one tile's logits to one SM at the device's nominal bandwidth
-    const int pace_ns = (int)((double)(2 * (size_t)kRegTileRows * A * sizeof(LT)) / di->hbm_bytes_per_ns_per_sm);
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W, pace_ns));
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W));
     return IMPACT_OK;
 }
 
