@@ -68,6 +68,7 @@ struct GaussParams {
     float* advantage;
     float* partials;
     unsigned int* counter;
+    unsigned long long* tagged_rows;
     TileGeometry geo;
     LossScalars k;
     int D, Ds;
@@ -1552,6 +1553,346 @@ __global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kern
 }
 
 // ------------------------------------------------------------------------------------------
+// Diagonal-Gaussian policy, persistent warp-specialised form (trajectories of at most 128 steps)
+// ------------------------------------------------------------------------------------------
+// The structure of impact_loss_categorical_ws_kernel with five input slabs per tile (learner mean /
+// log-std, target mean / log-std, actions) and two output slabs (dmean, dlogstd, written over the
+// learner's): a producer warp streams tiles through the ring, C consumer groups take them as they
+// land, every warp stores its own rows, the block's sums leave as one tagged row.  Row arithmetic is
+// that of impact_loss_gaussian_reg_kernel (log-probabilities accumulated in fp64).
+template <int D, int C>
+__global__ void __launch_bounds__(C * 128 + 32, 1)
+impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int S, const int W) {
+    constexpr int NT = 128;
+    constexpr int kRow = D * (int)sizeof(float);
+    constexpr int kSlab = NT * kRow;
+    constexpr int kStageBytes = 5 * kSlab;
+    constexpr float kLog2e = 1.4426950408889634f;
+    constexpr float kHalfLog2Pi = 0.91893853320467274178f;
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    __shared__ __align__(8) uint64_t full_bar[kWsMaxStages], empty_bar[kWsMaxStages];
+    __shared__ __align__(8) uint64_t sums_bar[C];
+    __shared__ float2 warp_agg[C][NT / 32];
+    __shared__ __align__(16) float red[C][NT / 32][8];
+    __shared__ int abort_s;
+
+    const int tid = threadIdx.x, lane = tid & 31;
+    const LossScalars& k = p.k;
+    const TileGeometry& g = p.geo;
+    const int n_tiles = (int)((g.nchunks - blockIdx.x + gridDim.x - 1) / gridDim.x);
+    const int rows_full = g.G * (int)g.T;
+    const long long total_rows = g.B * g.T;
+
+    if (tid >= C * NT) {
+        // ---- producer warp ----------------------------------------------------------------------------------
+        const float* const src[5] = {p.learner_mean, p.learner_logstd, p.target_mean, p.target_logstd, p.actions};
+        const long long step_rows = (long long)gridDim.x * rows_full;
+        const int n_first = n_tiles < W ? n_tiles : W;
+        // lane n asks L2 for the block's n-th tile before the stream dependency resolves (see the categorical kernel)
+        if (lane < n_first) {
+            const long long row0 = (long long)blockIdx.x * rows_full + lane * step_rows;
+            const long long left = total_rows - row0;
+            const uint32_t nrows = (uint32_t)(left < rows_full ? left : rows_full);
+            uintptr_t align = nrows * kRow;
+#pragma unroll
+            for (int q = 0; q < 5; ++q) align |= reinterpret_cast<uintptr_t>(src[q] + row0 * D);
+            if ((align & 15u) == 0) {
+#pragma unroll
+                for (int q = 0; q < 5; ++q) dev::bulk_prefetch_l2(src[q] + row0 * D, nrows * kRow);
+            }
+            if (((row0 | nrows) & 3) == 0) {
+                dev::bulk_prefetch_l2(p.worker_logp + row0, nrows * 4u);
+                dev::bulk_prefetch_l2(p.rewards + row0, nrows * 4u);
+                dev::bulk_prefetch_l2(p.discounts + row0, nrows * 4u);
+                dev::bulk_prefetch_l2(p.values + row0, nrows * 4u);
+            }
+        }
+        if (lane < S) {
+            dev::mbarrier_init_nofence(&full_bar[lane], 1);
+            dev::mbarrier_init_nofence(&empty_bar[lane], NT / 32);
+        }
+        if (lane < C) dev::mbarrier_init_nofence(&sums_bar[lane], NT / 32);
+        if (lane == 0) abort_s = 0;
+        dev::fence_mbarrier_init();
+        __syncwarp();
+
+        long long row0 = (long long)blockIdx.x * rows_full;
+        grid_dependency_wait();
+
+        int s = 0, ws = 0;
+        uint32_t ph = 0, wph = 0;
+        auto send_tile = [&](int n) {
+            const long long left = total_rows - row0;
+            const int nrows = left < rows_full ? (int)left : rows_full;
+            unsigned char* const d = smem_raw + s * kStageBytes;
+            const uint32_t bytes = (uint32_t)nrows * kRow;
+            uintptr_t align = bytes;
+#pragma unroll
+            for (int q = 0; q < 5; ++q) align |= reinterpret_cast<uintptr_t>(src[q] + row0 * D);
+            if ((align & 15u) == 0) {
+                dev::mbarrier_expect_tx(&full_bar[s], 5 * bytes);
+#pragma unroll
+                for (int q = 0; q < 5; ++q) dev::bulk_load(d + q * kSlab, src[q] + row0 * D, bytes, &full_bar[s]);
+            } else {  // ragged or unaligned slabs: element by element
+                const int nelem = nrows * D;
+#pragma unroll
+                for (int q = 0; q < 5; ++q)
+                    for (int e = 0; e < nelem; ++e) reinterpret_cast<float*>(d + q * kSlab)[e] = src[q][row0 * D + e];
+                dev::mbarrier_arrive(&full_bar[s]);
+            }
+            row0 += step_rows;
+            if (++s == S) { s = 0; ph ^= 1u; }
+            if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
+        };
+        if (lane == 0)
+            for (int n = 0; n < n_first; ++n) send_tile(n);
+        __syncthreads();  // the barriers are set up: the consumer warps may use them
+        if (lane == 0) {
+            for (int n = n_first; n < n_tiles; ++n) {
+                bool ok = true;
+                if (n >= S) ok = dev::mbarrier_wait(&empty_bar[s], ph ^ 1u, &abort_s);
+                if (ok && n >= W) ok = dev::mbarrier_wait(&full_bar[ws], wph, &abort_s);
+                if (!ok) { atomicExch(p.counter + 1, 1u); break; }
+                send_tile(n);
+            }
+        }
+        __syncwarp();
+        // the block's sums, once every group's are final: one tagged row (see the categorical kernel)
+        const unsigned int tag = dev::launch_tag(p.counter);
+        float yc[C];
+        unsigned int todo = (1u << C) - 1u;
+        for (unsigned int spin = 0; todo != 0u && spin < (1u << 24); ++spin) {
+#pragma unroll
+            for (int c = 0; c < C; ++c) {
+                if (!(todo & (1u << c))) continue;
+                bool ready = (lane == 0) && dev::mbarrier_test(&sums_bar[c], 0u);
+                ready = __shfl_sync(0xffffffffu, ready, 0);
+                if (!ready) continue;
+                float y = 0.0f;
+#pragma unroll
+                for (int w = 0; w < NT / 32; ++w) y += red[c][w][lane & 7];
+                yc[c] = y;
+                todo &= ~(1u << c);
+            }
+            if (*reinterpret_cast<volatile int*>(&abort_s)) break;
+        }
+        if (todo == 0u) {
+            float y = yc[0];
+#pragma unroll
+            for (int c = 1; c < C; ++c) y += yc[c];
+            if (lane < 8) dev::publish_tagged(p.tagged_rows + (size_t)blockIdx.x * 8 + lane, y, tag);
+        } else if (lane == 0) {
+            atomicExch(p.counter + 1, 1u);
+        }
+        return;
+    }
+
+    // ---- consumer groups ------------------------------------------------------------------
+    const int grp = tid >> 7, gtid = tid & (NT - 1), gwarp = gtid >> 5;
+    const int bar_id = grp + 1;
+    const bool want_kl = (k.kl_coef != 0.0f);
+
+    int q = 0, ts = gtid;
+    if (g.G > 1) { q = gtid / (int)g.T; ts = gtid - q * (int)g.T; }
+    const bool in_layout = gtid < rows_full;
+    const bool last_step = (ts == (int)g.T - 1);
+    long long row = ((long long)blockIdx.x + (long long)grp * gridDim.x) * rows_full + gtid;
+    long long traj = ((long long)blockIdx.x + (long long)grp * gridDim.x) * g.G + q;
+    const long long row_step = (long long)gridDim.x * C * rows_full, traj_step = (long long)gridDim.x * C * g.G;
+
+    struct StepRaw {
+        float l_worker, reward, discount, value, value_next;
+    };
+    auto load_scalars = [&](long long r, long long b, bool act) {
+        StepRaw x;
+        x.l_worker = 0.0f; x.reward = 0.0f; x.discount = 0.0f; x.value = 0.0f; x.value_next = 0.0f;
+        if (act) {
+            x.l_worker = p.worker_logp[r];
+            x.reward = p.rewards[r];
+            x.discount = p.discounts[r];
+            x.value = p.values[r];
+            x.value_next = last_step ? p.bootstrap[b] : p.values[r + 1];
+        }
+        return x;
+    };
+
+    float t_surr = 0.0f, t_val = 0.0f, t_ent = 0.0f, t_ratio = 0.0f, t_kl = 0.0f;
+    int n_clip = 0, n_trunc = 0;
+    auto hand_over_sums = [&]() {
+        const float x = dev::warp_sum4(t_surr, t_val, t_ent, t_ratio);
+        const float xk = want_kl ? dev::warp_sum(t_kl) : 0.0f;
+        if ((lane & 7) == 0) red[grp][gwarp][lane == 24 ? 6 : (lane >> 3)] = x;
+        if (lane == 0) {
+            red[grp][gwarp][3] = xk;
+            red[grp][gwarp][4] = (float)n_clip;
+            red[grp][gwarp][5] = (float)n_trunc;
+            red[grp][gwarp][7] = 0.0f;
+        }
+        __syncwarp();
+        if (lane == 0) dev::mbarrier_arrive(&sums_bar[grp]);
+    };
+    bool pending = false;
+    int pending_stage = 0;
+
+    grid_dependency_wait();
+    bool active = in_layout && row < total_rows;
+    StepRaw cur;
+    if (grp < n_tiles) cur = load_scalars(row, traj, active);
+    __syncthreads();  // the producer warp has set up the barriers
+    int s = grp % S;
+    uint32_t ph = (uint32_t)(grp / S) & 1u;
+
+    for (int n = grp; n < n_tiles; n += C) {
+        const bool active_next = (n + C < n_tiles) && in_layout && (row + row_step < total_rows);
+        const StepRaw nxt = load_scalars(row + row_step, traj + traj_step, active_next);
+        if (lane == 0 && pending) {
+            dev::bulk_store_wait_read();
+            dev::mbarrier_arrive(&empty_bar[pending_stage]);
+            pending = false;
+        }
+        if (!dev::mbarrier_wait(&full_bar[s], ph, &abort_s)) atomicExch(p.counter + 1, 1u);
+
+        unsigned char* const stage = smem_raw + s * kStageBytes;
+        float* const r_mu = reinterpret_cast<float*>(stage) + gtid * D;              // learner mean -> dmean
+        float* const r_ls = reinterpret_cast<float*>(stage + kSlab) + gtid * D;      // learner log-std -> dlogstd
+        const float* const r_mt = reinterpret_cast<const float*>(stage + 2 * kSlab) + gtid * D;
+        const float* const r_lt = reinterpret_cast<const float*>(stage + 3 * kSlab) + gtid * D;
+        const float* const r_ac = reinterpret_cast<const float*>(stage + 4 * kSlab) + gtid * D;
+        dev::StepIn st;
+        st.reward = cur.reward;
+        st.discount = cur.discount;
+        st.value = cur.value;
+        st.value_next = cur.value_next;
+        st.last_step = last_step;
+
+        // ---- row pass (every thread; rows beyond the tile hold stale bytes and are masked)
+        float ent, kl = 0.0f;
+        {
+            // log-probabilities: D-term sums of magnitude tens that end up in exponents, so they are
+            // accumulated in fp64
+            double lth = 0.0, ltg = 0.0;
+            float ls_sum = 0.0f;
+#pragma unroll
+            for (int j = 0; j < D; ++j) {
+                const float ls = r_ls[j], lt = r_lt[j], ac = r_ac[j], mu = r_mu[j], mt = r_mt[j];
+                const float inv_s = dev::exp2_fast(-ls * kLog2e), inv_st = dev::exp2_fast(-lt * kLog2e);
+                const float z1 = (ac - mu) * inv_s;
+                const float z2 = (ac - mt) * inv_st;
+                lth += (double)fmaf(-0.5f * z1, z1, -ls);
+                ltg += (double)fmaf(-0.5f * z2, z2, -lt);
+                ls_sum += ls;
+                if (want_kl) {  // KL(target || learner), per dimension
+                    const float dm = (mt - mu) * inv_s;
+                    const float sr = dev::exp2_fast((lt - ls) * kLog2e);
+                    kl += (ls - lt) + 0.5f * fmaf(sr, sr, dm * dm) - 0.5f;
+                }
+            }
+            ent = ls_sum + (float)D * (kHalfLog2Pi + 0.5f);
+            const double shift = (double)cur.l_worker + (double)D * (double)kHalfLog2Pi;
+            // everything downstream works on log-probabilities relative to the worker's
+            st.l_theta = (float)(lth - shift);
+            st.l_target = (float)(ltg - shift);
+            st.l_worker = 0.0f;
+            st.l_shift = cur.l_worker;
+        }
+        float fa, fb;
+        const bool truncated = dev::recursion_map(st, k, fa, fb);
+        if (!active) { fa = 1.0f; fb = 0.0f; }
+        const float adv = dev::suffix_affine_scan_group<NT>(fa, fb, warp_agg[grp], st.adv_next, bar_id);
+
+        float surr, ratio;
+        bool clipped;
+        const float wpg = dev::surrogate(st, k, adv, surr, ratio, clipped);
+        if (active) {
+            t_surr += surr;
+            t_val = fmaf(0.5f * adv, adv, t_val);
+            t_ent += ent;
+            t_ratio += ratio;
+            t_kl += kl;
+        }
+        n_clip += __popc(__ballot_sync(0xffffffffu, active && clipped));
+        n_trunc += __popc(__ballot_sync(0xffffffffu, active && truncated));
+        if (n + C >= n_tiles) hand_over_sums();
+
+        // ---- gradients, in place over the learner's slabs
+        {
+            const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = k.kl_coef * k.inv_M;
+#pragma unroll
+            for (int j = 0; j < D; ++j) {
+                const float ls = r_ls[j], mu = r_mu[j];
+                const float inv_s = dev::exp2_fast(-ls * kLog2e);
+                const float z = (r_ac[j] - mu) * inv_s;  // (a - mu) / sigma
+                // d log pi / d mu = z / sigma ;  d log pi / d logstd = z^2 - 1 ;  d H / d logstd = 1
+                float gm = -w1 * z;
+                float gs = -w1 * fmaf(z, z, -1.0f) - ce;
+                if (want_kl) {
+                    const float dm = (mu - r_mt[j]) * inv_s;
+                    const float sr = dev::exp2_fast((r_lt[j] - ls) * kLog2e);
+                    gm = fmaf(ck, dm, gm);
+                    gs = fmaf(ck, 1.0f - fmaf(sr, sr, dm * dm), gs);
+                }
+                r_mu[j] = gm * inv_s;
+                r_ls[j] = gs;
+            }
+            if (active) {
+                p.dvalues[row] = -k.vf_coef * k.inv_M * adv;
+                if (p.vtarget) p.vtarget[row] = st.value + adv;
+                if (p.advantage) p.advantage[row] = adv;
+            }
+        }
+        // ---- each warp sends its own 32 rows of both gradient slabs
+        {
+            const long long wrow0 = row - lane;
+            long long left = total_rows - wrow0;
+            const int cap = rows_full - (gtid - lane);
+            if (left > cap) left = cap;
+            const int wrows = left > 32 ? 32 : (left > 0 ? (int)left : 0);
+            float* const gm = p.dmean + wrow0 * D;
+            float* const gs = p.dlogstd + wrow0 * D;
+            const unsigned char* const src_m = stage + (gtid - lane) * kRow;
+            const unsigned char* const src_s = stage + kSlab + (gtid - lane) * kRow;
+            const uint32_t out_bytes = (uint32_t)wrows * kRow;
+            if (((reinterpret_cast<uintptr_t>(gm) | reinterpret_cast<uintptr_t>(gs) | out_bytes) & 15u) == 0) {
+                dev::fence_async_shared();
+                __syncwarp();
+                if (lane == 0) {
+                    if (out_bytes) {
+                        dev::bulk_store(gm, src_m, out_bytes);
+                        dev::bulk_store(gs, src_s, out_bytes);
+                    }
+                    pending = true;
+                    pending_stage = s;
+                }
+            } else {
+                __syncwarp();
+                const int nelem = wrows * D;
+                for (int i = lane; i < nelem; i += 32) {
+                    gm[i] = reinterpret_cast<const float*>(src_m)[i];
+                    gs[i] = reinterpret_cast<const float*>(src_s)[i];
+                }
+                __syncwarp();
+                if (lane == 0) dev::mbarrier_arrive(&empty_bar[s]);
+            }
+        }
+        cur = nxt;
+        active = active_next;
+        row += row_step;
+        traj += traj_step;
+        s += C;
+        while (s >= S) { s -= S; ph ^= 1u; }
+    }
+
+    if (grp >= n_tiles) hand_over_sums();
+    if (blockIdx.x == 0 && grp == (n_tiles - 1) % C) {
+        if (!dev::reduce_tagged_rows<NT>(p.tagged_rows, (int)gridDim.x, dev::launch_tag(p.counter), p.counter,
+                                         p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, (double)g.B * (double)g.T,
+                                         gtid, bar_id, &abort_s))
+            if (gtid == 0) atomicExch(p.counter + 1, 1u);
+    }
+    if (lane == 0) dev::bulk_store_wait_read();
+}
+
+// ------------------------------------------------------------------------------------------
 // Host side
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxGridBlocks = 4096;  // upper bound on blocks of a loss launch (sizes the workspace)
@@ -1673,7 +2014,7 @@ int32_t dispatch_nt(const CatParams& p, int nt, const DeviceInfo* di, cudaStream
 // only delays the first tiles), and room beyond that for the tiles being worked on and being stored.
 void ws_ring_shape(size_t stage_bytes, size_t tile_in_bytes, int groups, int max_smem, int* stages, int* in_flight) {
     int w = (int)((48 * 1024 + tile_in_bytes - 1) / tile_in_bytes);
-    if (w < 3) w = 3;
+    if (w < 2) w = 2;
     if (w > 12) w = 12;
     int s = w + groups + 3;
     if (s > kWsMaxStages) s = kWsMaxStages;
@@ -1775,7 +2116,27 @@ int32_t launch_gaussian(const GaussParams& p, const DeviceInfo* di, cudaStream_t
 }
 
 template <int D>
+int32_t launch_gaussian_ws(const GaussParams& p, const DeviceInfo* di, cudaStream_t stream) {
+    constexpr int C = 3;  // consumer groups: five slabs per tile leave room for five stages at D = 17
+    auto kernel = impact_loss_gaussian_ws_kernel<D, C>;
+    const size_t stage = (size_t)5 * kRegTileRows * D * sizeof(float);
+    int S = 0, W = 0;
+    ws_ring_shape(stage, stage, C, di->max_smem_optin, &S, &W);
+    if (S < 2) return IMPACT_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)S * stage;
+    static thread_local int configured_device = -1;
+    if (configured_device != di->device) {
+        IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
+        configured_device = di->device;
+    }
+    const long long grid = p.geo.nchunks < di->sm_count ? p.geo.nchunks : di->sm_count;
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W));
+    return IMPACT_OK;
+}
+
+template <int D>
 int32_t launch_gaussian_reg(const GaussParams& p, const DeviceInfo* di, cudaStream_t stream) {
+    if (p.geo.ntiles == 1) return launch_gaussian_ws<D>(p, di, stream);
     auto kernel = impact_loss_gaussian_reg_kernel<D>;
     const size_t smem = (size_t)5 * kRegTileRows * D * sizeof(float);
     int grid = 0;
@@ -1928,6 +2289,8 @@ extern "C" int32_t impact_loss_fwd_bwd_gaussian(
     p.partials = static_cast<float*>(workspace);
     p.counter = reinterpret_cast<unsigned int*>(static_cast<char*>(workspace) +
                                                 (size_t)kMaxGridBlocks * 8 * sizeof(float));
+    p.tagged_rows = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) +
+                                                          (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes);
     p.D = D;
     if (has_gaussian_reg_kernel(D)) {
         p.Ds = D;
