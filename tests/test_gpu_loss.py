@@ -77,6 +77,20 @@ def test_bf16_ragged(oracle, B, T, A):
     P.check_categorical(oracle, batch, h, torch.bfloat16, torch.float32)
 
 
+@pytest.mark.parametrize("B,T,D", [(41, 21, 17), (301, 50, 6), (1500, 128, 6), (900, 128, 3), (700, 100, 17),
+                                   (149, 128, 17), (33, 127, 3)])
+def test_gaussian_persistent_kernel_shapes(oracle, B, T, D):
+    """The compiled action dimensions with T <= 128: several trajectories per tile, tiles that end
+    unaligned, a ragged last tile, one tile more than there are SMs, and more tiles per block than the
+    ring has stages; with and without the KL term."""
+    batch = ii.gaussian_batch(B, T, D, seed=5000 + B + T + D, p_done=0.01)
+    P.check_gaussian(oracle, batch, LossHyper(rho_bar=1.0, c_bar=1.0, clip_eps=0.3, vf_coef=0.5, ent_coef=0.01,
+                                              kl_coef=0.0, rho_tw=1.0))
+    if B < 400:
+        P.check_gaussian(oracle, batch, LossHyper(rho_bar=1.3, c_bar=1.1, clip_eps=0.25, vf_coef=0.7, ent_coef=0.02,
+                                                  kl_coef=0.1, lam=0.97, rho_tw=2.0))
+
+
 @pytest.mark.parametrize("mode", [1, 2])
 @pytest.mark.parametrize("is_source", [0, 1])
 def test_variants(oracle, mode, is_source):
