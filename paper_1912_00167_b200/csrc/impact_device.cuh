@@ -365,6 +365,89 @@ __device__ __forceinline__ float suffix_affine_scan_group(float a, float b, floa
     return result;
 }
 
+// The scan as maps, for tiles that do not know yet what enters their last step: (ma, mb) is the
+// composition of the maps of this thread's step and all later steps of the tile, (la, lb) that of
+// all steps after this thread's warp (the identity for the last warp).  Thread 0's (ma, mb) is the
+// tile's aggregate.
+template <int NT>
+__device__ __forceinline__ void suffix_affine_maps_group(float a, float b, float2* warp_agg, float& ma, float& mb,
+                                                         float& la, float& lb, int bar_id) {
+    const int lane = threadIdx.x & 31, warp = (threadIdx.x & (NT - 1)) >> 5;
+#pragma unroll
+    for (int off = 1; off < 32; off <<= 1) {
+        const float a2 = __shfl_down_sync(0xffffffffu, a, off);
+        const float b2 = __shfl_down_sync(0xffffffffu, b, off);
+        if (lane + off < 32) {
+            b = fmaf(a, b2, b);
+            a = a * a2;
+        }
+    }
+    if (lane == 0) warp_agg[warp] = make_float2(a, b);
+    asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory");
+    la = 1.0f;
+    lb = 0.0f;
+#pragma unroll
+    for (int w = NT / 32 - 1; w > 0; --w) {
+        const float2 g = warp_agg[w];
+        if (w > warp) {  // (la, lb) <- g o (la, lb)
+            lb = fmaf(g.x, lb, g.y);
+            la = g.x * la;
+        }
+    }
+    ma = a * la;
+    mb = fmaf(a, lb, b);
+}
+
+__device__ __forceinline__ void publish_tagged(unsigned long long* slot, float value, unsigned int tag);
+
+// A tile's aggregate map, published as two (value, launch tag) pairs (see publish_tagged).
+__device__ __forceinline__ void publish_tile_aggregate(unsigned long long* slot, float a, float b, unsigned int tag) {
+    publish_tagged(slot, a, tag);
+    publish_tagged(slot + 1, b, tag);
+}
+
+// Run by one warp: `mine` points at this tile's pair of slots; the `r` tiles before it in the array are
+// the later tiles of its trajectory, the nearest first.  Reads their aggregates (a lane each, 32 at a
+// time, waiting -- bounded -- until a pair carries this launch's tag), composes them in time order and
+// returns the composition applied to 0: the value that enters this tile's last step.
+__device__ __forceinline__ float compose_later_aggregates(const unsigned long long* mine, int r, unsigned int tag,
+                                                          int* abort_flag) {
+    const int lane = threadIdx.x & 31;
+    // tile j (1 = the nearest later tile ... r = the trajectory's last) sits at mine - 2 j; the value flows
+    // from tile r down to tile 1: x <- agg_j(x).  Lanes take j = r - lane, r - lane - 32, ...: chunk by
+    // chunk from the far end, lane 0 holding the map that is applied first.
+    float x = 0.0f;
+    for (int base = r; base > 0; base -= 32) {
+        const int j = base - lane;
+        float a = 1.0f, b = 0.0f;  // identity for lanes beyond the chunk
+        if (j > 0) {
+            unsigned long long va = 0, vb = 0;
+            bool ok = false;
+            for (int tries = 0; tries < (1 << 22) && !ok; ++tries) {
+                asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(va), "=l"(vb) : "l"(mine - 2 * (long long)j) : "memory");
+                ok = ((unsigned int)(va >> 32) == tag) && ((unsigned int)(vb >> 32) == tag);
+                if (!ok && *reinterpret_cast<volatile int*>(abort_flag)) break;
+            }
+            if (!ok) *reinterpret_cast<volatile int*>(abort_flag) = 1;
+            a = __uint_as_float((unsigned int)va);
+            b = __uint_as_float((unsigned int)vb);
+        }
+        // compose over the warp: lane l ends up with map_{l+31} o ... o map_l; lane 0's is the chunk's
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const float a2 = __shfl_down_sync(0xffffffffu, a, off);
+            const float b2 = __shfl_down_sync(0xffffffffu, b, off);
+            if (lane + off < 32) {  // (a, b) <- (a2, b2) o (a, b): the higher lane's map is applied later
+                b = fmaf(a2, b, b2);
+                a = a2 * a;
+            }
+        }
+        const float ca = __shfl_sync(0xffffffffu, a, 0), cb = __shfl_sync(0xffffffffu, b, 0);
+        x = fmaf(ca, x, cb);
+    }
+    return x;
+}
+
 // Scalars of the loss that the kernels need; filled on the host.
 struct LossScalars {
     float rho_bar, c_bar, clip_lo, clip_hi;

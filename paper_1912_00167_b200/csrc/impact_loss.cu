@@ -44,6 +44,7 @@ struct CatParams {
     float* partials;
     unsigned int* counter;
     unsigned long long* tagged_rows;  // persistent kernel: rows of (value, launch tag) pairs, see publish_tagged_row
+    unsigned long long* tile_aggregates;  // persistent kernel, T > 128: two (value, launch tag) pairs per tile
     TileGeometry geo;
     LossScalars k;
     int A, As;
@@ -861,7 +862,16 @@ struct RowMath {
 
 // kPlain: the configuration of the paper's experiments -- no KL term, the clipped surrogate with the
 // default ratio and importance weights, no optional outputs -- with those branches compiled out.
-template <typename LT, typename GT, int A, int C, bool kPlain>
+//
+// kLong: trajectories longer than a tile.  Tile g of the grid is tile g % ntiles, counted from the END, of
+// trajectory g / ntiles, so the tiles of one trajectory go to neighbouring blocks and are worked on at the same
+// time.  The recursion crosses tiles through their affine aggregates: a tile composes its 128 maps into one
+// (a, b), publishes it as two (value, launch tag) pairs, reads the aggregates of the later tiles of its
+// trajectory -- all of them at once, a lane each -- and composes them, applied to 0, into the value that enters
+// its own last step.  Nothing waits on a chain of tiles: every tile waits only for aggregates, which need
+// nothing but their own tile's rows, and only of tiles with a smaller number, which no block starts later
+// than the waiting one.
+template <typename LT, typename GT, int A, int C, bool kPlain, bool kLong>
 __global__ void __launch_bounds__(C * 128 + 32, 1)
 impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W) {
     constexpr int NT = 128;
@@ -876,27 +886,51 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     __shared__ float2 warp_agg[C][NT / 32];
     __shared__ __align__(16) float red[C][NT / 32][8];
     __shared__ int abort_s;
+    __shared__ float carry_s[C];
 
     const int tid = threadIdx.x, lane = tid & 31;
     const LossScalars& k = p.k;
     const TileGeometry& g = p.geo;
-    const int n_tiles = (int)((g.nchunks - blockIdx.x + gridDim.x - 1) / gridDim.x);  // this block's tiles
-    const int rows_full = g.G * (int)g.T;                                                // rows of a full tile
+    const long long total_tiles = kLong ? g.nchunks * g.ntiles : g.nchunks;
+    const int n_tiles = (int)((total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);  // this block's tiles
+    const int rows_full = kLong ? NT : g.G * (int)g.T;                                   // rows of a full tile
     const long long total_rows = g.B * g.T;
+    // where the block's n-th tile sits: first row, rows, and (kLong) trajectory and tile number from its end
+    struct Place {
+        long long row0, traj;
+        int nrows, r;
+    };
+    auto place_of = [&](int n) {
+        Place pl;
+        const long long gt_ = (long long)blockIdx.x + (long long)n * gridDim.x;
+        if (kLong) {
+            pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
+            pl.r = (int)(gt_ - pl.traj * g.ntiles);
+            const long long t0 = (long long)(g.ntiles - 1 - pl.r) * NT;
+            const long long left = g.T - t0;
+            pl.nrows = left < NT ? (int)left : NT;
+            pl.row0 = pl.traj * g.T + t0;
+        } else {
+            pl.row0 = gt_ * rows_full;
+            pl.traj = gt_ * g.G;
+            const long long left = total_rows - pl.row0;
+            pl.nrows = left < rows_full ? (int)left : rows_full;
+            pl.r = 0;
+        }
+        return pl;
+    };
 
     if (tid >= C * NT) {
         // ---- producer warp ----------------------------------------------------------------------------------
-        const long long step_elems = (long long)gridDim.x * rows_full * A;
-        const long long step_rows = (long long)gridDim.x * rows_full;
         const int n_first = n_tiles < W ? n_tiles : W;
         // First of all, while the kernel before this one on the stream is still finishing, lane n asks L2 for
         // the block's n-th tile (logits and per-step scalars): a prefetch changes nothing that a program can
         // observe (L2 is where the device's writes meet, so later writes to these addresses are not lost), but
         // the pages are mapped and the bytes on their way when the dependency resolves.
         if (lane < n_first) {
-            const long long row0 = (long long)blockIdx.x * rows_full + lane * step_rows;
-            const long long left = total_rows - row0;
-            const uint32_t nrows = (uint32_t)(left < rows_full ? left : rows_full);
+            const Place pc = place_of(lane);
+            const long long row0 = pc.row0;
+            const uint32_t nrows = (uint32_t)pc.nrows;
             const LT* const pl = static_cast<const LT*>(p.learner_logits) + row0 * A;
             const LT* const pt = static_cast<const LT*>(p.target_logits) + row0 * A;
             if (((reinterpret_cast<uintptr_t>(pl) | reinterpret_cast<uintptr_t>(pt) | (nrows * kInRow)) & 15u) == 0) {
@@ -922,15 +956,15 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         __syncwarp();
 
         // lane 0 streams the block's tiles into the ring
-        const LT* gl = static_cast<const LT*>(p.learner_logits) + (long long)blockIdx.x * rows_full * A;
-        const LT* gt = static_cast<const LT*>(p.target_logits) + (long long)blockIdx.x * rows_full * A;
-        long long rows_left = total_rows - (long long)blockIdx.x * rows_full;
         grid_dependency_wait();
 
         int s = 0, ws = 0;         // stage of tile n, stage of tile n - W
         uint32_t ph = 0, wph = 0;  // their phase parities
         auto send_tile = [&](int n) {
-            const int nrows = rows_left < rows_full ? (int)rows_left : rows_full;
+            const Place pc = place_of(n);
+            const int nrows = pc.nrows;
+            const LT* const gl = static_cast<const LT*>(p.learner_logits) + pc.row0 * A;
+            const LT* const gt = static_cast<const LT*>(p.target_logits) + pc.row0 * A;
             unsigned char* const d0 = smem_raw + s * kStageBytes;
             unsigned char* const d1 = d0 + NT * kInRow;
             const uint32_t bytes = (uint32_t)nrows * kInRow;
@@ -946,9 +980,6 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
                 }
                 dev::mbarrier_arrive(&full_bar[s]);
             }
-            gl += step_elems;
-            gt += step_elems;
-            rows_left -= step_rows;
             if (++s == S) { s = 0; ph ^= 1u; }
             if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
         };
@@ -1005,31 +1036,42 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     const int bar_id = grp + 1;
     const bool want_kl = !kPlain && (k.kl_coef != 0.0f);
 
-    // the thread's place in a tile never changes: step ts of trajectory q of the tile
+    // (short trajectories) the thread's place in a tile never changes: step ts of trajectory q of the tile
     int q = 0, ts = gtid;
-    if (g.G > 1) { q = gtid / (int)g.T; ts = gtid - q * (int)g.T; }
-    const bool in_layout = gtid < rows_full;
-    const bool last_step = (ts == (int)g.T - 1);
-    // row and trajectory of this thread in the group's current tile, and their advance per tile
-    long long row = ((long long)blockIdx.x + (long long)grp * gridDim.x) * rows_full + gtid;
-    long long traj = ((long long)blockIdx.x + (long long)grp * gridDim.x) * g.G + q;
-    const long long row_step = (long long)gridDim.x * C * rows_full, traj_step = (long long)gridDim.x * C * g.G;
+    if (!kLong && g.G > 1) { q = gtid / (int)g.T; ts = gtid - q * (int)g.T; }
+    // this thread's row, trajectory, whether it has a row at all and whether that row ends its trajectory,
+    // in the block's n-th tile
+    struct Mine {
+        long long row, traj;
+        bool active, last_step;
+        Place pc;
+    };
+    auto mine_in = [&](int n) {
+        Mine m;
+        m.pc = place_of(n < n_tiles ? n : 0);
+        m.row = m.pc.row0 + gtid;
+        m.traj = m.pc.traj + q;
+        m.active = n < n_tiles && gtid < m.pc.nrows;
+        m.last_step = kLong ? (m.pc.r == 0 && gtid == m.pc.nrows - 1) : (ts == (int)g.T - 1);
+        return m;
+    };
 
     struct StepRaw {
         int a;
         float l_worker, reward, discount, value, value_next;
     };
-    auto load_scalars = [&](long long r, long long b, bool act) {
+    auto load_scalars = [&](const Mine& m) {
         StepRaw x;
         x.a = 0; x.l_worker = 0.0f; x.reward = 0.0f; x.discount = 0.0f; x.value = 0.0f; x.value_next = 0.0f;
-        if (act) {
+        if (m.active) {
+            const long long r = m.row;
             const int a = p.actions[r];
             x.a = min(max(a, 0), A - 1);
             x.l_worker = p.worker_logp[r];
             x.reward = p.rewards[r];
             x.discount = p.discounts[r];
             x.value = p.values[r];
-            x.value_next = last_step ? p.bootstrap[b] : p.values[r + 1];
+            x.value_next = m.last_step ? p.bootstrap[m.traj] : p.values[r + 1];
         }
         return x;
     };
@@ -1055,17 +1097,18 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     int pending_stage = 0;
 
     grid_dependency_wait();
-    bool active = in_layout && row < total_rows;
-    StepRaw cur;
-    if (grp < n_tiles) cur = load_scalars(row, traj, active);
+    Mine me = mine_in(grp);
+    StepRaw cur = load_scalars(me);
     __syncthreads();  // the producer warp has set up the barriers
     int s = grp % S;
     uint32_t ph = (uint32_t)(grp / S) & 1u;
 
     for (int n = grp; n < n_tiles; n += C) {
         // the next tile's scalars travel while this tile is worked on
-        const bool active_next = (n + C < n_tiles) && in_layout && (row + row_step < total_rows);
-        const StepRaw nxt = load_scalars(row + row_step, traj + traj_step, active_next);
+        const Mine me_next = mine_in(n + C);
+        const StepRaw nxt = load_scalars(me_next);
+        const bool active = me.active;
+        const long long row = me.row;
         if (lane == 0 && pending) {  // this warp's previous rows have left shared memory: hand the stage back
             dev::bulk_store_wait_read();
             dev::mbarrier_arrive(&empty_bar[pending_stage]);
@@ -1085,7 +1128,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         st.discount = cur.discount;
         st.value = cur.value;
         st.value_next = cur.value_next;
-        st.last_step = last_step;
+        st.last_step = me.last_step;
 
         // ---- row passes (every thread; rows beyond the tile hold stale bytes and are masked)
         float2 e[NP];
@@ -1111,7 +1154,30 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         if (kPlain) truncated = dev::recursion_map_plain(st, k, fa, fb);
         else truncated = dev::recursion_map(st, k, fa, fb);
         if (!active) { fa = 1.0f; fb = 0.0f; }
-        const float adv = dev::suffix_affine_scan_group<NT>(fa, fb, warp_agg[grp], st.adv_next, bar_id);
+        float adv;
+        if (!kLong) {
+            adv = dev::suffix_affine_scan_group<NT>(fa, fb, warp_agg[grp], st.adv_next, bar_id);
+        } else {
+            // maps instead of values: (ma, mb) takes the value that enters the tile's last step to A of this
+            // step, (la, lb) to A of the step after this warp's last
+            float ma, mb, la, lb;
+            dev::suffix_affine_maps_group<NT>(fa, fb, warp_agg[grp], ma, mb, la, lb, bar_id);
+            const long long gtile = (long long)blockIdx.x + (long long)n * gridDim.x;
+            if (gtid == 0) dev::publish_tile_aggregate(p.tile_aggregates + 2 * gtile, ma, mb, dev::launch_tag(p.counter));
+            float carry = 0.0f;
+            if (me.pc.r > 0) {  // uniform over the group
+                if (gwarp == 0) {
+                    const float c = dev::compose_later_aggregates(p.tile_aggregates + 2 * gtile, me.pc.r,
+                                                                  dev::launch_tag(p.counter), &abort_s);
+                    if (lane == 0) carry_s[grp] = c;
+                }
+                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+                carry = carry_s[grp];
+            }
+            adv = fmaf(ma, carry, mb);
+            const float below = __shfl_down_sync(0xffffffffu, adv, 1);
+            st.adv_next = (lane == 31) ? fmaf(la, carry, lb) : below;
+        }
 
         float surr, ratio;
         bool clipped;
@@ -1167,10 +1233,8 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         // ---- each warp sends its own 32 rows: no barrier across the group
         {
             const long long wrow0 = row - lane;  // first row of this warp
-            long long left = total_rows - wrow0;
-            const int cap = rows_full - (gtid - lane);
-            if (left > cap) left = cap;
-            const int wrows = left > 32 ? 32 : (left > 0 ? (int)left : 0);
+            const int left = me.pc.nrows - (gtid - lane);
+            const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
             GT* const gd = static_cast<GT*>(p.dlogits) + wrow0 * A;
             const unsigned char* const src = so + (gtid - lane) * kOutRow;
             const uint32_t out_bytes = (uint32_t)wrows * kOutRow;
@@ -1191,9 +1255,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             }
         }
         cur = nxt;
-        active = active_next;
-        row += row_step;
-        traj += traj_step;
+        me = me_next;
         s += C;
         while (s >= S) { s -= S; ph ^= 1u; }
     }
@@ -1897,7 +1959,15 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
 // ------------------------------------------------------------------------------------------
 constexpr int kMaxGridBlocks = 4096;  // upper bound on blocks of a loss launch (sizes the workspace)
 constexpr size_t kCounterBytes = 256; // words after the partials: [0] completion counter, [1] error flag, [2] launch number
+// Long trajectories (T > 128 steps): two (value, tag) pairs per 128-step tile, after everything else.
+size_t tile_aggregate_bytes(int64_t B, int64_t T) {
+    if (T <= kRegTileRows) return 0;
+    return (size_t)B * (size_t)((T + kRegTileRows - 1) / kRegTileRows) * 2 * sizeof(unsigned long long);
+}
 constexpr int kMaxTaggedRows = 1024;  // rows of eight (value, tag) pairs after the counter words: one per block of the persistent kernel
+
+constexpr size_t kWorkspaceFixedBytes = (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes +
+                                        (size_t)kMaxTaggedRows * 8 * sizeof(unsigned long long);
 
 int pad_odd(int w) { return (w & 1) ? w : w + 1; }
 
@@ -2025,10 +2095,10 @@ void ws_ring_shape(size_t stage_bytes, size_t tile_in_bytes, int groups, int max
     *in_flight = w;
 }
 
-template <typename LT, typename GT, int A, bool kPlain>
+template <typename LT, typename GT, int A, bool kPlain, bool kLong>
 int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
     constexpr int C = kWsGroups;
-    auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain>;
+    auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong>;
     const size_t stage = reg_kernel_stage_bytes<LT, GT, A>();
     int S = 0, W = 0;
     ws_ring_shape(stage, 2 * (size_t)kRegTileRows * A * sizeof(LT), C, di->max_smem_optin, &S, &W);
@@ -2039,22 +2109,28 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
         IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured_device = di->device;
     }
-    const long long grid = p.geo.nchunks < di->sm_count ? p.geo.nchunks : di->sm_count;
+    const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
+    const long long grid = tiles < di->sm_count ? tiles : di->sm_count;
     IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W));
     return IMPACT_OK;
 }
 
-// The persistent kernel serves every batch whose trajectories fit a tile (T <= 128); longer
-// trajectories go to the kernel that carries the recursion from tile to tile.
+// The persistent kernel serves every batch: trajectories that fit a tile (T <= 128) and, where the caller's
+// scratch has room for the tiles' aggregates, longer ones; the kernel that sweeps a long trajectory tile by
+// tile inside one block remains for scratch without that room.
 template <typename LT, typename GT, int A>
 int32_t launch_categorical_reg(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
     if (p.geo.ntiles == 1) {
         const bool plain = p.k.kl_coef == 0.0f && p.k.objective == IMPACT_OBJECTIVE_CLIPPED_SURROGATE &&
                            p.k.is_source == IMPACT_IS_TARGET_OVER_WORKER && p.k.ratio_mode == IMPACT_RATIO_R3 &&
                            !p.vtarget && !p.advantage;
-        if (plain) return launch_categorical_ws<LT, GT, A, true>(p, di, stream);
-        return launch_categorical_ws<LT, GT, A, false>(p, di, stream);
+        if (plain) return launch_categorical_ws<LT, GT, A, true, false>(p, di, stream);
+        return launch_categorical_ws<LT, GT, A, false, false>(p, di, stream);
     }
+    // Split across blocks while there are too few trajectories to give every consumer group of the device one of
+    // its own; from there on the sweep inside a block keeps the device busy without any exchange between tiles.
+    if (p.tile_aggregates && p.geo.B < (long long)kWsGroups * di->sm_count)
+        return launch_categorical_ws<LT, GT, A, false, true>(p, di, stream);
     auto kernel = impact_loss_categorical_reg_kernel<LT, GT, A>;
     const size_t smem = reg_kernel_smem<LT, GT, A>();
     int grid = 0;
@@ -2156,7 +2232,7 @@ using namespace impact;
 
 extern "C" size_t impact_loss_workspace_bytes(int64_t B, int64_t T) {
     if (B <= 0 || T <= 0) return 0;
-    return (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes + (size_t)kMaxTaggedRows * 8 * sizeof(unsigned long long);
+    return kWorkspaceFixedBytes + tile_aggregate_bytes(B, T);
 }
 
 extern "C" int32_t impact_loss_workspace_init(void* workspace, size_t workspace_bytes, void* stream) {
@@ -2226,6 +2302,9 @@ extern "C" int32_t impact_loss_fwd_bwd(
                                                 (size_t)kMaxGridBlocks * 8 * sizeof(float));
     p.tagged_rows = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) +
                                                           (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes);
+    p.tile_aggregates = T > kRegTileRows
+                            ? reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWorkspaceFixedBytes)
+                            : nullptr;
     p.A = A;
     return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
                            di, static_cast<cudaStream_t>(stream));
@@ -2402,6 +2481,7 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     p.partials = reinterpret_cast<float*>(scratch);
     p.counter = reinterpret_cast<unsigned int*>(counter);
     p.tagged_rows = reinterpret_cast<unsigned long long*>(counter + kCounterBytes);
+    p.tile_aggregates = nullptr;  // long trajectories are swept tile by tile inside a block
     // the same kernels, chosen the same way, as impact_loss_fwd_bwd
     return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
                            di, s);

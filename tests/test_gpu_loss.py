@@ -77,6 +77,22 @@ def test_bf16_ragged(oracle, B, T, A):
     P.check_categorical(oracle, batch, h, torch.bfloat16, torch.float32)
 
 
+@pytest.mark.parametrize("B,T,A,dtype", [(2, 4500, 6, torch.float32), (5, 1300, 9, torch.float32),
+                                         (1, 130, 18, torch.float32), (40, 257, 18, torch.bfloat16),
+                                         (700, 256, 18, torch.float32), (3, 640, 4, torch.float32)])
+def test_long_trajectories_split_across_blocks(oracle, B, T, A, dtype):
+    """T > 128: the tiles of a trajectory are worked on by different blocks at once and linked through their
+    published aggregates (more than 32 tiles per trajectory, a partial first tile, rows that end unaligned);
+    from a few hundred trajectories on a block sweeps a trajectory by itself."""
+    batch = ii.categorical_batch(B, T, A, seed=900 + B + T + A, p_done=0.003)
+    h = LossHyper(rho_bar=1.2, c_bar=1.0, clip_eps=0.3, vf_coef=0.5, ent_coef=0.01, kl_coef=0.05, lam=0.99, rho_tw=2.0)
+    if dtype == torch.bfloat16:
+        P.check_categorical(oracle, batch, h, torch.bfloat16, torch.float32)
+    else:
+        P.check_categorical(oracle, batch, h)
+    P.check_categorical(oracle, batch, dataclasses.replace(h, objective=1, kl_coef=0.0), dtype, torch.float32)
+
+
 @pytest.mark.parametrize("B,T,D", [(41, 21, 17), (301, 50, 6), (1500, 128, 6), (900, 128, 3), (700, 100, 17),
                                    (149, 128, 17), (33, 127, 3)])
 def test_gaussian_persistent_kernel_shapes(oracle, B, T, D):
