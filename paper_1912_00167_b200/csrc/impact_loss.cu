@@ -70,6 +70,7 @@ struct GaussParams {
     float* partials;
     unsigned int* counter;
     unsigned long long* tagged_rows;
+    unsigned long long* tile_aggregates;
     TileGeometry geo;
     LossScalars k;
     int D, Ds;
@@ -1621,8 +1622,9 @@ __global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kern
 // log-std, target mean / log-std, actions) and two output slabs (dmean, dlogstd, written over the
 // learner's): a producer warp streams tiles through the ring, C consumer groups take them as they
 // land, every warp stores its own rows, the block's sums leave as one tagged row.  Row arithmetic is
-// that of impact_loss_gaussian_reg_kernel (log-probabilities accumulated in fp64).
-template <int D, int C>
+// that of impact_loss_gaussian_reg_kernel (log-probabilities accumulated in fp64).  kLong as in the
+// categorical kernel: tiles of a long trajectory on neighbouring blocks, linked through their aggregates.
+template <int D, int C, bool kLong>
 __global__ void __launch_bounds__(C * 128 + 32, 1)
 impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int S, const int W) {
     constexpr int NT = 128;
@@ -1637,24 +1639,48 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     __shared__ float2 warp_agg[C][NT / 32];
     __shared__ __align__(16) float red[C][NT / 32][8];
     __shared__ int abort_s;
+    __shared__ float carry_s[C];
 
     const int tid = threadIdx.x, lane = tid & 31;
     const LossScalars& k = p.k;
     const TileGeometry& g = p.geo;
-    const int n_tiles = (int)((g.nchunks - blockIdx.x + gridDim.x - 1) / gridDim.x);
-    const int rows_full = g.G * (int)g.T;
+    const long long total_tiles = kLong ? g.nchunks * g.ntiles : g.nchunks;
+    const int n_tiles = (int)((total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+    const int rows_full = kLong ? NT : g.G * (int)g.T;
     const long long total_rows = g.B * g.T;
+    struct Place {
+        long long row0, traj;
+        int nrows, r;
+    };
+    auto place_of = [&](int n) {
+        Place pl;
+        const long long gt_ = (long long)blockIdx.x + (long long)n * gridDim.x;
+        if (kLong) {
+            pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
+            pl.r = (int)(gt_ - pl.traj * g.ntiles);
+            const long long t0 = (long long)(g.ntiles - 1 - pl.r) * NT;
+            const long long left = g.T - t0;
+            pl.nrows = left < NT ? (int)left : NT;
+            pl.row0 = pl.traj * g.T + t0;
+        } else {
+            pl.row0 = gt_ * rows_full;
+            pl.traj = gt_ * g.G;
+            const long long left = total_rows - pl.row0;
+            pl.nrows = left < rows_full ? (int)left : rows_full;
+            pl.r = 0;
+        }
+        return pl;
+    };
 
     if (tid >= C * NT) {
         // ---- producer warp ----------------------------------------------------------------------------------
         const float* const src[5] = {p.learner_mean, p.learner_logstd, p.target_mean, p.target_logstd, p.actions};
-        const long long step_rows = (long long)gridDim.x * rows_full;
         const int n_first = n_tiles < W ? n_tiles : W;
         // lane n asks L2 for the block's n-th tile before the stream dependency resolves (see the categorical kernel)
         if (lane < n_first) {
-            const long long row0 = (long long)blockIdx.x * rows_full + lane * step_rows;
-            const long long left = total_rows - row0;
-            const uint32_t nrows = (uint32_t)(left < rows_full ? left : rows_full);
+            const Place pc = place_of(lane);
+            const long long row0 = pc.row0;
+            const uint32_t nrows = (uint32_t)pc.nrows;
             uintptr_t align = nrows * kRow;
 #pragma unroll
             for (int q = 0; q < 5; ++q) align |= reinterpret_cast<uintptr_t>(src[q] + row0 * D);
@@ -1678,14 +1704,14 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
         dev::fence_mbarrier_init();
         __syncwarp();
 
-        long long row0 = (long long)blockIdx.x * rows_full;
         grid_dependency_wait();
 
         int s = 0, ws = 0;
         uint32_t ph = 0, wph = 0;
         auto send_tile = [&](int n) {
-            const long long left = total_rows - row0;
-            const int nrows = left < rows_full ? (int)left : rows_full;
+            const Place pc = place_of(n);
+            const long long row0 = pc.row0;
+            const int nrows = pc.nrows;
             unsigned char* const d = smem_raw + s * kStageBytes;
             const uint32_t bytes = (uint32_t)nrows * kRow;
             uintptr_t align = bytes;
@@ -1702,7 +1728,6 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
                     for (int e = 0; e < nelem; ++e) reinterpret_cast<float*>(d + q * kSlab)[e] = src[q][row0 * D + e];
                 dev::mbarrier_arrive(&full_bar[s]);
             }
-            row0 += step_rows;
             if (++s == S) { s = 0; ph ^= 1u; }
             if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
         };
@@ -1755,25 +1780,35 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     const bool want_kl = (k.kl_coef != 0.0f);
 
     int q = 0, ts = gtid;
-    if (g.G > 1) { q = gtid / (int)g.T; ts = gtid - q * (int)g.T; }
-    const bool in_layout = gtid < rows_full;
-    const bool last_step = (ts == (int)g.T - 1);
-    long long row = ((long long)blockIdx.x + (long long)grp * gridDim.x) * rows_full + gtid;
-    long long traj = ((long long)blockIdx.x + (long long)grp * gridDim.x) * g.G + q;
-    const long long row_step = (long long)gridDim.x * C * rows_full, traj_step = (long long)gridDim.x * C * g.G;
+    if (!kLong && g.G > 1) { q = gtid / (int)g.T; ts = gtid - q * (int)g.T; }
+    struct Mine {
+        long long row, traj;
+        bool active, last_step;
+        Place pc;
+    };
+    auto mine_in = [&](int n) {
+        Mine m;
+        m.pc = place_of(n < n_tiles ? n : 0);
+        m.row = m.pc.row0 + gtid;
+        m.traj = m.pc.traj + q;
+        m.active = n < n_tiles && gtid < m.pc.nrows;
+        m.last_step = kLong ? (m.pc.r == 0 && gtid == m.pc.nrows - 1) : (ts == (int)g.T - 1);
+        return m;
+    };
 
     struct StepRaw {
         float l_worker, reward, discount, value, value_next;
     };
-    auto load_scalars = [&](long long r, long long b, bool act) {
+    auto load_scalars = [&](const Mine& m) {
         StepRaw x;
         x.l_worker = 0.0f; x.reward = 0.0f; x.discount = 0.0f; x.value = 0.0f; x.value_next = 0.0f;
-        if (act) {
+        if (m.active) {
+            const long long r = m.row;
             x.l_worker = p.worker_logp[r];
             x.reward = p.rewards[r];
             x.discount = p.discounts[r];
             x.value = p.values[r];
-            x.value_next = last_step ? p.bootstrap[b] : p.values[r + 1];
+            x.value_next = m.last_step ? p.bootstrap[m.traj] : p.values[r + 1];
         }
         return x;
     };
@@ -1797,16 +1832,17 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     int pending_stage = 0;
 
     grid_dependency_wait();
-    bool active = in_layout && row < total_rows;
-    StepRaw cur;
-    if (grp < n_tiles) cur = load_scalars(row, traj, active);
+    Mine me = mine_in(grp);
+    StepRaw cur = load_scalars(me);
     __syncthreads();  // the producer warp has set up the barriers
     int s = grp % S;
     uint32_t ph = (uint32_t)(grp / S) & 1u;
 
     for (int n = grp; n < n_tiles; n += C) {
-        const bool active_next = (n + C < n_tiles) && in_layout && (row + row_step < total_rows);
-        const StepRaw nxt = load_scalars(row + row_step, traj + traj_step, active_next);
+        const Mine me_next = mine_in(n + C);
+        const StepRaw nxt = load_scalars(me_next);
+        const bool active = me.active;
+        const long long row = me.row;
         if (lane == 0 && pending) {
             dev::bulk_store_wait_read();
             dev::mbarrier_arrive(&empty_bar[pending_stage]);
@@ -1825,7 +1861,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
         st.discount = cur.discount;
         st.value = cur.value;
         st.value_next = cur.value_next;
-        st.last_step = last_step;
+        st.last_step = me.last_step;
 
         // ---- row pass (every thread; rows beyond the tile hold stale bytes and are masked)
         float ent, kl = 0.0f;
@@ -1860,7 +1896,28 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
         float fa, fb;
         const bool truncated = dev::recursion_map(st, k, fa, fb);
         if (!active) { fa = 1.0f; fb = 0.0f; }
-        const float adv = dev::suffix_affine_scan_group<NT>(fa, fb, warp_agg[grp], st.adv_next, bar_id);
+        float adv;
+        if (!kLong) {
+            adv = dev::suffix_affine_scan_group<NT>(fa, fb, warp_agg[grp], st.adv_next, bar_id);
+        } else {
+            float ma, mb, la, lb;
+            dev::suffix_affine_maps_group<NT>(fa, fb, warp_agg[grp], ma, mb, la, lb, bar_id);
+            const long long gtile = (long long)blockIdx.x + (long long)n * gridDim.x;
+            if (gtid == 0) dev::publish_tile_aggregate(p.tile_aggregates + 2 * gtile, ma, mb, dev::launch_tag(p.counter));
+            float carry = 0.0f;
+            if (me.pc.r > 0) {  // uniform over the group
+                if (gwarp == 0) {
+                    const float c = dev::compose_later_aggregates(p.tile_aggregates + 2 * gtile, me.pc.r,
+                                                                  dev::launch_tag(p.counter), &abort_s);
+                    if (lane == 0) carry_s[grp] = c;
+                }
+                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+                carry = carry_s[grp];
+            }
+            adv = fmaf(ma, carry, mb);
+            const float below = __shfl_down_sync(0xffffffffu, adv, 1);
+            st.adv_next = (lane == 31) ? fmaf(la, carry, lb) : below;
+        }
 
         float surr, ratio;
         bool clipped;
@@ -1905,10 +1962,8 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
         // ---- each warp sends its own 32 rows of both gradient slabs
         {
             const long long wrow0 = row - lane;
-            long long left = total_rows - wrow0;
-            const int cap = rows_full - (gtid - lane);
-            if (left > cap) left = cap;
-            const int wrows = left > 32 ? 32 : (left > 0 ? (int)left : 0);
+            const int left = me.pc.nrows - (gtid - lane);
+            const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
             float* const gm = p.dmean + wrow0 * D;
             float* const gs = p.dlogstd + wrow0 * D;
             const unsigned char* const src_m = stage + (gtid - lane) * kRow;
@@ -1937,9 +1992,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
             }
         }
         cur = nxt;
-        active = active_next;
-        row += row_step;
-        traj += traj_step;
+        me = me_next;
         s += C;
         while (s >= S) { s -= S; ph ^= 1u; }
     }
@@ -2191,10 +2244,12 @@ int32_t launch_gaussian(const GaussParams& p, const DeviceInfo* di, cudaStream_t
     return IMPACT_OK;
 }
 
-template <int D>
+constexpr int kWsGroupsGaussian = 3;  // consumer groups: five slabs per tile leave room for five stages at D = 17
+
+template <int D, bool kLong>
 int32_t launch_gaussian_ws(const GaussParams& p, const DeviceInfo* di, cudaStream_t stream) {
-    constexpr int C = 3;  // consumer groups: five slabs per tile leave room for five stages at D = 17
-    auto kernel = impact_loss_gaussian_ws_kernel<D, C>;
+    constexpr int C = kWsGroupsGaussian;
+    auto kernel = impact_loss_gaussian_ws_kernel<D, C, kLong>;
     const size_t stage = (size_t)5 * kRegTileRows * D * sizeof(float);
     int S = 0, W = 0;
     ws_ring_shape(stage, stage, C, di->max_smem_optin, &S, &W);
@@ -2205,14 +2260,17 @@ int32_t launch_gaussian_ws(const GaussParams& p, const DeviceInfo* di, cudaStrea
         IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
         configured_device = di->device;
     }
-    const long long grid = p.geo.nchunks < di->sm_count ? p.geo.nchunks : di->sm_count;
+    const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
+    const long long grid = tiles < di->sm_count ? tiles : di->sm_count;
     IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W));
     return IMPACT_OK;
 }
 
 template <int D>
 int32_t launch_gaussian_reg(const GaussParams& p, const DeviceInfo* di, cudaStream_t stream) {
-    if (p.geo.ntiles == 1) return launch_gaussian_ws<D>(p, di, stream);
+    if (p.geo.ntiles == 1) return launch_gaussian_ws<D, false>(p, di, stream);
+    if (p.tile_aggregates && p.geo.B < (long long)kWsGroupsGaussian * di->sm_count)
+        return launch_gaussian_ws<D, true>(p, di, stream);
     auto kernel = impact_loss_gaussian_reg_kernel<D>;
     const size_t smem = (size_t)5 * kRegTileRows * D * sizeof(float);
     int grid = 0;
@@ -2370,6 +2428,9 @@ extern "C" int32_t impact_loss_fwd_bwd_gaussian(
                                                 (size_t)kMaxGridBlocks * 8 * sizeof(float));
     p.tagged_rows = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) +
                                                           (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes);
+    p.tile_aggregates = T > kRegTileRows
+                            ? reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWorkspaceFixedBytes)
+                            : nullptr;
     p.D = D;
     if (has_gaussian_reg_kernel(D)) {
         p.Ds = D;

@@ -93,6 +93,16 @@ def test_long_trajectories_split_across_blocks(oracle, B, T, A, dtype):
     P.check_categorical(oracle, batch, dataclasses.replace(h, objective=1, kl_coef=0.0), dtype, torch.float32)
 
 
+@pytest.mark.parametrize("B,T,D", [(2, 4500, 3), (5, 1024, 17), (1, 130, 6), (30, 300, 17), (500, 256, 6)])
+def test_gaussian_long_trajectories(oracle, B, T, D):
+    """T > 128 for the compiled action dimensions: tiles of a trajectory on different blocks, linked through their
+    aggregates (few trajectories), or swept inside one block (many)."""
+    batch = ii.gaussian_batch(B, T, D, seed=7000 + B + T + D, p_done=0.003)
+    P.check_gaussian(oracle, batch, LossHyper(rho_bar=1.2, c_bar=1.0, clip_eps=0.3, vf_coef=0.5, ent_coef=0.01,
+                                              kl_coef=0.05, lam=0.99, rho_tw=2.0))
+    P.check_gaussian(oracle, batch, LossHyper(objective=1))
+
+
 @pytest.mark.parametrize("B,T,D", [(41, 21, 17), (301, 50, 6), (1500, 128, 6), (900, 128, 3), (700, 100, 17),
                                    (149, 128, 17), (33, 127, 3)])
 def test_gaussian_persistent_kernel_shapes(oracle, B, T, D):
