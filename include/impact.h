@@ -29,7 +29,7 @@
 extern "C" {
 #endif
 
-#define IMPACT_VERSION 100 /* major*10000 + minor*100 + patch */
+#define IMPACT_VERSION 200 /* major*10000 + minor*100 + patch */
 
 /* ---- status codes -------------------------------------------------------------------- */
 #define IMPACT_OK 0
@@ -101,6 +101,11 @@ typedef struct impact_coefficients {
     int32_t ratio_mode;    /* IMPACT_RATIO_* */
     int32_t dlogits_dtype; /* IMPACT_DTYPE_*: storage type of the policy-gradient outputs */
     int32_t objective;     /* IMPACT_OBJECTIVE_* */
+    int64_t global_steps;  /* the M of the 1/M normaliser (Algorithm 1); 0 = B*T, this call's own steps.  A caller
+                              that splits one train batch over several calls or GPUs (trajectories are
+                              independent) passes the steps of the WHOLE batch here in every call: gradients then
+                              carry the whole batch's 1/M, and the calls' loss_terms ADD UP to the whole batch's
+                              (they are sums over this call's steps divided by M).  Must be 0 or >= B*T. */
 } impact_coefficients;
 
 /* ---- housekeeping --------------------------------------------------------------------- */

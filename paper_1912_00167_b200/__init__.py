@@ -12,3 +12,4 @@ from .binding import (  # noqa: F401
     prepare_loss_fwd_bwd_gaussian,
 )
 from . import binding  # noqa: F401
+from .sharded import impact_loss_fwd_bwd_sharded, reduce_loss_terms, shard_bounds  # noqa: F401

@@ -47,7 +47,7 @@ class impact_coefficients(ctypes.Structure):
     _fields_ = [("vf_coef", ctypes.c_float), ("ent_coef", ctypes.c_float), ("kl_coef", ctypes.c_float),
                 ("lambda_", ctypes.c_float), ("rho_tw", ctypes.c_float), ("is_source", ctypes.c_int32),
                 ("ratio_mode", ctypes.c_int32), ("dlogits_dtype", ctypes.c_int32),
-                ("objective", ctypes.c_int32)]
+                ("objective", ctypes.c_int32), ("global_steps", ctypes.c_int64)]
 
 
 class impact_loss_call(ctypes.Structure):
@@ -175,10 +175,12 @@ class Coefficients:
     is_source: int = IS_TARGET_OVER_WORKER
     ratio_mode: int = RATIO_R3
     objective: int = OBJECTIVE_CLIPPED_SURROGATE
+    global_steps: int = 0  # steps of the whole train batch when it is split over several calls; 0 = this call's B*T
 
     def c_struct(self, dlogits_dtype: int) -> impact_coefficients:
         return impact_coefficients(self.vf_coef, self.ent_coef, self.kl_coef, self.lam, self.rho_tw,
-                                   int(self.is_source), int(self.ratio_mode), int(dlogits_dtype), int(self.objective))
+                                   int(self.is_source), int(self.ratio_mode), int(dlogits_dtype), int(self.objective),
+                                   int(self.global_steps))
 
 
 def impact_loss_workspace_bytes(B: int, T: int) -> int:

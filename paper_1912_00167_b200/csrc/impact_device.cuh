@@ -454,6 +454,7 @@ struct LossScalars {
     float vf_coef, ent_coef, kl_coef, lambda_, log_rho_tw;
     float inv_M;
     int is_source, ratio_mode, objective;
+    double steps_total;  // M: the steps the means are taken over (this call's, or the whole batch's when it is split)
 };
 
 // Per-step quantities once the three log-probabilities are known.

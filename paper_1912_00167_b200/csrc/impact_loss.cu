@@ -326,7 +326,7 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
         }
     }
     if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef,
-                                                   (double)g.B * (double)g.T);
+                                                   k.steps_total);
     if (tid == 0) dev::bulk_store_wait_read();
 }
 
@@ -790,7 +790,7 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
         }
     }
     if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef,
-                                                   (double)g.B * (double)g.T);
+                                                   k.steps_total);
     if (tid == 0) dev::bulk_store_wait_read();  // shared memory must outlive the store's reads
 }
 
@@ -1267,7 +1267,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     // as it appears and writes the loss terms
     if (blockIdx.x == 0 && grp == (n_tiles - 1) % C) {
         if (!dev::reduce_tagged_rows<NT>(p.tagged_rows, (int)gridDim.x, dev::launch_tag(p.counter), p.counter,
-                                         p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, (double)g.B * (double)g.T,
+                                         p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, k.steps_total,
                                          gtid, bar_id, &abort_s))
             if (gtid == 0) atomicExch(p.counter + 1, 1u);
     }
@@ -1406,7 +1406,7 @@ __global__ void __launch_bounds__(NT) impact_loss_gaussian_kernel(const GaussPar
         }
     }
     dev::finish_loss_terms<NT>(acc, p.partials, p.counter, p.loss_terms, k,
-                               (double)g.B * (double)g.T);
+                               k.steps_total);
 }
 
 // ------------------------------------------------------------------------------------------
@@ -1611,7 +1611,7 @@ __global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kern
         }
     }
     if (is_last_s) dev::reduce_published_sums<NT>(p.partials, p.counter, p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef,
-                                                   (double)g.B * (double)g.T);
+                                                   k.steps_total);
     if (tid == 0) dev::bulk_store_wait_read();
 }
 
@@ -2000,7 +2000,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     if (grp >= n_tiles) hand_over_sums();
     if (blockIdx.x == 0 && grp == (n_tiles - 1) % C) {
         if (!dev::reduce_tagged_rows<NT>(p.tagged_rows, (int)gridDim.x, dev::launch_tag(p.counter), p.counter,
-                                         p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, (double)g.B * (double)g.T,
+                                         p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, k.steps_total,
                                          gtid, bar_id, &abort_s))
             if (gtid == 0) atomicExch(p.counter + 1, 1u);
     }
@@ -2081,7 +2081,10 @@ int32_t fill_scalars(LossScalars& k, float rho_bar, float c_bar, float clip_eps,
     k.kl_coef = coef->kl_coef;
     k.lambda_ = coef->lambda_;
     k.log_rho_tw = (float)log((double)coef->rho_tw);
-    k.inv_M = (float)(1.0 / ((double)B * (double)T));
+    const double own = (double)B * (double)T;
+    if (coef->global_steps != 0 && (double)coef->global_steps < own) return IMPACT_ERR_INVALID_ARG;
+    k.steps_total = coef->global_steps != 0 ? (double)coef->global_steps : own;
+    k.inv_M = (float)(1.0 / k.steps_total);
     k.is_source = coef->is_source;
     k.ratio_mode = coef->ratio_mode;
     k.objective = coef->objective;

@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_housekeeping_calls(lib):
-    assert lib.impact_version() == 100
+    assert lib.impact_version() == 200
     assert lib.impact_status_string(0) == b"ok"
     assert b"full" in lib.impact_status_string(-5)
     assert b"empty" in lib.impact_status_string(-4)
@@ -41,8 +41,9 @@ def test_housekeeping_calls(lib):
 
 def test_struct_layout_matches_header():
     from paper_1912_00167_b200.binding import impact_coefficients
-    assert ctypes.sizeof(impact_coefficients) == 36
+    assert ctypes.sizeof(impact_coefficients) == 48
     assert impact_coefficients.rho_tw.offset == 16 and impact_coefficients.objective.offset == 32
+    assert impact_coefficients.global_steps.offset == 40
 
 
 def test_host_side_validation_needs_no_gpu(lib):

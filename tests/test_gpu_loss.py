@@ -301,3 +301,42 @@ def test_baseline_objectives_gaussian(oracle):
     P.check_gaussian(oracle, batch, dataclasses.replace(cfg.hyper, objective=1, is_source=1, lam=1.0))
     small = ii.gaussian_batch(3, 140, 5, seed=77, p_done=0.05)
     P.check_gaussian(oracle, small, LossHyper(objective=1, is_source=1, ent_coef=0.01, kl_coef=0.2))
+
+
+@pytest.mark.parametrize("B,T,A,parts", [(37, 50, 18, 2), (300, 128, 6, 3), (9, 300, 9, 2)])
+def test_batch_split_over_calls_adds_up_to_the_whole(oracle, B, T, A, parts):
+    """Data parallel over trajectories, every share run on this one GPU in turn: with `global_steps` set to the whole
+    batch's M the shares' gradients are the whole batch's rows and their loss terms add up to the whole batch's --
+    which is what the oracle computes for the unsplit batch."""
+    import paper_1912_00167_b200 as ip
+    batch = ii.categorical_batch(B, T, A, seed=77 + B, p_done=0.01)
+    h = P.f32_hyper(LossHyper(clip_eps=0.3, kl_coef=0.1, rho_tw=2.0, lam=0.98))
+    ref = oracle.loss_categorical(batch, h)
+    M = B * T
+    terms = np.zeros(8)
+    dz, dv = np.zeros((B, T, A)), np.zeros((B, T))
+    for r in range(parts):
+        lo, hi = ip.shard_bounds(B, parts, r)
+        t = {k_: torch.from_numpy(np.ascontiguousarray(v[lo:hi])).cuda() for k_, v in batch.items()}
+        out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(hi - lo, T, A, device="cuda"),
+                   dvalues=torch.empty(hi - lo, T, device="cuda"))
+        ip.impact_loss_fwd_bwd_sharded(t["learner_logits"], t["target_logits"], t["worker_logp"], t["actions"],
+                                       t["rewards"], t["discounts"], t["values"], t["bootstrap_values"], P.to_coef(h),
+                                       global_B=B, workspace=ip.new_workspace(hi - lo, T), **out)
+        torch.cuda.synchronize()
+        terms += out["loss_terms"].cpu().numpy().astype(np.float64)
+        dz[lo:hi], dv[lo:hi] = out["dlogits"].cpu().numpy(), out["dvalues"].cpu().numpy()
+    np.testing.assert_allclose(terms, ref["loss_terms"], rtol=1e-4, atol=1e-6)
+    near = P.near_clip_bound(ref, h)
+    tol = 1e-5 * np.abs(ref["dlogits"] * M) + 1e-6 + 4e-6 * (ref["adv_cond"] * ref["ratio"])[..., None]
+    assert (np.abs(dz * M - ref["dlogits"] * M) <= tol)[~near].all()
+    np.testing.assert_array_less(np.abs(dv * M - ref["dvalues"] * M), 1e-5 * np.abs(ref["dvalues"] * M) + 1e-6 + 4e-6 * ref["adv_cond"])
+    # a normaliser smaller than the call's own steps is refused
+    with pytest.raises(ip.ImpactError):
+        lo, hi = 0, B
+        t = {k_: torch.from_numpy(v).cuda() for k_, v in batch.items()}
+        ip.impact_loss_fwd_bwd(t["learner_logits"], t["target_logits"], t["worker_logp"], t["actions"], t["rewards"],
+                               t["discounts"], t["values"], t["bootstrap_values"],
+                               dataclasses.replace(P.to_coef(h), global_steps=M - 1), workspace=ip.new_workspace(B, T),
+                               loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
+                               dvalues=torch.empty(B, T, device="cuda"))
