@@ -813,6 +813,7 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
 // workspace's error word and the block's abort flag, after which nobody waits any more and
 // the block runs to its end on whatever the stages hold.
 constexpr int kWsMaxStages = 24;
+constexpr int kWsFewTiles = 32;  // up to this many tiles per block the producer works for latency, beyond for throughput
 constexpr int kWsGroups = 4;  // consumer groups per block: 16 consumer warps + the producer warp, <= 120 registers each
 
 // Row passes of one step, shared by the kernels with a compile-time action count.  `zr` / `tr`
@@ -874,7 +875,7 @@ struct RowMath {
 // than the waiting one.
 template <typename LT, typename GT, int A, int C, bool kPlain, bool kLong>
 __global__ void __launch_bounds__(C * 128 + 32, 1)
-impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W) {
+impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W, const int lanes) {
     constexpr int NT = 128;
     constexpr int NP = (A + 1) / 2;
     constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
@@ -956,12 +957,9 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         dev::fence_mbarrier_init();
         __syncwarp();
 
-        // lane 0 streams the block's tiles into the ring
         grid_dependency_wait();
 
-        int s = 0, ws = 0;         // stage of tile n, stage of tile n - W
-        uint32_t ph = 0, wph = 0;  // their phase parities
-        auto send_tile = [&](int n) {
+        auto send_tile = [&](int n, int s) {
             const Place pc = place_of(n);
             const int nrows = pc.nrows;
             const LT* const gl = static_cast<const LT*>(p.learner_logits) + pc.row0 * A;
@@ -981,20 +979,57 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
                 }
                 dev::mbarrier_arrive(&full_bar[s]);
             }
-            if (++s == S) { s = 0; ph ^= 1u; }
-            if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
         };
-        // the first W tiles need no wait, and leave before the rest of the block has even started
-        if (lane == 0)
-            for (int n = 0; n < n_first; ++n) send_tile(n);
+        // the first W tiles need no wait (tile n goes to stage n), and leave, a lane each, before the rest of the
+        // block has even started
+        if (lane < n_first) send_tile(lane, lane);
         __syncthreads();  // the barriers are set up: the consumer warps may use them
-        if (lane == 0) {
-            for (int n = n_first; n < n_tiles; ++n) {
-                bool ok = true;
-                if (n >= S) ok = dev::mbarrier_wait(&empty_bar[s], ph ^ 1u, &abort_s);   // the stage's previous tile has left
-                if (ok && n >= W) ok = dev::mbarrier_wait(&full_bar[ws], wph, &abort_s);  // at most W tiles in flight
-                if (!ok) { atomicExch(p.counter + 1, 1u); break; }
-                send_tile(n);
+        // The rest.  Tile n goes to stage n % S once that stage's previous tile has left (the "empty" phase
+        // before this one) and tile n - W has landed (at most W tiles in flight).
+        if (n_tiles <= kWsFewTiles) {
+            // few tiles per block (a launch of a few microseconds): lane 0 alone, in blocking waits that the
+            // hardware ends the moment the barrier completes -- what counts here is how soon the next request
+            // leaves
+            if (lane == 0) {
+                int s = n_first % S, ws = 0;
+                uint32_t ph = (uint32_t)(n_first / S) & 1u, wph = 0;
+                for (int n = n_first; n < n_tiles; ++n) {
+                    bool ok = true;
+                    if (n >= S) ok = dev::mbarrier_wait(&empty_bar[s], ph ^ 1u, &abort_s);
+                    if (ok) ok = dev::mbarrier_wait(&full_bar[ws], wph, &abort_s);  // n >= W here
+                    if (!ok) { atomicExch(p.counter + 1, 1u); break; }
+                    send_tile(n, s);
+                    if (++s == S) { s = 0; ph ^= 1u; }
+                    if (++ws == S) { ws = 0; wph ^= 1u; }
+                }
+            }
+        } else {
+            // many tiles per block: `lanes` tiles per round, a lane each, polling.  One thread walking through a
+            // tile's address arithmetic and barrier operations needs about half a microsecond, more than an SM has
+            // per tile when tiles are small.  Within a round no lane can get S - W tiles ahead of another
+            // (lanes <= S - W), so the barrier of tile n - W is still in the phase that the test asks about.
+            for (int base = n_first; base < n_tiles; base += lanes) {
+                const int n = base + lane;
+                bool pending = lane < lanes && n < n_tiles;
+                const int cyc = n / S, s = n - cyc * S;
+                const int wcyc = (n - W) / S, ws = (n - W) - wcyc * S;
+                for (unsigned int spin = 0; spin < (1u << 22); ++spin) {
+                    if (pending && (cyc == 0 || dev::mbarrier_test(&empty_bar[s], (uint32_t)(cyc - 1) & 1u)) &&
+                        dev::mbarrier_test(&full_bar[ws], (uint32_t)wcyc & 1u)) {
+                        send_tile(n, s);
+                        pending = false;
+                    }
+                    if (!__any_sync(0xffffffffu, pending)) break;
+                    if (*reinterpret_cast<volatile int*>(&abort_s)) break;
+                    __nanosleep(32);
+                }
+                if (__any_sync(0xffffffffu, pending)) {  // a stage never came back, or a tile never landed
+                    if (lane == 0) {
+                        atomicExch(p.counter + 1, 1u);
+                        *reinterpret_cast<volatile int*>(&abort_s) = 1;
+                    }
+                    break;
+                }
             }
         }
         __syncwarp();
@@ -1020,6 +1055,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
                 todo &= ~(1u << c);
             }
             if (*reinterpret_cast<volatile int*>(&abort_s)) break;
+            if (n_tiles > kWsFewTiles) __nanosleep(64);  // a long launch: leave the issue slots to the consumers
         }
         if (todo == 0u) {
             float y = yc[0];
@@ -1762,6 +1798,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
                 todo &= ~(1u << c);
             }
             if (*reinterpret_cast<volatile int*>(&abort_s)) break;
+            __nanosleep(64);
         }
         if (todo == 0u) {
             float y = yc[0];
@@ -2167,7 +2204,8 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     }
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
     const long long grid = tiles < di->sm_count ? tiles : di->sm_count;
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W));
+    const int lanes = (S - W) < 4 ? ((S - W) < 1 ? 1 : (S - W)) : 4;  // producer lanes that request tiles side by side
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W, lanes));
     return IMPACT_OK;
 }
 
