@@ -814,7 +814,7 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
 // the block runs to its end on whatever the stages hold.
 constexpr int kWsMaxStages = 24;
 constexpr int kWsFewTiles = 32;  // up to this many tiles per block the producer works for latency, beyond for throughput
-constexpr int kWsGroups = 4;  // consumer groups per block: 16 consumer warps + the producer warp, <= 120 registers each
+constexpr int kWsGroups = 4;  // consumer groups per block at least (16 consumer warps + the producer warp)
 
 // Row passes of one step, shared by the kernels with a compile-time action count.  `zr` / `tr`
 // point at the thread's learner / target row in shared memory.
@@ -2190,7 +2190,9 @@ void ws_ring_shape(size_t stage_bytes, size_t tile_in_bytes, int groups, int max
 
 template <typename LT, typename GT, int A, bool kPlain, bool kLong>
 int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
-    constexpr int C = kWsGroups;
+    // Consumer groups: four with every switch compiled in (96 registers); five in the default configuration (80
+    // registers, no spills); six there for small action sets, which are bound by arithmetic, not bytes, and fit 72.
+    constexpr int C = !kPlain ? kWsGroups : (A <= 9 ? kWsGroups + 2 : kWsGroups + 1);
     auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong>;
     const size_t stage = reg_kernel_stage_bytes<LT, GT, A>();
     int S = 0, W = 0;
