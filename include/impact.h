@@ -257,8 +257,8 @@ int32_t impact_loss_fwd_bwd_gaussian(
  *
  * Limits: A <= 64, and the batch must split into at most 1024 tiles of 128 steps:
  * ceil(B / floor(128 / T)) <= 1024 when T <= 128, else B <= 1024.  (B=1024, T=128 is the
- * largest batch of full-length trajectories.  One combination works on tiles of 64 steps and
- * so fits half as much: 32 < A <= 64 with fp32 logits and bf16 gradients.)  Larger batches return
+ * largest batch of full-length trajectories.  Rows wider than 32 actions may be worked on in
+ * tiles of 64 steps and then fit half as much: count 64 for 128 above.)  Larger batches return
  * IMPACT_ERR_WORKSPACE_TOO_SMALL, A > 64 returns IMPACT_ERR_UNSUPPORTED; use
  * impact_loss_fwd_bwd with a workspace for those.
  *

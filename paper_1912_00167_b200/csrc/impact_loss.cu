@@ -812,6 +812,12 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
 // stage) says it may be refilled.  Every wait is bounded; a wait that gives up raises the
 // workspace's error word and the block's abort flag, after which nobody waits any more and
 // the block runs to its end on whatever the stages hold.
+template <typename LT, typename GT, int A, int NT>
+__host__ __device__ constexpr size_t ws_stage_bytes() {
+    constexpr size_t in_row = A * sizeof(LT), out_row = A * sizeof(GT);
+    return NT * (2 * in_row + (sizeof(LT) == sizeof(GT) ? 0 : out_row));
+}
+constexpr int ws_tile_rows(int A) { return A > 32 ? 64 : 128; }
 constexpr int kWsMaxStages = 24;
 constexpr int kWsFewTiles = 32;  // up to this many tiles per block the producer works for latency, beyond for throughput
 constexpr int kWsGroups = 4;  // consumer groups per block at least (16 consumer warps + the producer warp)
@@ -873,13 +879,19 @@ struct RowMath {
 // its own last step.  Nothing waits on a chain of tiles: every tile waits only for aggregates, which need
 // nothing but their own tile's rows, and only of tiles with a smaller number, which no block starts later
 // than the waiting one.
-template <typename LT, typename GT, int A, int C, bool kPlain, bool kLong>
-__global__ void __launch_bounds__(C * 128 + 32, 1)
+//
+// NT: steps per tile = threads per consumer group (128; 64 for A = 64, whose rows are four times as long).
+// Rows wider than 32 actions are not held in registers: every pass streams the row from shared memory, the
+// gradient pass forms the exponentials again, and thread r starts its walk at pair r mod (A/2), because a row
+// pitch of 256 bytes would otherwise put all threads of a warp on the same banks.
+template <typename LT, typename GT, int A, int C, bool kPlain, bool kLong, int NT>
+__global__ void __launch_bounds__(C * NT + 32, 1)
 impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W, const int lanes) {
-    constexpr int NT = 128;
     constexpr int NP = (A + 1) / 2;
+    constexpr bool kStream = (A > 32);
+    static_assert(!kStream || (A % 2 == 0 && (NP & (NP - 1)) == 0), "streamed rows: an even, power-of-two pair count");
     constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
-    constexpr int kStageBytes = (int)reg_kernel_stage_bytes<LT, GT, A>();
+    constexpr int kStageBytes = (int)ws_stage_bytes<LT, GT, A, NT>();
     constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
     using RM = RowMath<LT, A>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -1069,7 +1081,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     }
 
     // ---- consumer groups ------------------------------------------------------------------
-    const int grp = tid >> 7, gtid = tid & (NT - 1), gwarp = gtid >> 5;
+    const int grp = tid / NT, gtid = tid & (NT - 1), gwarp = gtid >> 5;
     const int bar_id = grp + 1;
     const bool want_kl = !kPlain && (k.kl_coef != 0.0f);
 
@@ -1168,24 +1180,78 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         st.last_step = me.last_step;
 
         // ---- row passes (every thread; rows beyond the tile hold stale bytes and are masked)
-        float2 e[NP];
-        float m2_t, sum_t, unused, m2_l, sum_l, sez;
-        const float lse2_t = RM::template lse2<false>(s1, gtid, e, m2_t, sum_t, unused);
-        st.l_target = fmaf(RowIO<LT, A>::at(s1, gtid, a), kLog2e, -lse2_t) * kLn2;
-        const float lse2_l = RM::template lse2<true>(s0, gtid, e, m2_l, sum_l, sez);
-        const float inv_s = dev::rcp_fast(sum_l);
-        // H = -sum_j pi_j lp_j = (m + ln S) - sum_j e_j z_j / S
-        const float ent = fmaf(lse2_l, kLn2, -sez * inv_s);
-        st.l_theta = fmaf(RowIO<LT, A>::at(s0, gtid, a), kLog2e, -lse2_l) * kLn2;
+        float2 e[kStream ? 1 : NP];
+        float lse2_t, lse2_l, inv_s, ent, m2_l = 0.0f;
         float kl = 0.0f;
-        if (want_kl) {
+        if constexpr (!kStream) {
+            float m2_t, sum_t, unused, sum_l, sez;
+            lse2_t = RM::template lse2<false>(s1, gtid, e, m2_t, sum_t, unused);
+            lse2_l = RM::template lse2<true>(s0, gtid, e, m2_l, sum_l, sez);
+            inv_s = dev::rcp_fast(sum_l);
+            // H = -sum_j pi_j lp_j = (m + ln S) - sum_j e_j z_j / S
+            ent = fmaf(lse2_l, kLn2, -sez * inv_s);
+            if (want_kl) {
 #pragma unroll
-            for (int j = 0; j < A; ++j) {
-                const float lpt2 = fmaf(RowIO<LT, A>::at(s1, gtid, j), kLog2e, -lse2_t);
-                const float lpl2 = fmaf(RowIO<LT, A>::at(s0, gtid, j), kLog2e, -lse2_l);
-                kl = fmaf(dev::exp2_fast(lpt2), (lpt2 - lpl2) * kLn2, kl);
+                for (int j = 0; j < A; ++j) {
+                    const float lpt2 = fmaf(RowIO<LT, A>::at(s1, gtid, j), kLog2e, -lse2_t);
+                    const float lpl2 = fmaf(RowIO<LT, A>::at(s0, gtid, j), kLog2e, -lse2_l);
+                    kl = fmaf(dev::exp2_fast(lpt2), (lpt2 - lpl2) * kLn2, kl);
+                }
+            }
+        } else {
+            const int skew = gtid & (NP - 1);
+            const float2 log2e2 = make_float2(kLog2e, kLog2e);
+            auto row_max2 = [&](const unsigned char* slab) {
+                float2 mx = RowIO<LT, A>::load_pair(slab, gtid, skew);
+#pragma unroll 8
+                for (int j = 1; j < NP; ++j) {
+                    const float2 v = RowIO<LT, A>::load_pair(slab, gtid, (j + skew) & (NP - 1));
+                    mx.x = fmaxf(mx.x, v.x);
+                    mx.y = fmaxf(mx.y, v.y);
+                }
+                return fmaxf(mx.x, mx.y) * kLog2e;
+            };
+            {   // target row: its log-sum-exp
+                const float m2 = row_max2(s1);
+                const float2 neg_m2 = make_float2(-m2, -m2);
+                float2 sum2 = make_float2(0.0f, 0.0f);
+#pragma unroll 8
+                for (int j = 0; j < NP; ++j) {
+                    const float2 t2 = __ffma2_rn(RowIO<LT, A>::load_pair(s1, gtid, (j + skew) & (NP - 1)), log2e2, neg_m2);
+                    sum2 = __fadd2_rn(sum2, make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y)));
+                }
+                lse2_t = m2 + dev::log2_fast(sum2.x + sum2.y);
+            }
+            {   // learner row: log-sum-exp and sum_j e_j z_j
+                m2_l = row_max2(s0);
+                const float2 neg_m2 = make_float2(-m2_l, -m2_l);
+                float2 sum2 = make_float2(0.0f, 0.0f), sez2 = make_float2(0.0f, 0.0f);
+#pragma unroll 8
+                for (int j = 0; j < NP; ++j) {
+                    const float2 z = RowIO<LT, A>::load_pair(s0, gtid, (j + skew) & (NP - 1));
+                    const float2 t2 = __ffma2_rn(z, log2e2, neg_m2);
+                    const float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
+                    sum2 = __fadd2_rn(sum2, ex);
+                    sez2 = __ffma2_rn(ex, z, sez2);
+                }
+                const float sum_l = sum2.x + sum2.y;
+                lse2_l = m2_l + dev::log2_fast(sum_l);
+                inv_s = dev::rcp_fast(sum_l);
+                ent = fmaf(lse2_l, kLn2, -(sez2.x + sez2.y) * inv_s);
+            }
+            if (want_kl) {
+#pragma unroll 8
+                for (int j = 0; j < NP; ++j) {
+                    const int jj = (j + skew) & (NP - 1);
+                    const float2 zt2 = RowIO<LT, A>::load_pair(s1, gtid, jj), zl2 = RowIO<LT, A>::load_pair(s0, gtid, jj);
+                    const float ax = fmaf(zt2.x, kLog2e, -lse2_t), ay = fmaf(zt2.y, kLog2e, -lse2_t);
+                    kl = fmaf(dev::exp2_fast(ax), (ax - fmaf(zl2.x, kLog2e, -lse2_l)) * kLn2, kl);
+                    kl = fmaf(dev::exp2_fast(ay), (ay - fmaf(zl2.y, kLog2e, -lse2_l)) * kLn2, kl);
+                }
             }
         }
+        st.l_target = fmaf(RowIO<LT, A>::at(s1, gtid, a), kLog2e, -lse2_t) * kLn2;
+        st.l_theta = fmaf(RowIO<LT, A>::at(s0, gtid, a), kLog2e, -lse2_l) * kLn2;
         float fa, fb;
         bool truncated;
         if (kPlain) truncated = dev::recursion_map_plain(st, k, fa, fb);
@@ -1208,7 +1274,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
                                                                   dev::launch_tag(p.counter), &abort_s);
                     if (lane == 0) carry_s[grp] = c;
                 }
-                asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
+                asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory");
                 carry = carry_s[grp];
             }
             adv = fmaf(ma, carry, mb);
@@ -1238,21 +1304,40 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             const float h_off = fmaf(-lse2_l, kLn2, ent);
             const float ga = ce * inv_s, gb = (fmaf(ce, h_off, w1) + ck) * inv_s;
             const float2 ga2 = make_float2(ga, ga), gb2 = make_float2(gb, gb);
-            if (!want_kl) {
+            if constexpr (!kStream) {
+                if (!want_kl) {
 #pragma unroll
-                for (int j = 0; j < NP; ++j) {
-                    const float2 z = RowIO<LT, A>::load_pair(s0, gtid, j);
-                    RowIO<GT, A>::store_pair(so, gtid, j, __fmul2_rn(e[j], __ffma2_rn(z, ga2, gb2)));
+                    for (int j = 0; j < NP; ++j) {
+                        const float2 z = RowIO<LT, A>::load_pair(s0, gtid, j);
+                        RowIO<GT, A>::store_pair(so, gtid, j, __fmul2_rn(e[j], __ffma2_rn(z, ga2, gb2)));
+                    }
+                } else {
+                    const float2 neg_lse2 = make_float2(-lse2_t, -lse2_t), nck2 = make_float2(-ck, -ck);
+                    const float2 log2e2 = make_float2(kLog2e, kLog2e);
+#pragma unroll
+                    for (int j = 0; j < NP; ++j) {
+                        const float2 z = RowIO<LT, A>::load_pair(s0, gtid, j);
+                        const float2 tt = __ffma2_rn(RowIO<LT, A>::load_pair(s1, gtid, j), log2e2, neg_lse2);
+                        const float2 pt = make_float2(dev::exp2_fast(tt.x), dev::exp2_fast(tt.y));
+                        RowIO<GT, A>::store_pair(so, gtid, j, __ffma2_rn(nck2, pt, __fmul2_rn(e[j], __ffma2_rn(z, ga2, gb2))));
+                    }
                 }
             } else {
+                const int skew = gtid & (NP - 1);
+                const float2 log2e2 = make_float2(kLog2e, kLog2e), neg_m2 = make_float2(-m2_l, -m2_l);
                 const float2 neg_lse2 = make_float2(-lse2_t, -lse2_t), nck2 = make_float2(-ck, -ck);
-                const float2 log2e2 = make_float2(kLog2e, kLog2e);
-#pragma unroll
+#pragma unroll 8
                 for (int j = 0; j < NP; ++j) {
-                    const float2 z = RowIO<LT, A>::load_pair(s0, gtid, j);
-                    const float2 tt = __ffma2_rn(RowIO<LT, A>::load_pair(s1, gtid, j), log2e2, neg_lse2);
-                    const float2 pt = make_float2(dev::exp2_fast(tt.x), dev::exp2_fast(tt.y));
-                    RowIO<GT, A>::store_pair(so, gtid, j, __ffma2_rn(nck2, pt, __fmul2_rn(e[j], __ffma2_rn(z, ga2, gb2))));
+                    const int jj = (j + skew) & (NP - 1);
+                    const float2 z = RowIO<LT, A>::load_pair(s0, gtid, jj);
+                    const float2 t2 = __ffma2_rn(z, log2e2, neg_m2);
+                    const float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
+                    float2 gr = __fmul2_rn(ex, __ffma2_rn(z, ga2, gb2));
+                    if (want_kl) {
+                        const float2 tt = __ffma2_rn(RowIO<LT, A>::load_pair(s1, gtid, jj), log2e2, neg_lse2);
+                        gr = __ffma2_rn(nck2, make_float2(dev::exp2_fast(tt.x), dev::exp2_fast(tt.y)), gr);
+                    }
+                    RowIO<GT, A>::store_pair(so, gtid, jj, gr);
                 }
             }
             const float pi_a = dev::exp2_fast(st.l_theta * kLog2e);
@@ -2050,9 +2135,10 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
 constexpr int kMaxGridBlocks = 4096;  // upper bound on blocks of a loss launch (sizes the workspace)
 constexpr size_t kCounterBytes = 256; // words after the partials: [0] completion counter, [1] error flag, [2] launch number
 // Long trajectories (T > 128 steps): two (value, tag) pairs per 128-step tile, after everything else.
+constexpr int kMinTileRows = 64;  // the smallest tile of a persistent kernel
 size_t tile_aggregate_bytes(int64_t B, int64_t T) {
-    if (T <= kRegTileRows) return 0;
-    return (size_t)B * (size_t)((T + kRegTileRows - 1) / kRegTileRows) * 2 * sizeof(unsigned long long);
+    if (T <= kMinTileRows) return 0;
+    return (size_t)B * (size_t)((T + kMinTileRows - 1) / kMinTileRows) * 2 * sizeof(unsigned long long);
 }
 constexpr int kMaxTaggedRows = 1024;  // rows of eight (value, tag) pairs after the counter words: one per block of the persistent kernel
 
@@ -2192,11 +2278,13 @@ template <typename LT, typename GT, int A, bool kPlain, bool kLong>
 int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
     // Consumer groups: four with every switch compiled in (96 registers); five in the default configuration (80
     // registers, no spills); six there for small action sets, which are bound by arithmetic, not bytes, and fit 72.
-    constexpr int C = !kPlain ? kWsGroups : (A <= 9 ? kWsGroups + 2 : kWsGroups + 1);
-    auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong>;
-    const size_t stage = reg_kernel_stage_bytes<LT, GT, A>();
+    // Wide rows (A = 64): tiles of 64 steps, six groups of 64 threads.
+    constexpr int NT = ws_tile_rows(A);
+    constexpr int C = A > 32 ? 6 : (!kPlain ? kWsGroups : (A <= 9 ? kWsGroups + 2 : kWsGroups + 1));
+    auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong, NT>;
+    const size_t stage = ws_stage_bytes<LT, GT, A, NT>();
     int S = 0, W = 0;
-    ws_ring_shape(stage, 2 * (size_t)kRegTileRows * A * sizeof(LT), C, di->max_smem_optin, &S, &W);
+    ws_ring_shape(stage, 2 * (size_t)NT * A * sizeof(LT), C, di->max_smem_optin, &S, &W);
     if (S < 2) return IMPACT_ERR_UNSUPPORTED;
     const size_t smem = (size_t)S * stage;
     static thread_local int configured_device = -1;
@@ -2207,7 +2295,7 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
     const long long grid = tiles < di->sm_count ? tiles : di->sm_count;
     const int lanes = (S - W) < 4 ? ((S - W) < 1 ? 1 : (S - W)) : 4;  // producer lanes that request tiles side by side
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W, lanes));
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * NT + 32), smem, stream, p, S, W, lanes));
     return IMPACT_OK;
 }
 
@@ -2225,19 +2313,23 @@ int32_t launch_categorical_reg(const CatParams& p, const DeviceInfo* di, cudaStr
     }
     // Split across blocks while there are too few trajectories to give every consumer group of the device one of
     // its own; from there on the sweep inside a block keeps the device busy without any exchange between tiles.
-    if (p.tile_aggregates && p.geo.B < (long long)kWsGroups * di->sm_count)
+    if constexpr (A > 32) {  // no sweeping kernel for wide rows: run_categorical sends long trajectories here only with aggregates
         return launch_categorical_ws<LT, GT, A, false, true>(p, di, stream);
-    auto kernel = impact_loss_categorical_reg_kernel<LT, GT, A>;
-    const size_t smem = reg_kernel_smem<LT, GT, A>();
-    int grid = 0;
-    int32_t st = grid_for(kernel, kRegTileRows, smem, p.geo.nchunks, di, &grid);
-    if (st != IMPACT_OK) return st;
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3(grid), dim3(kRegTileRows), smem, stream, p));
-    return IMPACT_OK;
+    } else {
+        if (p.tile_aggregates && p.geo.B < (long long)kWsGroups * di->sm_count)
+            return launch_categorical_ws<LT, GT, A, false, true>(p, di, stream);
+        auto kernel = impact_loss_categorical_reg_kernel<LT, GT, A>;
+        const size_t smem = reg_kernel_smem<LT, GT, A>();
+        int grid = 0;
+        int32_t st = grid_for(kernel, kRegTileRows, smem, p.geo.nchunks, di, &grid);
+        if (st != IMPACT_OK) return st;
+        IMPACT_CUDA_TRY(launch_serialized(kernel, dim3(grid), dim3(kRegTileRows), smem, stream, p));
+        return IMPACT_OK;
+    }
 }
 
-// Action counts with a compiled register-resident kernel (the Atari action sets).
-constexpr bool has_reg_kernel(int A) { return A == 4 || A == 6 || A == 9 || A == 18; }
+// Action counts with a compiled kernel (the Atari action sets, and 64).
+constexpr bool has_reg_kernel(int A) { return A == 4 || A == 6 || A == 9 || A == 18 || A == 64; }
 
 template <typename LT, typename GT>
 int32_t dispatch_reg(const CatParams& p, const DeviceInfo* di, cudaStream_t stream) {
@@ -2245,13 +2337,14 @@ int32_t dispatch_reg(const CatParams& p, const DeviceInfo* di, cudaStream_t stre
         case 4: return launch_categorical_reg<LT, GT, 4>(p, di, stream);
         case 6: return launch_categorical_reg<LT, GT, 6>(p, di, stream);
         case 9: return launch_categorical_reg<LT, GT, 9>(p, di, stream);
+        case 64: return launch_categorical_reg<LT, GT, 64>(p, di, stream);
         default: return launch_categorical_reg<LT, GT, 18>(p, di, stream);
     }
 }
 
 // Steps per tile of the kernel that run_categorical picks for this call.
-int categorical_tile_rows(int A, bool logits_bf16, bool grads_bf16) {
-    if (has_reg_kernel(A)) return kRegTileRows;
+int categorical_tile_rows(int A, bool logits_bf16, bool grads_bf16, bool long_without_aggregates) {
+    if (has_reg_kernel(A) && !(A > 32 && long_without_aggregates)) return ws_tile_rows(A);
     return pick_nt_categorical(A, logits_bf16 ? 2 : 4, grads_bf16 ? 2 : 4, 72 * 1024);
 }
 
@@ -2259,16 +2352,19 @@ int categorical_tile_rows(int A, bool logits_bf16, bool grads_bf16) {
 // the generic one.  `p` arrives complete except for As and geo.
 int32_t run_categorical(CatParams& p, int64_t B, int64_t T, bool logits_bf16, bool grads_bf16,
                         const DeviceInfo* di, cudaStream_t s) {
-    if (has_reg_kernel(p.A)) {
+    // (wide rows have no kernel that sweeps a long trajectory inside one block: without room for the tiles'
+    // aggregates such a call takes the runtime-width kernel)
+    const bool long_without_aggregates = T > ws_tile_rows(p.A) && !p.tile_aggregates;
+    if (has_reg_kernel(p.A) && !(p.A > 32 && long_without_aggregates)) {
         p.As = p.A;
-        p.geo = make_geometry(B, T, kRegTileRows);
+        p.geo = make_geometry(B, T, ws_tile_rows(p.A));
         if (!logits_bf16 && !grads_bf16) return dispatch_reg<float, float>(p, di, s);
         if (!logits_bf16 && grads_bf16) return dispatch_reg<float, __nv_bfloat16>(p, di, s);
         if (logits_bf16 && !grads_bf16) return dispatch_reg<__nv_bfloat16, float>(p, di, s);
         return dispatch_reg<__nv_bfloat16, __nv_bfloat16>(p, di, s);
     }
     p.As = p.A;
-    const int nt = categorical_tile_rows(p.A, logits_bf16, grads_bf16);
+    const int nt = categorical_tile_rows(p.A, logits_bf16, grads_bf16, long_without_aggregates);
     p.geo = make_geometry(B, T, nt);
     if (!logits_bf16 && !grads_bf16) return dispatch_nt<float, float>(p, nt, di, s);
     if (!logits_bf16 && grads_bf16) return dispatch_nt<float, __nv_bfloat16>(p, nt, di, s);
@@ -2403,7 +2499,7 @@ extern "C" int32_t impact_loss_fwd_bwd(
                                                 (size_t)kMaxGridBlocks * 8 * sizeof(float));
     p.tagged_rows = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) +
                                                           (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes);
-    p.tile_aggregates = T > kRegTileRows
+    p.tile_aggregates = T > kMinTileRows
                             ? reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWorkspaceFixedBytes)
                             : nullptr;
     p.A = A;
@@ -2546,7 +2642,7 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     if (logits_dtype != IMPACT_DTYPE_F32 && logits_dtype != IMPACT_DTYPE_BF16) return IMPACT_ERR_INVALID_ARG;
     if (coef->dlogits_dtype != IMPACT_DTYPE_F32 && coef->dlogits_dtype != IMPACT_DTYPE_BF16)
         return IMPACT_ERR_INVALID_ARG;
-    if (A > 64) return IMPACT_ERR_UNSUPPORTED;  // keeps the tile at 128 steps, which the limit below counts in
+    if (A > 64) return IMPACT_ERR_UNSUPPORTED;  // keeps the tile at 64 steps or more, which the limit below counts in
 
     CatParams p;
     int32_t st = fill_scalars(p.k, rho_bar, c_bar, clip_eps, coef, B, T);
@@ -2554,7 +2650,7 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     p.A = A;
     // one block's sums per tile at most: more tiles than the built-in scratch holds are refused
     const bool logits_bf16 = logits_dtype == IMPACT_DTYPE_BF16, grads_bf16 = coef->dlogits_dtype == IMPACT_DTYPE_BF16;
-    const int tile_rows_here = categorical_tile_rows(A, logits_bf16, grads_bf16);
+    const int tile_rows_here = categorical_tile_rows(A, logits_bf16, grads_bf16, T > ws_tile_rows(A));  // no aggregates here
     if (make_geometry(B, T, tile_rows_here).nchunks > kStaticMaxBlocks) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
 
     const DeviceInfo* di = current_device_info();

@@ -77,6 +77,24 @@ def test_bf16_ragged(oracle, B, T, A):
     P.check_categorical(oracle, batch, h, torch.bfloat16, torch.float32)
 
 
+@pytest.mark.parametrize("B,T,A", [(300, 64, 64), (7, 128, 64), (3, 200, 64), (1500, 20, 64), (33, 63, 64)])
+@pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
+def test_wide_rows_in_the_persistent_kernel(oracle, B, T, A, dtype):
+    """A = 64: tiles of 64 steps, rows streamed from shared memory with a skewed walk; one tile per trajectory,
+    several trajectories per tile, trajectories over two and four tiles, more tiles per block than stages; the
+    default configuration (switches compiled out) and the full one."""
+    batch = ii.categorical_batch(B, T, A, seed=640 + B + T, p_done=0.01)
+    plain = LossHyper(rho_bar=1.0, c_bar=1.0, clip_eps=0.3, vf_coef=0.5, ent_coef=0.01, kl_coef=0.0, rho_tw=1.0)
+    full = LossHyper(rho_bar=1.3, c_bar=1.1, clip_eps=0.25, vf_coef=0.7, ent_coef=0.02, kl_coef=0.1, lam=0.97, rho_tw=2.0)
+    if dtype == torch.bfloat16:
+        P.check_categorical(oracle, batch, plain, torch.bfloat16, torch.bfloat16, extra=False, rtol=P.RTOL_BF16,
+                            atol=P.ATOL_BF16)
+        P.check_categorical(oracle, batch, full, torch.bfloat16, torch.float32)
+    else:
+        P.check_categorical(oracle, batch, plain, extra=False)
+        P.check_categorical(oracle, batch, full)
+
+
 @pytest.mark.parametrize("B,T,A,dtype", [(2, 4500, 6, torch.float32), (5, 1300, 9, torch.float32),
                                          (1, 130, 18, torch.float32), (40, 257, 18, torch.bfloat16),
                                          (700, 256, 18, torch.float32), (3, 640, 4, torch.float32)])
