@@ -406,25 +406,34 @@ __device__ __forceinline__ void publish_tile_aggregate(unsigned long long* slot,
     publish_tagged(slot + 1, b, tag);
 }
 
-// Run by one warp: `mine` points at this tile's pair of slots; the `r` tiles before it in the array are
-// the later tiles of its trajectory, the nearest first.  Reads their aggregates (a lane each, 32 at a
-// time, waiting -- bounded -- until a pair carries this launch's tag), composes them in time order and
-// returns the composition applied to 0: the value that enters this tile's last step.
-__device__ __forceinline__ float compose_later_aggregates(const unsigned long long* mine, int r, unsigned int tag,
-                                                          int* abort_flag) {
+// The two slots of the aggregate of the tile `j` places later in this tile's trajectory (they lie j * stride
+// before `mine`), as they are right now.  The values are not looked at here, so the load can be issued long before
+// it is needed.
+__device__ __forceinline__ void load_aggregate(const unsigned long long* mine, long long stride, int j,
+                                               unsigned long long& va, unsigned long long& vb) {
+    asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(va), "=l"(vb) : "l"(mine - (long long)j * stride) : "memory");
+}
+
+// Run by one warp: `mine` points at this tile's pair of slots; tile j (1 = the nearest later tile ... r = the
+// trajectory's last) has its slots at mine - j * stride.  Reads their aggregates (a lane each, 32 at a time,
+// waiting -- bounded -- until a pair carries this launch's tag), composes them in time order and returns the
+// composition applied to 0: the value that enters this tile's last step.  `peeked` / (pa, pb): lane l brings along
+// what load_aggregate found earlier for tile r - l; it counts if it carries the tag.
+__device__ __forceinline__ float compose_later_aggregates(const unsigned long long* mine, long long stride, int r,
+                                                          unsigned int tag, int* abort_flag, bool peeked,
+                                                          unsigned long long pa, unsigned long long pb) {
     const int lane = threadIdx.x & 31;
-    // tile j (1 = the nearest later tile ... r = the trajectory's last) sits at mine - 2 j; the value flows
-    // from tile r down to tile 1: x <- agg_j(x).  Lanes take j = r - lane, r - lane - 32, ...: chunk by
-    // chunk from the far end, lane 0 holding the map that is applied first.
+    // the value flows from tile r down to tile 1: x <- agg_j(x).  Lanes take j = r - lane, r - lane - 32, ...:
+    // chunk by chunk from the far end, lane 0 holding the map that is applied first.
     float x = 0.0f;
     for (int base = r; base > 0; base -= 32) {
         const int j = base - lane;
         float a = 1.0f, b = 0.0f;  // identity for lanes beyond the chunk
         if (j > 0) {
-            unsigned long long va = 0, vb = 0;
-            bool ok = false;
+            unsigned long long va = pa, vb = pb;
+            bool ok = peeked && base == r && ((unsigned int)(va >> 32) == tag) && ((unsigned int)(vb >> 32) == tag);
             for (int tries = 0; tries < (1 << 22) && !ok; ++tries) {
-                asm volatile("ld.relaxed.gpu.global.v2.u64 {%0, %1}, [%2];" : "=l"(va), "=l"(vb) : "l"(mine - 2 * (long long)j) : "memory");
+                load_aggregate(mine, stride, j, va, vb);
                 ok = ((unsigned int)(va >> 32) == tag) && ((unsigned int)(vb >> 32) == tag);
                 if (!ok && *reinterpret_cast<volatile int*>(abort_flag)) break;
             }

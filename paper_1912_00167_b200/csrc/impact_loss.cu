@@ -21,6 +21,7 @@ namespace {
 using dev::LossScalars;
 
 struct TileGeometry {
+    int tile_major;  // long trajectories in a persistent kernel: order of the grid's tiles (see place_of)
     long long B, T;
     long long nchunks;  // units of block-level work
     int G;              // whole trajectories per chunk (T <= NT), else 1
@@ -871,9 +872,11 @@ struct RowMath {
 // kPlain: the configuration of the paper's experiments -- no KL term, the clipped surrogate with the
 // default ratio and importance weights, no optional outputs -- with those branches compiled out.
 //
-// kLong: trajectories longer than a tile.  Tile g of the grid is tile g % ntiles, counted from the END, of
-// trajectory g / ntiles, so the tiles of one trajectory go to neighbouring blocks and are worked on at the same
-// time.  The recursion crosses tiles through their affine aggregates: a tile composes its 128 maps into one
+// kLong: trajectories longer than a tile.  The grid's tiles are numbered either trajectory by trajectory, each from
+// its END backwards (few tiles in all: the tiles of one trajectory go to neighbouring blocks, are contiguous in
+// memory and are worked on at the same time), or tile-major (many: all trajectories' last tiles first, then the tiles
+// before them, ..., so that the aggregates a tile needs were published a round earlier and one early look finds
+// them).  The recursion crosses tiles through their affine aggregates: a tile composes its 128 maps into one
 // (a, b), publishes it as two (value, launch tag) pairs, reads the aggregates of the later tiles of its
 // trajectory -- all of them at once, a lane each -- and composes them, applied to 0, into the value that enters
 // its own last step.  Nothing waits on a chain of tiles: every tile waits only for aggregates, which need
@@ -909,6 +912,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     const int n_tiles = (int)((total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);  // this block's tiles
     const int rows_full = kLong ? NT : g.G * (int)g.T;                                   // rows of a full tile
     const long long total_rows = g.B * g.T;
+    const long long agg_stride = g.tile_major ? 2 * g.B : 2;  // slots between a tile's aggregate and that of the tile after it in time
     // where the block's n-th tile sits: first row, rows, and (kLong) trajectory and tile number from its end
     struct Place {
         long long row0, traj;
@@ -918,8 +922,13 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         Place pl;
         const long long gt_ = (long long)blockIdx.x + (long long)n * gridDim.x;
         if (kLong) {
-            pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
-            pl.r = (int)(gt_ - pl.traj * g.ntiles);
+            if (g.tile_major) {  // the last tiles of all trajectories first, then the tiles before them, ...
+                pl.r = (int)((unsigned long long)gt_ / (unsigned long long)g.B);
+                pl.traj = gt_ - (long long)pl.r * g.B;
+            } else {  // trajectory by trajectory, each from its last tile backwards
+                pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
+                pl.r = (int)(gt_ - pl.traj * g.ntiles);
+            }
             const long long t0 = (long long)(g.ntiles - 1 - pl.r) * NT;
             const long long left = g.T - t0;
             pl.nrows = left < NT ? (int)left : NT;
@@ -1165,6 +1174,15 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         }
         // every thread waits for the stage itself (a bounded wait: on a time-out the flag is set and the
         // thread goes on with whatever the stage holds, so that all barriers below still pair up)
+        // (long trajectories) one early look at the aggregates of the later tiles of this tile's trajectory: with
+        // many trajectories they were published a round ago, and reading them now keeps that trip to L2 off the
+        // path between this tile's scan and its gradients
+        // (only where tiles are numbered tile-major; the values are first looked at after the scan)
+        const bool peeked = kLong && g.tile_major && gwarp == 0 && me.pc.r > lane;
+        unsigned long long early_a = 0, early_b = 0;
+        if (peeked)
+            dev::load_aggregate(p.tile_aggregates + 2 * ((long long)blockIdx.x + (long long)n * gridDim.x), agg_stride,
+                                me.pc.r - lane, early_a, early_b);
         if (!dev::mbarrier_wait(&full_bar[s], ph, &abort_s)) atomicExch(p.counter + 1, 1u);
 
         unsigned char* const s0 = smem_raw + s * kStageBytes;  // learner logits
@@ -1270,8 +1288,9 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             float carry = 0.0f;
             if (me.pc.r > 0) {  // uniform over the group
                 if (gwarp == 0) {
-                    const float c = dev::compose_later_aggregates(p.tile_aggregates + 2 * gtile, me.pc.r,
-                                                                  dev::launch_tag(p.counter), &abort_s);
+                    const float c = dev::compose_later_aggregates(p.tile_aggregates + 2 * gtile, agg_stride, me.pc.r,
+                                                                  dev::launch_tag(p.counter), &abort_s, peeked,
+                                                                  early_a, early_b);
                     if (lane == 0) carry_s[grp] = c;
                 }
                 asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory");
@@ -1769,6 +1788,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     const int n_tiles = (int)((total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
     const int rows_full = kLong ? NT : g.G * (int)g.T;
     const long long total_rows = g.B * g.T;
+    const long long agg_stride = g.tile_major ? 2 * g.B : 2;  // slots between a tile's aggregate and that of the tile after it in time
     struct Place {
         long long row0, traj;
         int nrows, r;
@@ -1777,8 +1797,13 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
         Place pl;
         const long long gt_ = (long long)blockIdx.x + (long long)n * gridDim.x;
         if (kLong) {
-            pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
-            pl.r = (int)(gt_ - pl.traj * g.ntiles);
+            if (g.tile_major) {  // the last tiles of all trajectories first, then the tiles before them, ...
+                pl.r = (int)((unsigned long long)gt_ / (unsigned long long)g.B);
+                pl.traj = gt_ - (long long)pl.r * g.B;
+            } else {  // trajectory by trajectory, each from its last tile backwards
+                pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
+                pl.r = (int)(gt_ - pl.traj * g.ntiles);
+            }
             const long long t0 = (long long)(g.ntiles - 1 - pl.r) * NT;
             const long long left = g.T - t0;
             pl.nrows = left < NT ? (int)left : NT;
@@ -1970,6 +1995,15 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
             dev::mbarrier_arrive(&empty_bar[pending_stage]);
             pending = false;
         }
+        // (long trajectories) one early look at the aggregates of the later tiles of this tile's trajectory: with
+        // many trajectories they were published a round ago, and reading them now keeps that trip to L2 off the
+        // path between this tile's scan and its gradients
+        // (only where tiles are numbered tile-major; the values are first looked at after the scan)
+        const bool peeked = kLong && g.tile_major && gwarp == 0 && me.pc.r > lane;
+        unsigned long long early_a = 0, early_b = 0;
+        if (peeked)
+            dev::load_aggregate(p.tile_aggregates + 2 * ((long long)blockIdx.x + (long long)n * gridDim.x), agg_stride,
+                                me.pc.r - lane, early_a, early_b);
         if (!dev::mbarrier_wait(&full_bar[s], ph, &abort_s)) atomicExch(p.counter + 1, 1u);
 
         unsigned char* const stage = smem_raw + s * kStageBytes;
@@ -2029,8 +2063,9 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
             float carry = 0.0f;
             if (me.pc.r > 0) {  // uniform over the group
                 if (gwarp == 0) {
-                    const float c = dev::compose_later_aggregates(p.tile_aggregates + 2 * gtile, me.pc.r,
-                                                                  dev::launch_tag(p.counter), &abort_s);
+                    const float c = dev::compose_later_aggregates(p.tile_aggregates + 2 * gtile, agg_stride, me.pc.r,
+                                                                  dev::launch_tag(p.counter), &abort_s, peeked,
+                                                                  early_a, early_b);
                     if (lane == 0) carry_s[grp] = c;
                 }
                 asm volatile("bar.sync %0, 128;" ::"r"(bar_id) : "memory");
@@ -2169,6 +2204,7 @@ int pick_nt(int width_padded, int n_slabs, size_t budget) {
 
 TileGeometry make_geometry(int64_t B, int64_t T, int nt) {
     TileGeometry g;
+    g.tile_major = 0;
     g.B = B;
     g.T = T;
     if (T <= nt) {
@@ -2295,7 +2331,10 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
     const long long grid = tiles < di->sm_count ? tiles : di->sm_count;
     const int lanes = (S - W) < 4 ? ((S - W) < 1 ? 1 : (S - W)) : 4;  // producer lanes that request tiles side by side
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * NT + 32), smem, stream, p, S, W, lanes));
+    CatParams q = p;
+    // tile-major once every block has a trajectory of its own: the aggregates a tile needs are then a round old
+    q.geo.tile_major = (kLong && p.geo.B >= grid) ? 1 : 0;
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * NT + 32), smem, stream, q, S, W, lanes));
     return IMPACT_OK;
 }
 
@@ -2316,6 +2355,7 @@ int32_t launch_categorical_reg(const CatParams& p, const DeviceInfo* di, cudaStr
     if constexpr (A > 32) {  // no sweeping kernel for wide rows: run_categorical sends long trajectories here only with aggregates
         return launch_categorical_ws<LT, GT, A, false, true>(p, di, stream);
     } else {
+        // with trajectories for every consumer group of the device the sweep inside a block is a little faster still
         if (p.tile_aggregates && p.geo.B < (long long)kWsGroups * di->sm_count)
             return launch_categorical_ws<LT, GT, A, false, true>(p, di, stream);
         auto kernel = impact_loss_categorical_reg_kernel<LT, GT, A>;
@@ -2401,15 +2441,16 @@ int32_t launch_gaussian_ws(const GaussParams& p, const DeviceInfo* di, cudaStrea
     }
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
     const long long grid = tiles < di->sm_count ? tiles : di->sm_count;
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, p, S, W));
+    GaussParams q = p;
+    q.geo.tile_major = (kLong && p.geo.B >= grid) ? 1 : 0;
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, q, S, W));
     return IMPACT_OK;
 }
 
 template <int D>
 int32_t launch_gaussian_reg(const GaussParams& p, const DeviceInfo* di, cudaStream_t stream) {
     if (p.geo.ntiles == 1) return launch_gaussian_ws<D, false>(p, di, stream);
-    if (p.tile_aggregates && p.geo.B < (long long)kWsGroupsGaussian * di->sm_count)
-        return launch_gaussian_ws<D, true>(p, di, stream);
+    if (p.tile_aggregates) return launch_gaussian_ws<D, true>(p, di, stream);
     auto kernel = impact_loss_gaussian_reg_kernel<D>;
     const size_t smem = (size_t)5 * kRegTileRows * D * sizeof(float);
     int grid = 0;
