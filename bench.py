@@ -224,13 +224,13 @@ def run_sweep(args):
             best = ms if best is None else min(best, ms)
         return best
 
-    ws = ip.new_workspace(1, 1)
     targets = [4096 * 4 ** i for i in range(6)]  # 4,096 ... 4,194,304 timesteps
     for A in (6, 18, 64):
         for T in (20, 50, 128):
             for M_target in targets:
                 B = -(-M_target // T)
                 M = B * T
+                ws = ip.new_workspace(B, T)
                 for dtype, name, lb in ((torch.float32, "fp32", 4), (torch.bfloat16, "bf16", 2)):
                     per_step = algorithmic_bytes_per_step(A, lb, lb)
                     foot = per_step * M

@@ -119,8 +119,12 @@ int32_t impact_last_cuda_error(void);
 
 /*
  * Bytes of scratch that impact_loss_fwd_bwd / impact_loss_fwd_bwd_gaussian need for a batch
- * of B x T steps (per-block partial sums and a completion counter).  Returns 0 for
- * non-positive sizes.
+ * of B x T steps: partial sums and counter words (a fixed 193 KB), plus, for trajectories
+ * longer than 64 steps, 16 bytes per 64 steps of every trajectory (the aggregates that link
+ * the tiles of a trajectory that is worked on by several thread blocks at once).  A workspace
+ * with the fixed part only -- impact_loss_workspace_bytes(1, 1) -- serves every batch too: long
+ * trajectories are then swept by one thread block each, which is slower when there are few of
+ * them.  Returns 0 for non-positive sizes.
  */
 size_t impact_loss_workspace_bytes(int64_t B, int64_t T);
 

@@ -1,18 +1,18 @@
 // Device building blocks of the fused IMPACT loss kernels (sm_100a).
 //
 // Work decomposition shared by all loss kernels:
-//   * one thread per time step ("row"); a block of NT threads owns a tile of up to NT
-//     consecutive rows of the row-major [B*T, width] tensors, which is one contiguous slab
-//     of global memory;
-//   * short trajectories (T <= NT) are packed, floor(NT/T) whole trajectories per tile;
-//     long ones (T > NT) are swept tile by tile from their END backwards, because the
-//     advantage recursion runs backward in time -- one scalar carry links the tiles, so
-//     every byte is still read once;
+//   * one thread per time step ("row"); a tile is up to NT consecutive rows of the row-major
+//     [B*T, width] tensors, which is one contiguous slab of global memory;
+//   * short trajectories (T <= NT) are packed, floor(NT/T) whole trajectories per tile; long
+//     ones are cut into tiles that are linked by one scalar (swept from the END backwards inside
+//     one block) or by published affine aggregates (tiles on different blocks) -- either way
+//     every byte is read once;
 //   * slabs reach shared memory by bulk asynchronous copies (one instruction per slab) and
-//     keep their dense layout; the runtime-width Gaussian fallback instead stages them with
-//     16-byte streaming loads into rows of odd stride;
-//   * gradients overwrite the staged rows in place and leave by bulk stores;
-//   * per-block sums are published early and added by the last block to arrive.
+//     keep their dense layout; gradients overwrite the staged rows in place and leave by bulk
+//     stores;
+//   * sums are reduced in a fixed order: per thread, per warp, per block, and across blocks
+//     either by the last block to arrive (ticket) or, in the persistent kernels, by one
+//     collecting group that reads every block's tagged row.
 #pragma once
 
 #include <cuda_bf16.h>
@@ -641,14 +641,6 @@ __device__ __forceinline__ unsigned int publish_block_sums(const float (&acc)[kN
     asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(ticket) : "l"(counter) : "memory");
     return ticket;
 }
-// The ticket alone, for blocks whose row was written by several lanes of the calling warp
-// (with a __syncwarp() between those stores and this call).
-__device__ __forceinline__ unsigned int take_ticket(unsigned int* counter) {
-    unsigned int ticket;
-    asm volatile("atom.add.acq_rel.gpu.global.u32 %0, [%1], 1;" : "=r"(ticket) : "l"(counter) : "memory");
-    return ticket;
-}
-
 // Run by every thread of the block that drew the last ticket: add all blocks' sums in index
 // order (fp64), write the eight loss terms, and leave the counter at 0 for the next launch.
 template <int NT>

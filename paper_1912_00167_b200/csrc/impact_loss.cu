@@ -44,7 +44,7 @@ struct CatParams {
     float* advantage;
     float* partials;
     unsigned int* counter;
-    unsigned long long* tagged_rows;  // persistent kernel: rows of (value, launch tag) pairs, see publish_tagged_row
+    unsigned long long* tagged_rows;  // persistent kernel: rows of (value, launch tag) pairs, see dev::publish_tagged
     unsigned long long* tile_aggregates;  // persistent kernel, T > 128: two (value, launch tag) pairs per tile
     TileGeometry geo;
     LossScalars k;
@@ -332,7 +332,8 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
 }
 
 // ------------------------------------------------------------------------------------------
-// Categorical policy, action count known at compile time (the hot variant)
+// Categorical policy, action count known at compile time: resident blocks that sweep a trajectory
+// (long trajectories, many of them; every other batch goes to the persistent kernel further down)
 // ------------------------------------------------------------------------------------------
 // Same decomposition as the kernel above (128 steps per block, one thread per step), but:
 //   * the two logits slabs of a tile arrive by ONE bulk asynchronous copy each, issued by a
@@ -345,9 +346,7 @@ __global__ void __launch_bounds__(NT) impact_loss_categorical_kernel(const CatPa
 //   * A is a template parameter and every loop is unrolled; rows are streamed pair by pair from
 //     shared memory in each pass, so that few registers are live;
 //   * the softmax runs on exp2 of pre-scaled differences (one multiply + one MUFU each).
-// Five blocks per SM (<= 102 registers, no spills) measured faster than seven at 72 registers,
-// with or without the second stage, even though 740 blocks then walk the 1024 tiles of a
-// B*T = 131072 batch.
+// Five blocks per SM (<= 102 registers, no spills), two slab stages per block.
 template <typename ST, int W> struct RowIO;
 
 // Rows are handled as NP = ceil(W/2) pairs; for odd W the second lane of the last pair is
@@ -2514,7 +2513,7 @@ extern "C" int32_t impact_loss_fwd_bwd(
     if (A > 512) return IMPACT_ERR_UNSUPPORTED;
     if ((double)B * (double)T * (double)A >= 1099511627776.0 || (double)B * (double)T >= 4.0e12)
         return IMPACT_ERR_UNSUPPORTED;
-    if (workspace_bytes < impact_loss_workspace_bytes(B, T)) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
+    if (workspace_bytes < kWorkspaceFixedBytes) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
 
     CatParams p;
     int32_t st = fill_scalars(p.k, rho_bar, c_bar, clip_eps, coef, B, T);
@@ -2540,7 +2539,8 @@ extern "C" int32_t impact_loss_fwd_bwd(
                                                 (size_t)kMaxGridBlocks * 8 * sizeof(float));
     p.tagged_rows = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) +
                                                           (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes);
-    p.tile_aggregates = T > kMinTileRows
+    // room for the tiles' aggregates is optional: without it long trajectories are swept inside one block
+    p.tile_aggregates = (T > kMinTileRows && workspace_bytes >= impact_loss_workspace_bytes(B, T))
                             ? reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWorkspaceFixedBytes)
                             : nullptr;
     p.A = A;
@@ -2579,7 +2579,7 @@ extern "C" int32_t impact_loss_fwd_bwd_gaussian(
     if (D > 256) return IMPACT_ERR_UNSUPPORTED;
     if ((double)B * (double)T * (double)D >= 1099511627776.0 || (double)B * (double)T >= 4.0e12)
         return IMPACT_ERR_UNSUPPORTED;
-    if (workspace_bytes < impact_loss_workspace_bytes(B, T)) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
+    if (workspace_bytes < kWorkspaceFixedBytes) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
 
     GaussParams p;
     int32_t st = fill_scalars(p.k, rho_bar, c_bar, clip_eps, coef, B, T);
@@ -2608,7 +2608,7 @@ extern "C" int32_t impact_loss_fwd_bwd_gaussian(
                                                 (size_t)kMaxGridBlocks * 8 * sizeof(float));
     p.tagged_rows = reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) +
                                                           (size_t)kMaxGridBlocks * 8 * sizeof(float) + kCounterBytes);
-    p.tile_aggregates = T > kRegTileRows
+    p.tile_aggregates = (T > kRegTileRows && workspace_bytes >= impact_loss_workspace_bytes(B, T))
                             ? reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWorkspaceFixedBytes)
                             : nullptr;
     p.D = D;

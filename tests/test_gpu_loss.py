@@ -211,6 +211,29 @@ def test_workspace_is_reusable_across_calls_and_shapes(oracle):
     assert ip.impact_loss_workspace_status(ws) == 0  # no bounded wait ever ran out
 
 
+@pytest.mark.parametrize("B,T,A", [(5, 300, 18), (3, 200, 64)])
+def test_workspace_without_room_for_tile_aggregates(oracle, B, T, A):
+    """The fixed part of the workspace serves long trajectories too (a block then sweeps a trajectory by itself);
+    the result is the same as with the full workspace, and both match the oracle."""
+    import paper_1912_00167_b200 as ip
+    batch = ii.categorical_batch(B, T, A, seed=11 + T, p_done=0.01)
+    h = P.f32_hyper(LossHyper(kl_coef=0.05))
+    ref = oracle.loss_categorical(batch, h)
+    t = {k: torch.from_numpy(v).cuda() for k, v in batch.items()}
+    got = []
+    for ws in (ip.new_workspace(1, 1), ip.new_workspace(B, T)):
+        out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
+                   dvalues=torch.empty(B, T, device="cuda"))
+        ip.impact_loss_fwd_bwd(t["learner_logits"], t["target_logits"], t["worker_logp"], t["actions"], t["rewards"],
+                               t["discounts"], t["values"], t["bootstrap_values"], P.to_coef(h), workspace=ws, **out)
+        torch.cuda.synchronize()
+        got.append(out)
+        np.testing.assert_allclose(out["loss_terms"].cpu().numpy(), ref["loss_terms"], rtol=1e-4, atol=1e-7)
+    assert ip.new_workspace(B, T).numel() > ip.new_workspace(1, 1).numel()
+    M = B * T
+    np.testing.assert_allclose(got[0]["dvalues"].cpu().numpy() * M, got[1]["dvalues"].cpu().numpy() * M, rtol=1e-4, atol=1e-5)
+
+
 def test_rows_of_dlogits_sum_to_zero_at_full_size():
     # softmax invariance: every term of the logit gradient sums to zero over the actions
     import paper_1912_00167_b200 as ip
