@@ -220,6 +220,12 @@ typedef struct impact_loss_call {
     float* advantage;
     void* workspace;
     size_t workspace_bytes;
+    void* target_logits_copy; /* optional (NULL = none): [B,T,A], same type as the logits.  The call also writes
+                                 target_logits there, byte for byte -- the "store the target network's output with
+                                 the batch" of a batch's first traversal (Algorithm 1; impact_buffer_append) done by
+                                 the loss kernel itself, which has the rows in shared memory anyway, instead of by a
+                                 copy of its own.  Typically a slot of the circular buffer
+                                 (impact_buffer_slot_ptr).  Must not overlap any other argument. */
 } impact_loss_call;
 
 /* impact_loss_fwd_bwd with its arguments taken from `call` (Algorithm 1, gradient step). */

@@ -58,7 +58,8 @@ class impact_loss_call(ctypes.Structure):
                 ("logits_dtype", ctypes.c_int32), ("coef", impact_coefficients), ("A", ctypes.c_int32),
                 ("B", ctypes.c_int64), ("T", ctypes.c_int64), ("loss_terms", ctypes.c_void_p),
                 ("dlogits", ctypes.c_void_p), ("dvalues", ctypes.c_void_p), ("vtarget", ctypes.c_void_p),
-                ("advantage", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t)]
+                ("advantage", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
+                ("target_logits_copy", ctypes.c_void_p)]
 
 
 _lib = None
@@ -234,7 +235,7 @@ class PreparedCall:
 
 def prepare_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
                          bootstrap_values, coef: Coefficients, *, loss_terms, dlogits, dvalues,
-                         vtarget=None, advantage=None, workspace) -> PreparedCall:
+                         vtarget=None, advantage=None, workspace, target_logits_copy=None) -> PreparedCall:
     lib = load_library()
     B, T, A = learner_logits.shape
     ldt = learner_logits.dtype
@@ -251,17 +252,19 @@ def prepare_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, re
         _dev(loss_terms, f32, (NUM_TERMS,), "loss_terms"), _dev(dlogits, dlogits.dtype, (B, T, A), "dlogits"),
         _dev(dvalues, f32, bt, "dvalues"), _dev(vtarget, f32, bt, "vtarget", True),
         _dev(advantage, f32, bt, "advantage", True),
-        _dev(workspace, torch.uint8, workspace.shape, "workspace"), workspace.numel())
+        _dev(workspace, torch.uint8, workspace.shape, "workspace"), workspace.numel(),
+        _dev(target_logits_copy, ldt, (B, T, A), "target_logits_copy", True))
     return PreparedCall(lib.impact_loss_fwd_bwd_call, [ctypes.byref(call), 0], "impact_loss_fwd_bwd_call", (call,))
 
 
 def impact_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
                         bootstrap_values, coef: Coefficients, *, loss_terms, dlogits, dvalues,
-                        vtarget=None, advantage=None, workspace, stream=None) -> None:
+                        vtarget=None, advantage=None, workspace, target_logits_copy=None, stream=None) -> None:
     """Enqueues the categorical IMPACT loss + gradients on `stream` (see include/impact.h)."""
     prepare_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
                          bootstrap_values, coef, loss_terms=loss_terms, dlogits=dlogits, dvalues=dvalues,
-                         vtarget=vtarget, advantage=advantage, workspace=workspace)(stream)
+                         vtarget=vtarget, advantage=advantage, workspace=workspace,
+                         target_logits_copy=target_logits_copy)(stream)
 
 
 def impact_loss_fwd_bwd_static_scratch(learner_logits, target_logits, worker_logp, actions, rewards, discounts,

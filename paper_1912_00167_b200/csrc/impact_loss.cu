@@ -46,6 +46,7 @@ struct CatParams {
     unsigned int* counter;
     unsigned long long* tagged_rows;  // persistent kernel: rows of (value, launch tag) pairs, see dev::publish_tagged
     unsigned long long* tile_aggregates;  // persistent kernel, T > 128: two (value, launch tag) pairs per tile
+    void* target_copy;  // persistent kernel: where the target logits are written as well (NULL = nowhere)
     TileGeometry geo;
     LossScalars k;
     int A, As;
@@ -1187,6 +1188,21 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         unsigned char* const s0 = smem_raw + s * kStageBytes;  // learner logits
         unsigned char* const s1 = s0 + NT * kInRow;             // target logits
         unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : s0 + 2 * NT * kInRow;
+        // (first traversal of a batch) the target rows go to the circular buffer as well, each warp's 32 rows by a
+        // bulk store straight from the stage, which nothing writes to
+        if (p.target_copy) {
+            const int left = me.pc.nrows - (gtid - lane);
+            const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
+            LT* const dst = static_cast<LT*>(p.target_copy) + (me.row - lane) * A;
+            const unsigned char* const src = s1 + (gtid - lane) * kInRow;
+            const uint32_t bytes = (uint32_t)wrows * kInRow;
+            if (((reinterpret_cast<uintptr_t>(dst) | bytes) & 15u) == 0) {
+                if (lane == 0 && bytes) dev::bulk_store(dst, src, bytes);
+            } else {
+                const int nelem = wrows * A;
+                for (int i = lane; i < nelem; i += 32) dst[i] = reinterpret_cast<const LT*>(src)[i];
+            }
+        }
         const int a = cur.a;
         dev::StepIn st;
         st.l_worker = cur.l_worker;
@@ -2293,6 +2309,15 @@ int32_t dispatch_nt(const CatParams& p, int nt, const DeviceInfo* di, cudaStream
     }
 }
 
+// The copy of the target logits for the kernels that do not write it themselves: an ordinary device copy ahead
+// of the launch.
+int32_t copy_target_logits(const CatParams& p, size_t elem, cudaStream_t stream) {
+    if (!p.target_copy) return IMPACT_OK;
+    const size_t bytes = (size_t)p.geo.B * (size_t)p.geo.T * (size_t)p.A * elem;
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(p.target_copy, p.target_logits, bytes, cudaMemcpyDeviceToDevice, stream));
+    return IMPACT_OK;
+}
+
 // Tiles the producer keeps in flight and stages of the ring, for tiles of `tile_in_bytes` bytes of logits:
 // about 48 KB per SM on the way (enough, over 148 SMs, to cover HBM's latency at full bandwidth; more
 // only delays the first tiles), and room beyond that for the tiles being worked on and being stored.
@@ -2362,6 +2387,8 @@ int32_t launch_categorical_reg(const CatParams& p, const DeviceInfo* di, cudaStr
         int grid = 0;
         int32_t st = grid_for(kernel, kRegTileRows, smem, p.geo.nchunks, di, &grid);
         if (st != IMPACT_OK) return st;
+        st = copy_target_logits(p, sizeof(LT), stream);  // this kernel does not write the copy itself
+        if (st != IMPACT_OK) return st;
         IMPACT_CUDA_TRY(launch_serialized(kernel, dim3(grid), dim3(kRegTileRows), smem, stream, p));
         return IMPACT_OK;
     }
@@ -2405,6 +2432,10 @@ int32_t run_categorical(CatParams& p, int64_t B, int64_t T, bool logits_bf16, bo
     p.As = p.A;
     const int nt = categorical_tile_rows(p.A, logits_bf16, grads_bf16, long_without_aggregates);
     p.geo = make_geometry(B, T, nt);
+    {
+        const int32_t st = copy_target_logits(p, logits_bf16 ? 2 : 4, s);  // the runtime-width kernel does not write it
+        if (st != IMPACT_OK) return st;
+    }
     if (!logits_bf16 && !grads_bf16) return dispatch_nt<float, float>(p, nt, di, s);
     if (!logits_bf16 && grads_bf16) return dispatch_nt<float, __nv_bfloat16>(p, nt, di, s);
     if (logits_bf16 && !grads_bf16) return dispatch_nt<__nv_bfloat16, float>(p, nt, di, s);
@@ -2491,13 +2522,13 @@ extern "C" int32_t impact_loss_workspace_status(const void* workspace, size_t wo
     return IMPACT_OK;
 }
 
-extern "C" int32_t impact_loss_fwd_bwd(
+static int32_t loss_fwd_bwd_impl(
     const void* learner_logits, const void* target_logits, const float* worker_logp,
     const int32_t* actions, const float* rewards, const float* discounts, const float* values,
     const float* bootstrap_values, float rho_bar, float c_bar, float clip_eps,
     const impact_coefficients* coef, int64_t B, int64_t T, int32_t A, int32_t logits_dtype,
     float* loss_terms, void* dlogits, float* dvalues, float* vtarget, float* advantage,
-    void* workspace, size_t workspace_bytes, void* stream) {
+    void* workspace, size_t workspace_bytes, void* target_logits_copy, void* stream) {
     if (!learner_logits || !target_logits || !worker_logp || !actions || !rewards || !discounts ||
         !values || !bootstrap_values || !coef || !loss_terms || !dlogits || !dvalues || !workspace)
         return IMPACT_ERR_INVALID_ARG;
@@ -2507,6 +2538,8 @@ extern "C" int32_t impact_loss_fwd_bwd(
     for (const void* q : ptrs)
         if (!aligned16(q)) return IMPACT_ERR_INVALID_ARG;
     if ((vtarget && !aligned16(vtarget)) || (advantage && !aligned16(advantage))) return IMPACT_ERR_INVALID_ARG;
+    if (target_logits_copy && (!aligned16(target_logits_copy) || target_logits_copy == target_logits))
+        return IMPACT_ERR_INVALID_ARG;
     if (logits_dtype != IMPACT_DTYPE_F32 && logits_dtype != IMPACT_DTYPE_BF16) return IMPACT_ERR_INVALID_ARG;
     if (coef->dlogits_dtype != IMPACT_DTYPE_F32 && coef->dlogits_dtype != IMPACT_DTYPE_BF16)
         return IMPACT_ERR_INVALID_ARG;
@@ -2543,17 +2576,31 @@ extern "C" int32_t impact_loss_fwd_bwd(
     p.tile_aggregates = (T > kMinTileRows && workspace_bytes >= impact_loss_workspace_bytes(B, T))
                             ? reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWorkspaceFixedBytes)
                             : nullptr;
+    p.target_copy = target_logits_copy;
     p.A = A;
     return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
                            di, static_cast<cudaStream_t>(stream));
 }
 
+extern "C" int32_t impact_loss_fwd_bwd(
+    const void* learner_logits, const void* target_logits, const float* worker_logp,
+    const int32_t* actions, const float* rewards, const float* discounts, const float* values,
+    const float* bootstrap_values, float rho_bar, float c_bar, float clip_eps,
+    const impact_coefficients* coef, int64_t B, int64_t T, int32_t A, int32_t logits_dtype,
+    float* loss_terms, void* dlogits, float* dvalues, float* vtarget, float* advantage,
+    void* workspace, size_t workspace_bytes, void* stream) {
+    return loss_fwd_bwd_impl(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
+                             bootstrap_values, rho_bar, c_bar, clip_eps, coef, B, T, A, logits_dtype, loss_terms,
+                             dlogits, dvalues, vtarget, advantage, workspace, workspace_bytes, nullptr, stream);
+}
+
 extern "C" int32_t impact_loss_fwd_bwd_call(const impact_loss_call* c, void* stream) {
     if (!c) return IMPACT_ERR_INVALID_ARG;
-    return impact_loss_fwd_bwd(c->learner_logits, c->target_logits, c->worker_logp, c->actions, c->rewards,
-                               c->discounts, c->values, c->bootstrap_values, c->rho_bar, c->c_bar, c->clip_eps,
-                               &c->coef, c->B, c->T, c->A, c->logits_dtype, c->loss_terms, c->dlogits,
-                               c->dvalues, c->vtarget, c->advantage, c->workspace, c->workspace_bytes, stream);
+    return loss_fwd_bwd_impl(c->learner_logits, c->target_logits, c->worker_logp, c->actions, c->rewards,
+                             c->discounts, c->values, c->bootstrap_values, c->rho_bar, c->c_bar, c->clip_eps,
+                             &c->coef, c->B, c->T, c->A, c->logits_dtype, c->loss_terms, c->dlogits,
+                             c->dvalues, c->vtarget, c->advantage, c->workspace, c->workspace_bytes,
+                             c->target_logits_copy, stream);
 }
 
 extern "C" int32_t impact_loss_fwd_bwd_gaussian(
@@ -2723,6 +2770,7 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     p.counter = reinterpret_cast<unsigned int*>(counter);
     p.tagged_rows = reinterpret_cast<unsigned long long*>(counter + kCounterBytes);
     p.tile_aggregates = nullptr;  // long trajectories are swept tile by tile inside a block
+    p.target_copy = nullptr;
     // the same kernels, chosen the same way, as impact_loss_fwd_bwd
     return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
                            di, s);

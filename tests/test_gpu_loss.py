@@ -234,6 +234,34 @@ def test_workspace_without_room_for_tile_aggregates(oracle, B, T, A):
     np.testing.assert_allclose(got[0]["dvalues"].cpu().numpy() * M, got[1]["dvalues"].cpu().numpy() * M, rtol=1e-4, atol=1e-5)
 
 
+@pytest.mark.parametrize("B,T,A,dtype", [(1024, 128, 18, torch.float32), (37, 50, 18, torch.float32),
+                                         (5, 300, 18, torch.float32), (700, 200, 6, torch.float32),
+                                         (4, 33, 5, torch.float32), (40, 128, 18, torch.bfloat16),
+                                         (9, 100, 64, torch.float32), (301, 21, 9, torch.bfloat16)])
+def test_target_logits_are_copied_out_by_the_loss_call(B, T, A, dtype):
+    """First traversal of a batch: the call also stores the target logits (into a slot of the circular buffer, in
+    a learner loop).  The copy is bit-exact, whichever kernel serves the shape, and nothing else changes."""
+    import paper_1912_00167_b200 as ip
+    batch = ii.categorical_batch(B, T, A, seed=21 + B + A, p_done=0.01)
+    t = {k: torch.from_numpy(v).cuda() for k, v in batch.items()}
+    zl, zt = t["learner_logits"].to(dtype), t["target_logits"].to(dtype)
+    coef = ip.Coefficients(clip_eps=0.3, kl_coef=0.0)
+    outs = []
+    for with_copy in (False, True):
+        out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda", dtype=dtype),
+                   dvalues=torch.empty(B, T, device="cuda"))
+        copy = torch.full((B, T, A), -7.0, device="cuda", dtype=dtype) if with_copy else None
+        ip.impact_loss_fwd_bwd(zl, zt, t["worker_logp"], t["actions"], t["rewards"], t["discounts"], t["values"],
+                               t["bootstrap_values"], coef, workspace=ip.new_workspace(B, T), target_logits_copy=copy,
+                               **out)
+        torch.cuda.synchronize()
+        outs.append(out)
+        if with_copy:
+            assert torch.equal(copy.view(torch.uint8), zt.view(torch.uint8))
+    for k in ("loss_terms", "dlogits", "dvalues"):
+        assert torch.equal(outs[0][k], outs[1][k])
+
+
 def test_rows_of_dlogits_sum_to_zero_at_full_size():
     # softmax invariance: every term of the logit gradient sums to zero over the actions
     import paper_1912_00167_b200 as ip
