@@ -12,4 +12,5 @@ from .binding import (  # noqa: F401
     prepare_loss_fwd_bwd_gaussian,
 )
 from . import binding  # noqa: F401
+from .kl_controller import AdaptiveKL  # noqa: F401
 from .sharded import impact_loss_fwd_bwd_sharded, reduce_loss_terms, shard_bounds  # noqa: F401
