@@ -2353,7 +2353,8 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
         configured_device = di->device;
     }
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
-    const long long grid = tiles < di->sm_count ? tiles : di->sm_count;
+    long long grid = tiles < di->sm_count ? tiles : di->sm_count;
+    if (grid > kMaxTaggedRows) grid = kMaxTaggedRows;  // one tagged row per block
     const int lanes = (S - W) < 4 ? ((S - W) < 1 ? 1 : (S - W)) : 4;  // producer lanes that request tiles side by side
     CatParams q = p;
     // tile-major once every block has a trajectory of its own: the aggregates a tile needs are then a round old
@@ -2470,7 +2471,8 @@ int32_t launch_gaussian_ws(const GaussParams& p, const DeviceInfo* di, cudaStrea
         configured_device = di->device;
     }
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
-    const long long grid = tiles < di->sm_count ? tiles : di->sm_count;
+    long long grid = tiles < di->sm_count ? tiles : di->sm_count;
+    if (grid > kMaxTaggedRows) grid = kMaxTaggedRows;  // one tagged row per block
     GaussParams q = p;
     q.geo.tile_major = (kLong && p.geo.B >= grid) ? 1 : 0;
     IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, q, S, W));
