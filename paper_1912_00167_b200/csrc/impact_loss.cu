@@ -813,6 +813,38 @@ __global__ void __launch_bounds__(kRegTileRows, 5) impact_loss_categorical_reg_k
 // stage) says it may be refilled.  Every wait is bounded; a wait that gives up raises the
 // workspace's error word and the block's abort flag, after which nobody waits any more and
 // the block runs to its end on whatever the stages hold.
+// Where the n-th tile of a block of a persistent kernel sits: first row, rows, first trajectory, and (long
+// trajectories) the tile's number counted from its trajectory's end.
+struct Place {
+    long long row0, traj;
+    int nrows, r;
+};
+template <bool kLong, int NT>
+__device__ __forceinline__ Place tile_place(const TileGeometry& g, int n, int rows_full, long long total_rows) {
+    Place pl;
+    const long long gt_ = (long long)blockIdx.x + (long long)n * gridDim.x;
+    if (kLong) {
+        if (g.tile_major) {  // the last tiles of all trajectories first, then the tiles before them, ...
+            pl.r = (int)((unsigned long long)gt_ / (unsigned long long)g.B);
+            pl.traj = gt_ - (long long)pl.r * g.B;
+        } else {  // trajectory by trajectory, each from its last tile backwards
+            pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
+            pl.r = (int)(gt_ - pl.traj * g.ntiles);
+        }
+        const long long t0 = (long long)(g.ntiles - 1 - pl.r) * NT;
+        const long long left = g.T - t0;
+        pl.nrows = left < NT ? (int)left : NT;
+        pl.row0 = pl.traj * g.T + t0;
+    } else {
+        pl.row0 = gt_ * rows_full;
+        pl.traj = gt_ * g.G;
+        const long long left = total_rows - pl.row0;
+        pl.nrows = left < rows_full ? (int)left : rows_full;
+        pl.r = 0;
+    }
+    return pl;
+}
+
 template <typename LT, typename GT, int A, int NT>
 __host__ __device__ constexpr size_t ws_stage_bytes() {
     constexpr size_t in_row = A * sizeof(LT), out_row = A * sizeof(GT);
@@ -913,35 +945,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     const int rows_full = kLong ? NT : g.G * (int)g.T;                                   // rows of a full tile
     const long long total_rows = g.B * g.T;
     const long long agg_stride = g.tile_major ? 2 * g.B : 2;  // slots between a tile's aggregate and that of the tile after it in time
-    // where the block's n-th tile sits: first row, rows, and (kLong) trajectory and tile number from its end
-    struct Place {
-        long long row0, traj;
-        int nrows, r;
-    };
-    auto place_of = [&](int n) {
-        Place pl;
-        const long long gt_ = (long long)blockIdx.x + (long long)n * gridDim.x;
-        if (kLong) {
-            if (g.tile_major) {  // the last tiles of all trajectories first, then the tiles before them, ...
-                pl.r = (int)((unsigned long long)gt_ / (unsigned long long)g.B);
-                pl.traj = gt_ - (long long)pl.r * g.B;
-            } else {  // trajectory by trajectory, each from its last tile backwards
-                pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
-                pl.r = (int)(gt_ - pl.traj * g.ntiles);
-            }
-            const long long t0 = (long long)(g.ntiles - 1 - pl.r) * NT;
-            const long long left = g.T - t0;
-            pl.nrows = left < NT ? (int)left : NT;
-            pl.row0 = pl.traj * g.T + t0;
-        } else {
-            pl.row0 = gt_ * rows_full;
-            pl.traj = gt_ * g.G;
-            const long long left = total_rows - pl.row0;
-            pl.nrows = left < rows_full ? (int)left : rows_full;
-            pl.r = 0;
-        }
-        return pl;
-    };
+    auto place_of = [&](int n) { return tile_place<kLong, NT>(g, n, rows_full, total_rows); };
 
     if (tid >= C * NT) {
         // ---- producer warp ----------------------------------------------------------------------------------
@@ -1054,38 +1058,9 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             }
         }
         __syncwarp();
-        // ---- then it publishes the block's sums, once every group's are final: one row of (value, tag)
-        // pairs, the tag being this launch's number.  A pair is one 8-byte store, so whoever reads the tag of
-        // this launch reads this launch's value with it: no fence, no atomic, no round trip.  The groups'
-        // barriers are polled without blocking and their sums added in group order, whatever order they
-        // arrive in.
-        const unsigned int tag = dev::launch_tag(p.counter);
-        float yc[C];
-        unsigned int todo = (1u << C) - 1u;
-        for (unsigned int spin = 0; todo != 0u && spin < (1u << 24); ++spin) {
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                if (!(todo & (1u << c))) continue;
-                bool ready = (lane == 0) && dev::mbarrier_test(&sums_bar[c], 0u);
-                ready = __shfl_sync(0xffffffffu, ready, 0);
-                if (!ready) continue;
-                float y = 0.0f;
-#pragma unroll
-                for (int w = 0; w < NT / 32; ++w) y += red[c][w][lane & 7];
-                yc[c] = y;
-                todo &= ~(1u << c);
-            }
-            if (*reinterpret_cast<volatile int*>(&abort_s)) break;
-            if (n_tiles > kWsFewTiles) __nanosleep(64);  // a long launch: leave the issue slots to the consumers
-        }
-        if (todo == 0u) {
-            float y = yc[0];
-#pragma unroll
-            for (int c = 1; c < C; ++c) y += yc[c];
-            if (lane < 8) dev::publish_tagged(p.tagged_rows + (size_t)blockIdx.x * 8 + lane, y, tag);
-        } else if (lane == 0) {
+        // ---- then it publishes the block's sums, once every group's are final
+        if (!dev::publish_block_row<C, NT>(sums_bar, red, &abort_s, p.counter, p.tagged_rows, n_tiles > kWsFewTiles) && lane == 0)
             atomicExch(p.counter + 1, 1u);  // a group never delivered its sums
-        }
         return;
     }
 
@@ -1139,17 +1114,8 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     // The group's sums, once final: a butterfly per warp into `red`, then one arrival per warp tells the
     // producer warp that the row can be published (fixed order throughout).
     auto hand_over_sums = [&]() {
-        const float x = dev::warp_sum4(t_surr, t_val, t_ent, t_ratio);
-        const float xk = want_kl ? dev::warp_sum(t_kl) : 0.0f;
-        if ((lane & 7) == 0) red[grp][gwarp][lane == 24 ? 6 : (lane >> 3)] = x;
-        if (lane == 0) {
-            red[grp][gwarp][3] = xk;
-            red[grp][gwarp][4] = (float)n_clip;
-            red[grp][gwarp][5] = (float)n_trunc;
-            red[grp][gwarp][7] = 0.0f;
-        }
-        __syncwarp();
-        if (lane == 0) dev::mbarrier_arrive(&sums_bar[grp]);
+        dev::hand_over_group_sums(t_surr, t_val, t_ent, t_ratio, t_kl, want_kl, n_clip, n_trunc, red[grp][gwarp],
+                                  &sums_bar[grp]);
     };
     bool pending = false;  // lane 0 of each warp: a store of this warp may still be reading its stage
     int pending_stage = 0;
@@ -1804,34 +1770,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     const int rows_full = kLong ? NT : g.G * (int)g.T;
     const long long total_rows = g.B * g.T;
     const long long agg_stride = g.tile_major ? 2 * g.B : 2;  // slots between a tile's aggregate and that of the tile after it in time
-    struct Place {
-        long long row0, traj;
-        int nrows, r;
-    };
-    auto place_of = [&](int n) {
-        Place pl;
-        const long long gt_ = (long long)blockIdx.x + (long long)n * gridDim.x;
-        if (kLong) {
-            if (g.tile_major) {  // the last tiles of all trajectories first, then the tiles before them, ...
-                pl.r = (int)((unsigned long long)gt_ / (unsigned long long)g.B);
-                pl.traj = gt_ - (long long)pl.r * g.B;
-            } else {  // trajectory by trajectory, each from its last tile backwards
-                pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
-                pl.r = (int)(gt_ - pl.traj * g.ntiles);
-            }
-            const long long t0 = (long long)(g.ntiles - 1 - pl.r) * NT;
-            const long long left = g.T - t0;
-            pl.nrows = left < NT ? (int)left : NT;
-            pl.row0 = pl.traj * g.T + t0;
-        } else {
-            pl.row0 = gt_ * rows_full;
-            pl.traj = gt_ * g.G;
-            const long long left = total_rows - pl.row0;
-            pl.nrows = left < rows_full ? (int)left : rows_full;
-            pl.r = 0;
-        }
-        return pl;
-    };
+    auto place_of = [&](int n) { return tile_place<kLong, NT>(g, n, rows_full, total_rows); };
 
     if (tid >= C * NT) {
         // ---- producer warp ----------------------------------------------------------------------------------
@@ -1905,34 +1844,9 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
             }
         }
         __syncwarp();
-        // the block's sums, once every group's are final: one tagged row (see the categorical kernel)
-        const unsigned int tag = dev::launch_tag(p.counter);
-        float yc[C];
-        unsigned int todo = (1u << C) - 1u;
-        for (unsigned int spin = 0; todo != 0u && spin < (1u << 24); ++spin) {
-#pragma unroll
-            for (int c = 0; c < C; ++c) {
-                if (!(todo & (1u << c))) continue;
-                bool ready = (lane == 0) && dev::mbarrier_test(&sums_bar[c], 0u);
-                ready = __shfl_sync(0xffffffffu, ready, 0);
-                if (!ready) continue;
-                float y = 0.0f;
-#pragma unroll
-                for (int w = 0; w < NT / 32; ++w) y += red[c][w][lane & 7];
-                yc[c] = y;
-                todo &= ~(1u << c);
-            }
-            if (*reinterpret_cast<volatile int*>(&abort_s)) break;
-            __nanosleep(64);
-        }
-        if (todo == 0u) {
-            float y = yc[0];
-#pragma unroll
-            for (int c = 1; c < C; ++c) y += yc[c];
-            if (lane < 8) dev::publish_tagged(p.tagged_rows + (size_t)blockIdx.x * 8 + lane, y, tag);
-        } else if (lane == 0) {
+        // the block's sums, once every group's are final
+        if (!dev::publish_block_row<C, NT>(sums_bar, red, &abort_s, p.counter, p.tagged_rows, n_tiles > kWsFewTiles) && lane == 0)
             atomicExch(p.counter + 1, 1u);
-        }
         return;
     }
 
@@ -1978,17 +1892,8 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     float t_surr = 0.0f, t_val = 0.0f, t_ent = 0.0f, t_ratio = 0.0f, t_kl = 0.0f;
     int n_clip = 0, n_trunc = 0;
     auto hand_over_sums = [&]() {
-        const float x = dev::warp_sum4(t_surr, t_val, t_ent, t_ratio);
-        const float xk = want_kl ? dev::warp_sum(t_kl) : 0.0f;
-        if ((lane & 7) == 0) red[grp][gwarp][lane == 24 ? 6 : (lane >> 3)] = x;
-        if (lane == 0) {
-            red[grp][gwarp][3] = xk;
-            red[grp][gwarp][4] = (float)n_clip;
-            red[grp][gwarp][5] = (float)n_trunc;
-            red[grp][gwarp][7] = 0.0f;
-        }
-        __syncwarp();
-        if (lane == 0) dev::mbarrier_arrive(&sums_bar[grp]);
+        dev::hand_over_group_sums(t_surr, t_val, t_ent, t_ratio, t_kl, want_kl, n_clip, n_trunc, red[grp][gwarp],
+                                  &sums_bar[grp]);
     };
     bool pending = false;
     int pending_stage = 0;
