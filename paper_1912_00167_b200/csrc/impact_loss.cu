@@ -2224,12 +2224,12 @@ int32_t copy_target_logits(const CatParams& p, size_t elem, cudaStream_t stream)
 }
 
 // Tiles the producer keeps in flight and stages of the ring, for tiles of `tile_in_bytes` bytes of logits:
-// about 48 KB per SM on the way (enough, over 148 SMs, to cover HBM's latency at full bandwidth; more
+// about 64 KB per SM on the way (enough, over 148 SMs, to cover HBM's latency at full bandwidth; more
 // only delays the first tiles), and room beyond that for the tiles being worked on and being stored.
 void ws_ring_shape(size_t stage_bytes, size_t tile_in_bytes, int groups, int max_smem, int* stages, int* in_flight) {
-    int w = (int)((48 * 1024 + tile_in_bytes - 1) / tile_in_bytes);
+    int w = (int)((64 * 1024 + tile_in_bytes - 1) / tile_in_bytes);
     if (w < 2) w = 2;
-    if (w > 12) w = 12;
+    if (w > 8) w = 8;
     int s = w + groups + 3;
     if (s > kWsMaxStages) s = kWsMaxStages;
     const int fit = (int)((size_t)(max_smem - 4096) / stage_bytes);  // 4 KB left for static shared memory
@@ -2251,6 +2251,7 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     int S = 0, W = 0;
     ws_ring_shape(stage, 2 * (size_t)NT * A * sizeof(LT), C, di->max_smem_optin, &S, &W);
     if (S < 2) return IMPACT_ERR_UNSUPPORTED;
+
     const size_t smem = (size_t)S * stage;
     static thread_local int configured_device = -1;
     if (configured_device != di->device) {
