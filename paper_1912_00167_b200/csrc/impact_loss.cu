@@ -1039,10 +1039,17 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
                 const int cyc = n / S, s = n - cyc * S;
                 const int wcyc = (n - W) / S, ws = (n - W) - wcyc * S;
                 for (unsigned int spin = 0; spin < (1u << 22); ++spin) {
-                    if (pending && (cyc == 0 || dev::mbarrier_test(&empty_bar[s], (uint32_t)(cyc - 1) & 1u)) &&
-                        dev::mbarrier_test(&full_bar[ws], (uint32_t)wcyc & 1u)) {
-                        send_tile(n, s);
-                        pending = false;
+                    const bool ready = pending && (cyc == 0 || dev::mbarrier_test(&empty_bar[s], (uint32_t)(cyc - 1) & 1u)) &&
+                                       dev::mbarrier_test(&full_bar[ws], (uint32_t)wcyc & 1u);
+                    // the requests themselves leave one lane at a time: a bulk copy is issued from a warp-wide
+                    // (uniform) datapath, and several lanes inside it at once lost requests at four lanes with
+                    // four tiles in flight
+                    for (int l = 0; l < lanes; ++l) {
+                        if (lane == l && ready) {
+                            send_tile(n, s);
+                            pending = false;
+                        }
+                        __syncwarp();
                     }
                     if (!__any_sync(0xffffffffu, pending)) break;
                     if (*reinterpret_cast<volatile int*>(&abort_s)) break;
@@ -2224,10 +2231,10 @@ int32_t copy_target_logits(const CatParams& p, size_t elem, cudaStream_t stream)
 }
 
 // Tiles the producer keeps in flight and stages of the ring, for tiles of `tile_in_bytes` bytes of logits:
-// about 64 KB per SM on the way (enough, over 148 SMs, to cover HBM's latency at full bandwidth; more
+// about 48 KB per SM on the way (enough, over 148 SMs, to cover HBM's latency at full bandwidth; more
 // only delays the first tiles), and room beyond that for the tiles being worked on and being stored.
 void ws_ring_shape(size_t stage_bytes, size_t tile_in_bytes, int groups, int max_smem, int* stages, int* in_flight) {
-    int w = (int)((64 * 1024 + tile_in_bytes - 1) / tile_in_bytes);
+    int w = (int)((48 * 1024 + tile_in_bytes - 1) / tile_in_bytes);
     if (w < 2) w = 2;
     if (w > 8) w = 8;
     int s = w + groups + 3;
@@ -2251,6 +2258,7 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     int S = 0, W = 0;
     ws_ring_shape(stage, 2 * (size_t)NT * A * sizeof(LT), C, di->max_smem_optin, &S, &W);
     if (S < 2) return IMPACT_ERR_UNSUPPORTED;
+
 
     const size_t smem = (size_t)S * stage;
     static thread_local int configured_device = -1;

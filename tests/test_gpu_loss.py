@@ -262,6 +262,33 @@ def test_target_logits_are_copied_out_by_the_loss_call(B, T, A, dtype):
         assert torch.equal(outs[0][k], outs[1][k])
 
 
+@pytest.mark.parametrize("B,T,A", [(32768, 128, 18), (32768, 128, 6)])
+def test_no_wait_runs_out_in_long_launches(B, T, A):
+    """Hundreds of tiles per block: every bounded wait of the persistent kernel must end by itself (the workspace's
+    error word stays 0), launch after launch on the same workspace, and the launches agree bit for bit."""
+    import paper_1912_00167_b200 as ip
+    g = torch.Generator(device="cuda").manual_seed(3)
+    zl = torch.randn(B, T, A, device="cuda", generator=g)
+    zt = zl + 0.1 * torch.randn(B, T, A, device="cuda", generator=g)
+    act = torch.randint(0, A, (B, T), device="cuda", generator=g, dtype=torch.int32)
+    wl = torch.log_softmax(zl, -1).gather(-1, act.long().unsqueeze(-1)).squeeze(-1).contiguous()
+    rew = (torch.rand(B, T, device="cuda", generator=g) < 0.05).float()
+    dis = torch.where(torch.rand(B, T, device="cuda", generator=g) < 0.005, 0.0, 0.99).float()
+    val, boot = torch.randn(B, T, device="cuda", generator=g), torch.randn(B, device="cuda", generator=g)
+    ws = ip.new_workspace(B, T)
+    outs = []
+    for _ in range(6):
+        out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
+                   dvalues=torch.empty(B, T, device="cuda"))
+        ip.impact_loss_fwd_bwd(zl, zt, wl, act, rew, dis, val, boot, ip.Coefficients(clip_eps=0.4), workspace=ws, **out)
+        outs.append(out["loss_terms"].clone())
+    torch.cuda.synchronize()
+    assert ip.impact_loss_workspace_status(ws) == 0
+    assert torch.isfinite(outs[0]).all()
+    for o in outs[1:]:
+        assert torch.equal(o, outs[0])
+
+
 def test_rows_of_dlogits_sum_to_zero_at_full_size():
     # softmax invariance: every term of the logit gradient sums to zero over the actions
     import paper_1912_00167_b200 as ip
