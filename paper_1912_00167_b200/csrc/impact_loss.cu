@@ -1005,9 +1005,12 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
                 dev::mbarrier_arrive(&full_bar[s]);
             }
         };
-        // the first W tiles need no wait (tile n goes to stage n), and leave, a lane each, before the rest of the
-        // block has even started
-        if (lane < n_first) send_tile(lane, lane);
+        // the first W tiles need no wait (tile n goes to stage n), and leave before the rest of the block has even
+        // started: prepared a lane each, issued one lane at a time (see below)
+        for (int l = 0; l < n_first; ++l) {
+            if (lane == l) send_tile(l, l);
+            __syncwarp();
+        }
         __syncthreads();  // the barriers are set up: the consumer warps may use them
         // The rest.  Tile n goes to stage n % S once that stage's previous tile has left (the "empty" phase
         // before this one) and tile n - W has landed (at most W tiles in flight).
