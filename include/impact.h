@@ -29,7 +29,7 @@
 extern "C" {
 #endif
 
-#define IMPACT_VERSION 200 /* major*10000 + minor*100 + patch */
+#define IMPACT_VERSION 300 /* major*10000 + minor*100 + patch */
 
 /* ---- status codes -------------------------------------------------------------------- */
 #define IMPACT_OK 0
@@ -114,6 +114,29 @@ int32_t impact_version(void);
 const char* impact_status_string(int32_t status);
 /* cudaError_t value of the most recent CUDA failure seen by this thread's calls (0 if none). */
 int32_t impact_last_cuda_error(void);
+
+/*
+ * Launch options of the loss calls: process-wide performance knobs with working defaults; none changes a
+ * result.  (The paper prescribes no kernel design, so these have no counterpart there.)  A value set here is
+ * used by every later loss call of the process; setting one while another thread is inside a loss call is safe
+ * (that call uses the old or the new value).
+ *   IMPACT_OPT_EARLY_PREFETCH  1 (default): a loss call on a batch of at least a few megabytes enqueues a
+ *       one-warp-per-block companion kernel right before its loss kernel.  The companion runs beside whatever
+ *       kernel is still busy on the stream, asks L2 for the batch's first tiles, and then waits for the stream's
+ *       previous kernel, so stream order is kept exactly; the loss kernel finds its first tiles in L2 instead of
+ *       waiting for HBM.  0: no companion; the loss kernel asks for its first tiles itself when it starts.
+ *   IMPACT_OPT_PREFETCH_BYTES  upper bound on the bytes one call asks L2 for ahead of time (default 48 MiB).
+ *   IMPACT_OPT_WINDOW_BYTES    bytes of tiles a block keeps in flight from global to shared memory (default
+ *       72 KiB; 16 KiB .. 160 KiB).
+ * impact_set_option returns IMPACT_ERR_INVALID_ARG for an unknown option or a value out of range;
+ * impact_get_option returns -1 for an unknown option.
+ */
+#define IMPACT_OPT_EARLY_PREFETCH 0
+#define IMPACT_OPT_PREFETCH_BYTES 1
+#define IMPACT_OPT_WINDOW_BYTES 2
+#define IMPACT_NUM_OPTIONS 3
+int32_t impact_set_option(int32_t option, int64_t value);
+int64_t impact_get_option(int32_t option);
 
 /* ---- loss and gradients --------------------------------------------------------------- */
 

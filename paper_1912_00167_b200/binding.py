@@ -34,7 +34,9 @@ EXPORTS = (
     "impact_buffer_slot_ptr", "impact_buffer_live", "impact_buffer_state_bytes",
     "impact_buffer_export_state", "impact_buffer_import_state", "impact_gather_rows",
     "impact_loss_fwd_bwd_static_scratch", "impact_loss_fwd_bwd_call", "impact_loss_workspace_status",
+    "impact_set_option", "impact_get_option",
 )
+OPT_EARLY_PREFETCH, OPT_PREFETCH_BYTES, OPT_WINDOW_BYTES = 0, 1, 2
 
 
 class ImpactError(RuntimeError):
@@ -120,6 +122,10 @@ def load_library() -> ctypes.CDLL:
     lib.impact_buffer_import_state.argtypes = [_vp, _vp, _sz]
     lib.impact_gather_rows.restype = _i32
     lib.impact_gather_rows.argtypes = [_vp, _vp, _i64, _i64, _sz, _vp, _vp]
+    lib.impact_set_option.restype = _i32
+    lib.impact_set_option.argtypes = [_i32, _i64]
+    lib.impact_get_option.restype = _i64
+    lib.impact_get_option.argtypes = [_i32]
     _lib = lib
     return lib
 
@@ -140,6 +146,14 @@ def impact_version() -> int:
 
 def impact_status_string(status: int) -> str:
     return load_library().impact_status_string(status).decode()
+
+
+def impact_set_option(option: int, value: int) -> None:
+    _check(load_library().impact_set_option(option, value), "impact_set_option")
+
+
+def impact_get_option(option: int) -> int:
+    return load_library().impact_get_option(option)
 
 
 def _dev(t: torch.Tensor | None, dtype, shape, name: str, optional: bool = False) -> int | None:

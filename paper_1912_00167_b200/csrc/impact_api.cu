@@ -1,6 +1,8 @@
 // Housekeeping entry points and the host helpers shared by the other translation units.
 #include <cuda_runtime.h>
 
+#include <atomic>
+
 #include "impact.h"
 #include "impact_internal.h"
 
@@ -35,7 +37,27 @@ const DeviceInfo* current_device_info() {
     return &infos[dev];
 }
 
+// Launch options: process-wide, read by every loss call at launch time (defaults in the order of IMPACT_OPT_*).
+static std::atomic<int64_t> g_options[IMPACT_NUM_OPTIONS] = {
+    {1},           // IMPACT_OPT_EARLY_PREFETCH
+    {48ll << 20},  // IMPACT_OPT_PREFETCH_BYTES
+    {72ll << 10},  // IMPACT_OPT_WINDOW_BYTES
+};
+int64_t option(int32_t which) { return g_options[which].load(std::memory_order_relaxed); }
+
 }  // namespace impact
+
+extern "C" int32_t impact_set_option(int32_t option, int64_t value) {
+    if (option < 0 || option >= IMPACT_NUM_OPTIONS || value < 0) return IMPACT_ERR_INVALID_ARG;
+    if (option == IMPACT_OPT_WINDOW_BYTES && (value < 16 * 1024 || value > 160 * 1024)) return IMPACT_ERR_INVALID_ARG;
+    impact::g_options[option].store(value, std::memory_order_relaxed);
+    return IMPACT_OK;
+}
+
+extern "C" int64_t impact_get_option(int32_t option) {
+    if (option < 0 || option >= IMPACT_NUM_OPTIONS) return -1;
+    return impact::option(option);
+}
 
 extern "C" int32_t impact_version(void) { return IMPACT_VERSION; }
 

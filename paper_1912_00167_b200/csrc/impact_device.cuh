@@ -163,6 +163,62 @@ __device__ __forceinline__ void fence_async_shared() { asm volatile("fence.proxy
 // All bulk stores of this thread have finished READING shared memory (it may be reused).
 __device__ __forceinline__ void bulk_store_wait_read() { asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory"); }
 
+// ---- byte ranges that do not start or end on a 16-byte boundary ---------------------------
+// A tile of a dense tensor starts wherever its first row does: for row pitches that are not a
+// multiple of 16 bytes (A = 18 in bf16: 36 bytes) most tiles start and end inside a 16-byte
+// granule, which a bulk copy cannot do.  Loads are therefore widened to the enclosing granules:
+// the copy also brings the up to 15 bytes before the range and the up to 15 bytes after it (the
+// tensor's own neighbouring rows) into the padding of the shared-memory slab, and the range
+// itself lands at the same offset inside its granule as in global memory.  Only where the tensor
+// ENDS inside the last granule is that granule fetched by ordinary loads instead.
+struct WideRange {
+    long long first;  // byte offset (in the tensor) of the first granule
+    uint32_t span;    // bytes a bulk copy may move from there: a multiple of 16, possibly 0
+    uint32_t tail;    // bytes after the span that belong to the tensor's last, partial granule (0..15)
+};
+__device__ __forceinline__ WideRange widen_range(long long byte0, uint32_t bytes, long long tensor_bytes) {
+    WideRange w;
+    const uint32_t m = (uint32_t)byte0 & 15u;
+    w.first = byte0 - m;
+    w.span = (m + bytes + 15u) & ~15u;
+    w.tail = 0;
+    if (w.first + (long long)w.span > tensor_bytes) {
+        w.span -= 16u;
+        w.tail = (uint32_t)(tensor_bytes - (w.first + (long long)w.span));
+    }
+    return w;
+}
+// Asks L2 for the granules of a byte range of a tensor whose base is 16-byte aligned (one request to the copy
+// engine; nothing waits for it).  Ordinary per-line prefetch instructions were tried instead and slowed the
+// launches down by half.
+__device__ __forceinline__ void prefetch_range_l2(const void* base, long long byte0, uint32_t bytes, long long tensor_bytes) {
+    const WideRange w = widen_range(byte0, bytes, tensor_bytes);
+    if (w.span) bulk_prefetch_l2(static_cast<const unsigned char*>(base) + w.first, w.span);
+}
+
+// Run by a whole warp: sends `bytes` bytes of shared memory at `src` to global memory at `dst`, where src and
+// dst agree modulo 16.  The whole granules in between leave by one bulk store (lane 0); the up to 15 bytes before
+// the first whole granule and after the last one leave by byte stores, a lane each (a granule shared with a
+// neighbouring range is written by both neighbours, each its own bytes).  `wrote`: the bytes were written by
+// ordinary stores of this warp's threads, so they are fenced towards the copy engine first.  Lane 0 learns
+// whether a bulk store was issued (its group is committed; see bulk_store_wait_read).
+__device__ __forceinline__ bool warp_send_bytes(unsigned char* dst, const unsigned char* src, uint32_t bytes, bool wrote) {
+    const uint32_t lane = threadIdx.x & 31u;
+    uint32_t head = (16u - ((uint32_t)reinterpret_cast<uintptr_t>(dst) & 15u)) & 15u;
+    if (head > bytes) head = bytes;
+    const uint32_t body = (bytes - head) & ~15u;
+    const uint32_t tail = bytes - head - body;
+    if (wrote) fence_async_shared();
+    __syncwarp();
+    if (lane < head) dst[lane] = src[lane];
+    if (lane >= 16u && lane - 16u < tail) dst[head + body + lane - 16u] = src[head + body + lane - 16u];
+    if (lane == 0 && body) {
+        bulk_store(dst + head, src + head, body);
+        return true;
+    }
+    return false;
+}
+
 __device__ __forceinline__ float exp2_fast(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));

@@ -22,6 +22,9 @@ struct DeviceInfo {
 // Returns nullptr (and records the error) when no CUDA device is usable.
 const DeviceInfo* current_device_info();
 
+// Current value of a launch option (IMPACT_OPT_*).
+int64_t option(int32_t which);
+
 // Launch with programmatic stream serialization: the grid may be set up on the device while
 // the previous kernel of the stream is still running.  Every kernel of this library starts
 // with grid_dependency_wait(), which returns only once that previous kernel has completed

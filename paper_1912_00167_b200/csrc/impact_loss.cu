@@ -845,10 +845,91 @@ __device__ __forceinline__ Place tile_place(const TileGeometry& g, int n, int ro
     return pl;
 }
 
+// A slab of the persistent kernels in shared memory: NT rows of `row_bytes`, plus 32 bytes of padding, because a
+// tile's rows sit at the same offset inside their 16-byte granule as in global memory (0..15 bytes after the
+// slab's start) and the copy that brings them is widened to whole granules (see dev::widen_range).
+__host__ __device__ constexpr size_t ws_slab_pitch(size_t nt, size_t row_bytes) { return nt * row_bytes + 32; }
+
 template <typename LT, typename GT, int A, int NT>
 __host__ __device__ constexpr size_t ws_stage_bytes() {
     constexpr size_t in_row = A * sizeof(LT), out_row = A * sizeof(GT);
-    return NT * (2 * in_row + (sizeof(LT) == sizeof(GT) ? 0 : out_row));
+    constexpr size_t raw = 2 * ws_slab_pitch(NT, in_row) + (sizeof(LT) == sizeof(GT) ? 0 : ws_slab_pitch(NT, out_row));
+    return (raw + 127) / 128 * 128;
+}
+
+// The same placement with the tile size and the form of the grid as run-time values (the companion kernel that
+// only prefetches, below).
+__device__ __forceinline__ Place tile_place_rt(const TileGeometry& g, int n, int rows_full, long long total_rows,
+                                               bool is_long, int nt) {
+    Place pl;
+    const long long gt_ = (long long)blockIdx.x + (long long)n * gridDim.x;
+    if (is_long) {
+        if (g.tile_major) {
+            pl.r = (int)((unsigned long long)gt_ / (unsigned long long)g.B);
+            pl.traj = gt_ - (long long)pl.r * g.B;
+        } else {
+            pl.traj = (long long)((unsigned long long)gt_ / (unsigned int)g.ntiles);
+            pl.r = (int)(gt_ - pl.traj * g.ntiles);
+        }
+        const long long t0 = (long long)(g.ntiles - 1 - pl.r) * nt;
+        const long long left = g.T - t0;
+        pl.nrows = left < nt ? (int)left : nt;
+        pl.row0 = pl.traj * g.T + t0;
+    } else {
+        pl.row0 = gt_ * rows_full;
+        pl.traj = gt_ * g.G;
+        const long long left = total_rows - pl.row0;
+        pl.nrows = left < rows_full ? (int)left : rows_full;
+        pl.r = 0;
+    }
+    return pl;
+}
+
+// ---- early prefetch -------------------------------------------------------------------------------------------
+// What a block of a persistent kernel will read, as a list of row-major arrays: the first tiles of every block
+// are asked for in L2 before the launch's stream dependency has resolved.  A prefetch changes nothing that a
+// program can observe (L2 is where the device's writes meet, so a later write to these addresses is not lost);
+// it only moves the wait for HBM from the start of this launch into the end of the one before it.
+constexpr int kMaxPrefetchArrays = 10;
+struct PrefetchList {
+    const void* base[kMaxPrefetchArrays];
+    int row_bytes[kMaxPrefetchArrays];
+    int n_arrays;
+    int n_tiles_max;  // tiles of a block that are asked for (from its first)
+    int nt;           // rows per tile
+    int is_long;
+    TileGeometry geo;
+};
+
+// Run by one warp: tile after tile in the order the block will want them, lane a asking for array a's rows of
+// the tile, so that the memory system sees the requests in that order too.
+__device__ __forceinline__ void prefetch_block_tiles(const PrefetchList& pf) {
+    const int lane = threadIdx.x & 31;
+    const TileGeometry& g = pf.geo;
+    const long long total_tiles = pf.is_long ? g.nchunks * g.ntiles : g.nchunks;
+    int n_tiles = (int)((total_tiles - blockIdx.x + gridDim.x - 1) / gridDim.x);
+    if (n_tiles > pf.n_tiles_max) n_tiles = pf.n_tiles_max;
+    const int rows_full = pf.is_long ? pf.nt : g.G * (int)g.T;
+    const long long total_rows = g.B * g.T;
+    const void* base = nullptr;
+    long long pitch = 0;
+#pragma unroll
+    for (int a = 0; a < kMaxPrefetchArrays; ++a)
+        if (lane == a && a < pf.n_arrays) { base = pf.base[a]; pitch = pf.row_bytes[a]; }
+    for (int n = 0; n < n_tiles; ++n) {
+        const Place pc = tile_place_rt(g, n, rows_full, total_rows, pf.is_long != 0, pf.nt);
+        if (base) dev::prefetch_range_l2(base, pc.row0 * pitch, (uint32_t)(pc.nrows * pitch), total_rows * pitch);
+    }
+}
+
+// The companion of a loss launch: enqueued right before it, it becomes resident next to the blocks of whatever
+// kernel is still running on the stream (it needs one warp and no shared memory per block), asks L2 for the
+// loss launch's first tiles, and only then waits for the stream's previous kernel -- which keeps stream order
+// exact for the loss kernel behind it, whose own dependency is this kernel.
+__global__ void __launch_bounds__(32) impact_prefetch_kernel(const __grid_constant__ PrefetchList pf) {
+    asm volatile("griddepcontrol.launch_dependents;" ::: "memory");
+    prefetch_block_tiles(pf);
+    asm volatile("griddepcontrol.wait;" ::: "memory");
 }
 constexpr int ws_tile_rows(int A) { return A > 32 ? 64 : 128; }
 constexpr int kWsMaxStages = 24;
@@ -919,13 +1000,34 @@ struct RowMath {
 // Rows wider than 32 actions are not held in registers: every pass streams the row from shared memory, the
 // gradient pass forms the exponentials again, and thread r starts its walk at pair r mod (A/2), because a row
 // pitch of 256 bytes would otherwise put all threads of a warp on the same banks.
+// Barrier protocol of the persistent kernels (S stages, at most W tiles in flight, lanes <= S - W):
+//   full[s]     one arrival (a producer lane's, with the bytes the tile's two copies will deliver): stage s holds
+//               the rows of its current tile.
+//   empty[s]    one arrival per consumer warp, after that warp's stores have finished reading the stage.
+// A wait names a phase by its PARITY, which is only unambiguous while the waiter is at most one phase ahead of the
+// barrier: asked about phase k while phase k-1 is still open, the barrier answers "complete".  The producer
+// therefore issues tiles STRICTLY in order, and tile n only after (a) tile n-W has landed and
+// (b) every consumer warp has released tile n-S.  From that:
+//   * consumer of tile n waits on full[n % S] for phase n/S.  It got there after consuming tile n-C, so n-C was
+//     issued, so (in order) tile n-S+W <= n-C was issued, so by (a) tile n-S -- phase n/S - 1 of the same stage --
+//     had landed: the barrier is in phase n/S or later.  It cannot be beyond n/S + 1 open, because tile n+S is not
+//     issued before this consumer releases tile n (b).  (This is where S >= W + C is needed.)
+//   * producer's look at full[(n-W) % S] for phase (n-W)/S: tile n-W was issued, so by (b) tile n-W-S was consumed,
+//     hence had landed: phase (n-W)/S - 1 is complete; tile n-W+S > n is not issued yet.
+//   * producer's look at empty[n % S] for phase n/S - 1: tile n-S was issued, so by (b) phase n/S - 2 is complete;
+//     phase n/S needs the consumers of tile n, which is not issued yet.
+// Without the in-order rule (lanes that found their own tile ready first went first) the first argument fails for
+// tiles of one round: a consumer could be handed a stage whose previous tile had not landed, read stale rows,
+// release the stage early, and the phases slipped until one of the bounded waits ran out.
 template <typename LT, typename GT, int A, int C, bool kPlain, bool kLong, int NT>
 __global__ void __launch_bounds__(C * NT + 32, 1)
-impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W, const int lanes) {
+impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W, const int lanes,
+                                  const int n_prefetch) {
     constexpr int NP = (A + 1) / 2;
     constexpr bool kStream = (A > 32);
     static_assert(!kStream || (A % 2 == 0 && (NP & (NP - 1)) == 0), "streamed rows: an even, power-of-two pair count");
     constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
+    constexpr int kInPitch = (int)ws_slab_pitch(NT, kInRow);
     constexpr int kStageBytes = (int)ws_stage_bytes<LT, GT, A, NT>();
     constexpr float kLog2e = 1.4426950408889634f, kLn2 = 0.6931471805599453f;
     using RM = RowMath<LT, A>;
@@ -950,26 +1052,23 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     if (tid >= C * NT) {
         // ---- producer warp ----------------------------------------------------------------------------------
         const int n_first = n_tiles < W ? n_tiles : W;
-        // First of all, while the kernel before this one on the stream is still finishing, lane n asks L2 for
-        // the block's n-th tile (logits and per-step scalars): a prefetch changes nothing that a program can
-        // observe (L2 is where the device's writes meet, so later writes to these addresses are not lost), but
-        // the pages are mapped and the bytes on their way when the dependency resolves.
-        if (lane < n_first) {
-            const Place pc = place_of(lane);
-            const long long row0 = pc.row0;
-            const uint32_t nrows = (uint32_t)pc.nrows;
-            const LT* const pl = static_cast<const LT*>(p.learner_logits) + row0 * A;
-            const LT* const pt = static_cast<const LT*>(p.target_logits) + row0 * A;
-            if (((reinterpret_cast<uintptr_t>(pl) | reinterpret_cast<uintptr_t>(pt) | (nrows * kInRow)) & 15u) == 0) {
-                dev::bulk_prefetch_l2(pl, nrows * kInRow);
-                dev::bulk_prefetch_l2(pt, nrows * kInRow);
-            }
-            if (((row0 | nrows) & 3) == 0) {  // 4-byte scalars: 16-byte granules
-                dev::bulk_prefetch_l2(p.actions + row0, nrows * 4u);
-                dev::bulk_prefetch_l2(p.worker_logp + row0, nrows * 4u);
-                dev::bulk_prefetch_l2(p.rewards + row0, nrows * 4u);
-                dev::bulk_prefetch_l2(p.discounts + row0, nrows * 4u);
-                dev::bulk_prefetch_l2(p.values + row0, nrows * 4u);
+        // First of all, while the kernel before this one on the stream is still finishing, the warp asks L2 for
+        // the block's first tiles (logits and per-step scalars), unless the launch's companion kernel has done so
+        // already: the pages are mapped and the bytes on their way when the dependency resolves.
+        if (n_prefetch > 0) {
+            const void* base = nullptr;
+            long long pitch = 4;
+            if (lane == 0) { base = p.learner_logits; pitch = kInRow; }
+            else if (lane == 1) { base = p.target_logits; pitch = kInRow; }
+            else if (lane == 2) base = p.actions;
+            else if (lane == 3) base = p.worker_logp;
+            else if (lane == 4) base = p.rewards;
+            else if (lane == 5) base = p.discounts;
+            else if (lane == 6) base = p.values;
+            const int n_pf = n_tiles < n_prefetch ? n_tiles : n_prefetch;
+            for (int n = 0; n < n_pf; ++n) {
+                const Place pc = place_of(n);
+                if (base) dev::prefetch_range_l2(base, pc.row0 * pitch, (uint32_t)(pc.nrows * pitch), total_rows * pitch);
             }
         }
         // then the barriers
@@ -982,89 +1081,92 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         dev::fence_mbarrier_init();
         __syncwarp();
 
-        grid_dependency_wait();
-
-        auto send_tile = [&](int n, int s) {
-            const Place pc = place_of(n);
-            const int nrows = pc.nrows;
-            const LT* const gl = static_cast<const LT*>(p.learner_logits) + pc.row0 * A;
-            const LT* const gt = static_cast<const LT*>(p.target_logits) + pc.row0 * A;
-            unsigned char* const d0 = smem_raw + s * kStageBytes;
-            unsigned char* const d1 = d0 + NT * kInRow;
-            const uint32_t bytes = (uint32_t)nrows * kInRow;
-            if (((reinterpret_cast<uintptr_t>(gl) | reinterpret_cast<uintptr_t>(gt) | bytes) & 15u) == 0) {
-                dev::mbarrier_expect_tx(&full_bar[s], 2 * bytes);
-                dev::bulk_load(d0, gl, bytes, &full_bar[s]);
-                dev::bulk_load(d1, gt, bytes, &full_bar[s]);
-            } else {  // ragged or unaligned slab: element by element
-                const int nelem = nrows * A;
-                for (int e = 0; e < nelem; ++e) {
-                    reinterpret_cast<LT*>(d0)[e] = gl[e];
-                    reinterpret_cast<LT*>(d1)[e] = gt[e];
+        // One slab of a tile into stage s: a bulk copy of the 16-byte granules that enclose the tile's rows
+        // (dev::widen_range).  The lane with the learner's slab makes the barrier's one arrival, announcing the
+        // bytes of both slabs; where the tensors end inside the last granule, it also fetches that granule's bytes
+        // of both slabs by ordinary loads, fenced towards the copy engine because the consumers may send the target
+        // rows on from the stage by a bulk store.
+        const long long tensor_bytes = total_rows * kInRow;
+        struct SlabRequest {
+            unsigned char* d0;        // the learner's slab of the stage (the target's lies kInPitch further)
+            const unsigned char* gl;  // first granule of the tile in the learner's logits
+            const unsigned char* gt;  // ... in the target's
+            uint32_t span, tail;      // dev::WideRange
+        };
+        auto request_for = [&](const Place& pc, int s) {
+            const dev::WideRange w = dev::widen_range(pc.row0 * (long long)kInRow, (uint32_t)pc.nrows * kInRow, tensor_bytes);
+            SlabRequest r;
+            r.d0 = smem_raw + s * kStageBytes;  // the tile's first row starts (row0 * kInRow) mod 16 bytes in
+            r.gl = static_cast<const unsigned char*>(p.learner_logits) + w.first;
+            r.gt = static_cast<const unsigned char*>(p.target_logits) + w.first;
+            r.span = w.span;
+            r.tail = w.tail;
+            return r;
+        };
+        auto send_slab = [&](const SlabRequest& r, int s, bool target) {
+            uint64_t* const bar = &full_bar[s];
+            if (target) {
+                if (r.span) dev::bulk_load(r.d0 + kInPitch, r.gt, r.span, bar);
+                return;
+            }
+            if (r.tail) {
+                for (uint32_t i = 0; i < r.tail; ++i) {
+                    r.d0[r.span + i] = r.gl[r.span + i];
+                    r.d0[kInPitch + r.span + i] = r.gt[r.span + i];
                 }
-                dev::mbarrier_arrive(&full_bar[s]);
+                dev::fence_async_shared();
+            }
+            if (r.span) {
+                dev::mbarrier_expect_tx(bar, 2 * r.span);
+                dev::bulk_load(r.d0, r.gl, r.span, bar);
+            } else {
+                dev::mbarrier_arrive(bar);
             }
         };
-        // the first W tiles need no wait (tile n goes to stage n), and leave before the rest of the block has even
-        // started: prepared a lane each, issued one lane at a time (see below)
-        for (int l = 0; l < n_first; ++l) {
-            if (lane == l) send_tile(l, l);
-            __syncwarp();
-        }
+        // Tiles leave in rounds: lane l < 16 owns the round's l-th tile and requests its learner slab, lane l + 16
+        // requests the same tile's target slab, so that all requests of a round leave in the same few instructions
+        // (one thread gets at most four bulk requests under way, and needs about a third of a microsecond per
+        // tile; a lane per request reaches the HBM rate).
+        const int sub = lane & 15;
+        const bool second = lane >= 16;
+        // the first W tiles need no wait (tile n goes to stage n): their requests are worked out now and leave the
+        // moment the stream's previous kernel is done, before the rest of the block has even started
+        const SlabRequest first = request_for(place_of(sub < n_first ? sub : 0), sub);
+
+        grid_dependency_wait();
+
+        if (sub < n_first) send_slab(first, sub, second);
         __syncthreads();  // the barriers are set up: the consumer warps may use them
-        // The rest.  Tile n goes to stage n % S once that stage's previous tile has left (the "empty" phase
-        // before this one) and tile n - W has landed (at most W tiles in flight).
-        if (n_tiles <= kWsFewTiles) {
-            // few tiles per block (a launch of a few microseconds): lane 0 alone, in blocking waits that the
-            // hardware ends the moment the barrier completes -- what counts here is how soon the next request
-            // leaves
-            if (lane == 0) {
-                int s = n_first % S, ws = 0;
-                uint32_t ph = (uint32_t)(n_first / S) & 1u, wph = 0;
-                for (int n = n_first; n < n_tiles; ++n) {
-                    bool ok = true;
-                    if (n >= S) ok = dev::mbarrier_wait(&empty_bar[s], ph ^ 1u, &abort_s);
-                    if (ok) ok = dev::mbarrier_wait(&full_bar[ws], wph, &abort_s);  // n >= W here
-                    if (!ok) { atomicExch(p.counter + 1, 1u); break; }
-                    send_tile(n, s);
-                    if (++s == S) { s = 0; ph ^= 1u; }
-                    if (++ws == S) { ws = 0; wph ^= 1u; }
+        // The rest.  Tile n goes to stage n % S once that stage's previous tile has left (the "empty" phase before
+        // this one) and tile n - W has landed (at most W tiles in flight).  The owners look at their barriers side by
+        // side, but a tile is sent only when every earlier tile of the round has been sent or is sent in the same
+        // instruction: tiles leave in order.
+        for (int base = n_first; base < n_tiles; base += lanes) {
+            const int n = base + sub;
+            bool pending = sub < lanes && n < n_tiles;
+            const int cyc = n / S, s = n - cyc * S;
+            const int wcyc = (n - W) / S, ws = (n - W) - wcyc * S;
+            const SlabRequest req = request_for(place_of(pending ? n : 0), s);
+            for (unsigned int spin = 0; spin < (1u << 22); ++spin) {
+                const bool ready = !second && pending && (cyc == 0 || dev::mbarrier_test(&empty_bar[s], (uint32_t)(cyc - 1) & 1u)) &&
+                                   dev::mbarrier_test(&full_bar[ws], (uint32_t)wcyc & 1u);
+                const unsigned int waiting = __ballot_sync(0xffffffffu, !second && pending && !ready);
+                bool go = ready && (waiting & ((1u << sub) - 1u)) == 0u;
+                go = __shfl_sync(0xffffffffu, go, sub);  // the owner decides for both lanes of its tile
+                if (go && pending) {
+                    send_slab(req, s, second);
+                    pending = false;
                 }
+                if (!__any_sync(0xffffffffu, pending)) break;
+                if (*reinterpret_cast<volatile int*>(&abort_s)) break;
+                __nanosleep(32);
             }
-        } else {
-            // many tiles per block: `lanes` tiles per round, a lane each, polling.  One thread walking through a
-            // tile's address arithmetic and barrier operations needs about half a microsecond, more than an SM has
-            // per tile when tiles are small.  Within a round no lane can get S - W tiles ahead of another
-            // (lanes <= S - W), so the barrier of tile n - W is still in the phase that the test asks about.
-            for (int base = n_first; base < n_tiles; base += lanes) {
-                const int n = base + lane;
-                bool pending = lane < lanes && n < n_tiles;
-                const int cyc = n / S, s = n - cyc * S;
-                const int wcyc = (n - W) / S, ws = (n - W) - wcyc * S;
-                for (unsigned int spin = 0; spin < (1u << 22); ++spin) {
-                    const bool ready = pending && (cyc == 0 || dev::mbarrier_test(&empty_bar[s], (uint32_t)(cyc - 1) & 1u)) &&
-                                       dev::mbarrier_test(&full_bar[ws], (uint32_t)wcyc & 1u);
-                    // the requests themselves leave one lane at a time: a bulk copy is issued from a warp-wide
-                    // (uniform) datapath, and several lanes inside it at once lost requests at four lanes with
-                    // four tiles in flight
-                    for (int l = 0; l < lanes; ++l) {
-                        if (lane == l && ready) {
-                            send_tile(n, s);
-                            pending = false;
-                        }
-                        __syncwarp();
-                    }
-                    if (!__any_sync(0xffffffffu, pending)) break;
-                    if (*reinterpret_cast<volatile int*>(&abort_s)) break;
-                    __nanosleep(32);
+            if (__any_sync(0xffffffffu, pending)) {  // a stage never came back, or a tile never landed
+                if (lane == 0) {
+                    atomicExch(p.counter + 1, 1u);
+                    *reinterpret_cast<volatile int*>(&abort_s) = 1;
                 }
-                if (__any_sync(0xffffffffu, pending)) {  // a stage never came back, or a tile never landed
-                    if (lane == 0) {
-                        atomicExch(p.counter + 1, 1u);
-                        *reinterpret_cast<volatile int*>(&abort_s) = 1;
-                    }
-                    break;
-                }
+                break;
             }
         }
         __syncwarp();
@@ -1127,6 +1229,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         dev::hand_over_group_sums(t_surr, t_val, t_ent, t_ratio, t_kl, want_kl, n_clip, n_trunc, red[grp][gwarp],
                                   &sums_bar[grp]);
     };
+
     bool pending = false;  // lane 0 of each warp: a store of this warp may still be reading its stage
     int pending_stage = 0;
 
@@ -1143,7 +1246,10 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         const StepRaw nxt = load_scalars(me_next);
         const bool active = me.active;
         const long long row = me.row;
-        if (lane == 0 && pending) {  // this warp's previous rows have left shared memory: hand the stage back
+        // this warp's previous rows have left shared memory: hand the stage back.  (Only where stages are used
+        // more than once: the wait for the store's reads sits between two tiles of the warp, and a block with no
+        // more tiles than stages never needs a stage back.)
+        if (lane == 0 && pending) {
             dev::bulk_store_wait_read();
             dev::mbarrier_arrive(&empty_bar[pending_stage]);
             pending = false;
@@ -1161,23 +1267,21 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
                                 me.pc.r - lane, early_a, early_b);
         if (!dev::mbarrier_wait(&full_bar[s], ph, &abort_s)) atomicExch(p.counter + 1, 1u);
 
-        unsigned char* const s0 = smem_raw + s * kStageBytes;  // learner logits
-        unsigned char* const s1 = s0 + NT * kInRow;             // target logits
-        unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : s0 + 2 * NT * kInRow;
-        // (first traversal of a batch) the target rows go to the circular buffer as well, each warp's 32 rows by a
-        // bulk store straight from the stage, which nothing writes to
+        // rows keep their place inside their 16-byte granule: the tile's first row starts (row0 * pitch) mod 16
+        // bytes into the slab
+        unsigned char* const stage = smem_raw + s * kStageBytes;
+        const uint32_t m_in = (uint32_t)(me.pc.row0 * kInRow) & 15u;
+        unsigned char* const s0 = stage + m_in;     // learner logits
+        unsigned char* const s1 = s0 + kInPitch;    // target logits
+        unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : stage + 2 * kInPitch + ((uint32_t)(me.pc.row0 * kOutRow) & 15u);
+        bool stored = false;  // lane 0: a bulk store of this warp reads the stage
+        // (first traversal of a batch) the target rows go to the circular buffer as well, each warp's 32 rows
+        // straight from the stage, which nothing writes to
         if (p.target_copy) {
             const int left = me.pc.nrows - (gtid - lane);
             const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
-            LT* const dst = static_cast<LT*>(p.target_copy) + (me.row - lane) * A;
-            const unsigned char* const src = s1 + (gtid - lane) * kInRow;
-            const uint32_t bytes = (uint32_t)wrows * kInRow;
-            if (((reinterpret_cast<uintptr_t>(dst) | bytes) & 15u) == 0) {
-                if (lane == 0 && bytes) dev::bulk_store(dst, src, bytes);
-            } else {
-                const int nelem = wrows * A;
-                for (int i = lane; i < nelem; i += 32) dst[i] = reinterpret_cast<const LT*>(src)[i];
-            }
+            unsigned char* const dst = static_cast<unsigned char*>(p.target_copy) + (me.row - lane) * (long long)kInRow;
+            stored = dev::warp_send_bytes(dst, s1 + (gtid - lane) * kInRow, (uint32_t)wrows * kInRow, false);
         }
         const int a = cur.a;
         dev::StepIn st;
@@ -1367,23 +1471,15 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             const long long wrow0 = row - lane;  // first row of this warp
             const int left = me.pc.nrows - (gtid - lane);
             const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
-            GT* const gd = static_cast<GT*>(p.dlogits) + wrow0 * A;
-            const unsigned char* const src = so + (gtid - lane) * kOutRow;
-            const uint32_t out_bytes = (uint32_t)wrows * kOutRow;
-            if (((reinterpret_cast<uintptr_t>(gd) | out_bytes) & 15u) == 0) {
-                dev::fence_async_shared();
-                __syncwarp();
-                if (lane == 0) {
-                    if (out_bytes) dev::bulk_store(gd, src, out_bytes);
-                    pending = true;
+            unsigned char* const gd = static_cast<unsigned char*>(p.dlogits) + wrow0 * (long long)kOutRow;
+            if (dev::warp_send_bytes(gd, so + (gtid - lane) * kOutRow, (uint32_t)wrows * kOutRow, true)) stored = true;
+            if (lane == 0) {
+                if (stored) {  // the stage goes back once the stores have read it: before this warp's next tile
+                    pending = n_tiles > S;
                     pending_stage = s;
+                } else {
+                    dev::mbarrier_arrive(&empty_bar[s]);
                 }
-            } else {
-                __syncwarp();
-                const int nelem = wrows * A;
-                for (int i = lane; i < nelem; i += 32) gd[i] = reinterpret_cast<const GT*>(src)[i];
-                __syncwarp();
-                if (lane == 0) dev::mbarrier_arrive(&empty_bar[s]);
             }
         }
         cur = nxt;
@@ -1394,9 +1490,10 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
 
     // a group without tiles still hands over its (zero) sums, so that every row of the grid is defined
     if (grp >= n_tiles) hand_over_sums();
-    // ---- one group of the grid (block 0's, the one with that block's last tile) collects every block's row
+    // ---- one group of the grid (block 0's, the one that runs out of tiles first and so is polling long before the
+    // last rows appear) collects every block's row
     // as it appears and writes the loss terms
-    if (blockIdx.x == 0 && grp == (n_tiles - 1) % C) {
+    if (blockIdx.x == 0 && grp == n_tiles % C) {
         if (!dev::reduce_tagged_rows<NT>(p.tagged_rows, (int)gridDim.x, dev::launch_tag(p.counter), p.counter,
                                          p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, k.steps_total,
                                          gtid, bar_id, &abort_s))
@@ -1755,13 +1852,19 @@ __global__ void __launch_bounds__(kRegTileRows, 4) impact_loss_gaussian_reg_kern
 // land, every warp stores its own rows, the block's sums leave as one tagged row.  Row arithmetic is
 // that of impact_loss_gaussian_reg_kernel (log-probabilities accumulated in fp64).  kLong as in the
 // categorical kernel: tiles of a long trajectory on neighbouring blocks, linked through their aggregates.
+template <int D>
+__host__ __device__ constexpr size_t gaussian_ws_stage_bytes() {
+    return (5 * ws_slab_pitch(128, D * sizeof(float)) + 127) / 128 * 128;
+}
+
 template <int D, int C, bool kLong>
 __global__ void __launch_bounds__(C * 128 + 32, 1)
-impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int S, const int W) {
+impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int S, const int W, const int lanes,
+                               const int n_prefetch) {
     constexpr int NT = 128;
     constexpr int kRow = D * (int)sizeof(float);
-    constexpr int kSlab = NT * kRow;
-    constexpr int kStageBytes = 5 * kSlab;
+    constexpr int kSlab = (int)ws_slab_pitch(NT, kRow);  // rows keep their place inside their 16-byte granule
+    constexpr int kStageBytes = (int)gaussian_ws_stage_bytes<D>();
     constexpr float kLog2e = 1.4426950408889634f;
     constexpr float kHalfLog2Pi = 0.91893853320467274178f;
     extern __shared__ __align__(128) unsigned char smem_raw[];
@@ -1786,23 +1889,21 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
         // ---- producer warp ----------------------------------------------------------------------------------
         const float* const src[5] = {p.learner_mean, p.learner_logstd, p.target_mean, p.target_logstd, p.actions};
         const int n_first = n_tiles < W ? n_tiles : W;
-        // lane n asks L2 for the block's n-th tile before the stream dependency resolves (see the categorical kernel)
-        if (lane < n_first) {
-            const Place pc = place_of(lane);
-            const long long row0 = pc.row0;
-            const uint32_t nrows = (uint32_t)pc.nrows;
-            uintptr_t align = nrows * kRow;
-#pragma unroll
-            for (int q = 0; q < 5; ++q) align |= reinterpret_cast<uintptr_t>(src[q] + row0 * D);
-            if ((align & 15u) == 0) {
-#pragma unroll
-                for (int q = 0; q < 5; ++q) dev::bulk_prefetch_l2(src[q] + row0 * D, nrows * kRow);
-            }
-            if (((row0 | nrows) & 3) == 0) {
-                dev::bulk_prefetch_l2(p.worker_logp + row0, nrows * 4u);
-                dev::bulk_prefetch_l2(p.rewards + row0, nrows * 4u);
-                dev::bulk_prefetch_l2(p.discounts + row0, nrows * 4u);
-                dev::bulk_prefetch_l2(p.values + row0, nrows * 4u);
+        const long long tensor_bytes = total_rows * kRow;
+        // the block's first tiles are asked for in L2 before the stream dependency resolves, unless the launch's
+        // companion kernel has done so already (see the categorical kernel): lane a takes array a
+        if (n_prefetch > 0) {
+            const void* base = nullptr;
+            long long pitch = 4;
+            if (lane < 5) { base = src[lane]; pitch = kRow; }
+            else if (lane == 5) base = p.worker_logp;
+            else if (lane == 6) base = p.rewards;
+            else if (lane == 7) base = p.discounts;
+            else if (lane == 8) base = p.values;
+            const int n_pf = n_tiles < n_prefetch ? n_tiles : n_prefetch;
+            for (int n = 0; n < n_pf; ++n) {
+                const Place pc = place_of(n);
+                if (base) dev::prefetch_range_l2(base, pc.row0 * pitch, (uint32_t)(pc.nrows * pitch), total_rows * pitch);
             }
         }
         if (lane < S) {
@@ -1814,43 +1915,78 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
         dev::fence_mbarrier_init();
         __syncwarp();
 
+        // One slab of a tile into stage s (protocol, widened copies and in-order issue as in the categorical
+        // kernel): lane l < 4 owns the round's l-th tile, requests its first slab, makes the barrier's arrival
+        // with the bytes of all five slabs and fetches the bytes of a last, partial granule of the tensors; lanes
+        // l + 4, l + 8, l + 12, l + 16 request the tile's other slabs.
+        struct SlabRequest {
+            unsigned char* d;      // the stage
+            long long first;       // byte offset of the tile's first granule in each of the five tensors
+            uint32_t span, tail;   // dev::WideRange
+        };
+        auto request_for = [&](const Place& pc, int s) {
+            const dev::WideRange w = dev::widen_range(pc.row0 * (long long)kRow, (uint32_t)pc.nrows * kRow, tensor_bytes);
+            SlabRequest r;
+            r.d = smem_raw + s * kStageBytes;
+            r.first = w.first;
+            r.span = w.span;
+            r.tail = w.tail;
+            return r;
+        };
+        auto send_slab = [&](const SlabRequest& r, int s, int q) {
+            uint64_t* const bar = &full_bar[s];
+            const unsigned char* const gq = reinterpret_cast<const unsigned char*>(src[q]) + r.first;
+            if (q == 0) {
+                if (r.tail) {
+#pragma unroll
+                    for (int j = 0; j < 5; ++j) {
+                        const unsigned char* const gj = reinterpret_cast<const unsigned char*>(src[j]) + r.first;
+                        for (uint32_t i = 0; i < r.tail; ++i) r.d[j * kSlab + r.span + i] = gj[r.span + i];
+                    }
+                    dev::fence_async_shared();
+                }
+                if (r.span) dev::mbarrier_expect_tx(bar, 5 * r.span);
+                else dev::mbarrier_arrive(bar);
+            }
+            if (r.span) dev::bulk_load(r.d + q * kSlab, gq, r.span, bar);
+        };
+        const int sub = lane & 3, q_lane = lane >> 2;
+        const bool sends = q_lane < 5;
+        const SlabRequest first = request_for(place_of(sub < n_first ? sub : 0), sub);
+
         grid_dependency_wait();
 
-        int s = 0, ws = 0;
-        uint32_t ph = 0, wph = 0;
-        auto send_tile = [&](int n) {
-            const Place pc = place_of(n);
-            const long long row0 = pc.row0;
-            const int nrows = pc.nrows;
-            unsigned char* const d = smem_raw + s * kStageBytes;
-            const uint32_t bytes = (uint32_t)nrows * kRow;
-            uintptr_t align = bytes;
-#pragma unroll
-            for (int q = 0; q < 5; ++q) align |= reinterpret_cast<uintptr_t>(src[q] + row0 * D);
-            if ((align & 15u) == 0) {
-                dev::mbarrier_expect_tx(&full_bar[s], 5 * bytes);
-#pragma unroll
-                for (int q = 0; q < 5; ++q) dev::bulk_load(d + q * kSlab, src[q] + row0 * D, bytes, &full_bar[s]);
-            } else {  // ragged or unaligned slabs: element by element
-                const int nelem = nrows * D;
-#pragma unroll
-                for (int q = 0; q < 5; ++q)
-                    for (int e = 0; e < nelem; ++e) reinterpret_cast<float*>(d + q * kSlab)[e] = src[q][row0 * D + e];
-                dev::mbarrier_arrive(&full_bar[s]);
-            }
-            if (++s == S) { s = 0; ph ^= 1u; }
-            if (n >= W) { if (++ws == S) { ws = 0; wph ^= 1u; } }
-        };
-        if (lane == 0)
-            for (int n = 0; n < n_first; ++n) send_tile(n);
+        // the first W tiles need no wait (tile n goes to stage n), four at a time
+        if (sends && sub < n_first) send_slab(first, sub, q_lane);
+        for (int base = 4; base < n_first; base += 4)
+            if (sends && base + sub < n_first) send_slab(request_for(place_of(base + sub), base + sub), base + sub, q_lane);
         __syncthreads();  // the barriers are set up: the consumer warps may use them
-        if (lane == 0) {
-            for (int n = n_first; n < n_tiles; ++n) {
-                bool ok = true;
-                if (n >= S) ok = dev::mbarrier_wait(&empty_bar[s], ph ^ 1u, &abort_s);
-                if (ok && n >= W) ok = dev::mbarrier_wait(&full_bar[ws], wph, &abort_s);
-                if (!ok) { atomicExch(p.counter + 1, 1u); break; }
-                send_tile(n);
+        for (int base = n_first; base < n_tiles; base += lanes) {
+            const int n = base + sub;
+            bool pending = sends && sub < lanes && n < n_tiles;
+            const int cyc = n / S, s = n - cyc * S;
+            const int wcyc = (n - W) / S, ws = (n - W) - wcyc * S;
+            const SlabRequest req = request_for(place_of(pending ? n : 0), s);
+            for (unsigned int spin = 0; spin < (1u << 22); ++spin) {
+                const bool ready = q_lane == 0 && pending && (cyc == 0 || dev::mbarrier_test(&empty_bar[s], (uint32_t)(cyc - 1) & 1u)) &&
+                                   dev::mbarrier_test(&full_bar[ws], (uint32_t)wcyc & 1u);
+                const unsigned int waiting = __ballot_sync(0xffffffffu, q_lane == 0 && pending && !ready);
+                bool go = ready && (waiting & ((1u << sub) - 1u)) == 0u;
+                go = __shfl_sync(0xffffffffu, go, sub);  // the owner decides for all lanes of its tile
+                if (go && pending) {
+                    send_slab(req, s, q_lane);
+                    pending = false;
+                }
+                if (!__any_sync(0xffffffffu, pending)) break;
+                if (*reinterpret_cast<volatile int*>(&abort_s)) break;
+                __nanosleep(32);
+            }
+            if (__any_sync(0xffffffffu, pending)) {  // a stage never came back, or a tile never landed
+                if (lane == 0) {
+                    atomicExch(p.counter + 1, 1u);
+                    *reinterpret_cast<volatile int*>(&abort_s) = 1;
+                }
+                break;
             }
         }
         __syncwarp();
@@ -1936,7 +2072,8 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
                                 me.pc.r - lane, early_a, early_b);
         if (!dev::mbarrier_wait(&full_bar[s], ph, &abort_s)) atomicExch(p.counter + 1, 1u);
 
-        unsigned char* const stage = smem_raw + s * kStageBytes;
+        // the tile's first row starts (row0 * kRow) mod 16 bytes into each slab
+        unsigned char* const stage = smem_raw + s * kStageBytes + ((uint32_t)(me.pc.row0 * kRow) & 15u);
         float* const r_mu = reinterpret_cast<float*>(stage) + gtid * D;              // learner mean -> dmean
         float* const r_ls = reinterpret_cast<float*>(stage + kSlab) + gtid * D;      // learner log-std -> dlogstd
         const float* const r_mt = reinterpret_cast<const float*>(stage + 2 * kSlab) + gtid * D;
@@ -2051,31 +2188,18 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
             const long long wrow0 = row - lane;
             const int left = me.pc.nrows - (gtid - lane);
             const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
-            float* const gm = p.dmean + wrow0 * D;
-            float* const gs = p.dlogstd + wrow0 * D;
+            unsigned char* const gm = reinterpret_cast<unsigned char*>(p.dmean) + wrow0 * (long long)kRow;
+            unsigned char* const gs = reinterpret_cast<unsigned char*>(p.dlogstd) + wrow0 * (long long)kRow;
             const unsigned char* const src_m = stage + (gtid - lane) * kRow;
-            const unsigned char* const src_s = stage + kSlab + (gtid - lane) * kRow;
-            const uint32_t out_bytes = (uint32_t)wrows * kRow;
-            if (((reinterpret_cast<uintptr_t>(gm) | reinterpret_cast<uintptr_t>(gs) | out_bytes) & 15u) == 0) {
-                dev::fence_async_shared();
-                __syncwarp();
-                if (lane == 0) {
-                    if (out_bytes) {
-                        dev::bulk_store(gm, src_m, out_bytes);
-                        dev::bulk_store(gs, src_s, out_bytes);
-                    }
-                    pending = true;
+            bool stored = dev::warp_send_bytes(gm, src_m, (uint32_t)wrows * kRow, true);
+            if (dev::warp_send_bytes(gs, src_m + kSlab, (uint32_t)wrows * kRow, false)) stored = true;  // (fenced above)
+            if (lane == 0) {
+                if (stored) {
+                    pending = n_tiles > S;  // a block with no more tiles than stages never needs a stage back
                     pending_stage = s;
+                } else {
+                    dev::mbarrier_arrive(&empty_bar[s]);
                 }
-            } else {
-                __syncwarp();
-                const int nelem = wrows * D;
-                for (int i = lane; i < nelem; i += 32) {
-                    gm[i] = reinterpret_cast<const float*>(src_m)[i];
-                    gs[i] = reinterpret_cast<const float*>(src_s)[i];
-                }
-                __syncwarp();
-                if (lane == 0) dev::mbarrier_arrive(&empty_bar[s]);
             }
         }
         cur = nxt;
@@ -2085,7 +2209,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     }
 
     if (grp >= n_tiles) hand_over_sums();
-    if (blockIdx.x == 0 && grp == (n_tiles - 1) % C) {
+    if (blockIdx.x == 0 && grp == n_tiles % C) {
         if (!dev::reduce_tagged_rows<NT>(p.tagged_rows, (int)gridDim.x, dev::launch_tag(p.counter), p.counter,
                                          p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, k.steps_total,
                                          gtid, bar_id, &abort_s))
@@ -2233,20 +2357,65 @@ int32_t copy_target_logits(const CatParams& p, size_t elem, cudaStream_t stream)
     return IMPACT_OK;
 }
 
-// Tiles the producer keeps in flight and stages of the ring, for tiles of `tile_in_bytes` bytes of logits:
-// about 48 KB per SM on the way (enough, over 148 SMs, to cover HBM's latency at full bandwidth; more
-// only delays the first tiles), and room beyond that for the tiles being worked on and being stored.
-void ws_ring_shape(size_t stage_bytes, size_t tile_in_bytes, int groups, int max_smem, int* stages, int* in_flight) {
-    int w = (int)((48 * 1024 + tile_in_bytes - 1) / tile_in_bytes);
+// Tiles the producer keeps in flight and stages of the ring, for tiles of `tile_in_bytes` bytes of logits.
+// Bytes in flight per SM (IMPACT_OPT_WINDOW_BYTES; 0 = chosen here): 72 KB where a block streams many tiles (over
+// 148 SMs that covers HBM's latency at full bandwidth; measured: 64 KB and more reach the copy rate, 48 KB stop at
+// 0.9 of it), 48 KB where a block has only a few (a bigger first burst makes every tile of it land later, and the
+// first tile's landing is what such a launch waits for).  Beyond the window there is room for the tiles being
+// worked on and being stored.  The barrier protocol needs stages >= in_flight + groups, or exactly one stage per
+// group (then the stage's previous tile is the one the same group worked on last); 0 stages = no valid shape.
+void ws_ring_shape(size_t stage_bytes, size_t tile_in_bytes, int groups, int max_smem, long long tiles_per_block,
+                   int* stages, int* in_flight) {
+    size_t window = (size_t)option(IMPACT_OPT_WINDOW_BYTES);
+    if (window == 0) window = tiles_per_block <= 8 ? 48 * 1024 : 72 * 1024;
+    int w = (int)((window + tile_in_bytes - 1) / tile_in_bytes);
     if (w < 2) w = 2;
     if (w > 8) w = 8;
     int s = w + groups + 3;
     if (s > kWsMaxStages) s = kWsMaxStages;
     const int fit = (int)((size_t)(max_smem - 4096) / stage_bytes);  // 4 KB left for static shared memory
     if (s > fit) s = fit;
-    if (w > s) w = s;
+    if (s > groups) {
+        if (w > s - groups) w = s - groups;
+    } else if (s == groups) {
+        if (w > s) w = s;
+    } else {
+        s = 0;
+    }
     *stages = s;
     *in_flight = w;
+}
+
+// How a persistent kernel is launched for a batch of `tiles` tiles on `grid` blocks.
+struct WsPlan {
+    int prefetch_tiles;  // tiles per block asked for in L2 ahead of time
+    bool companion;      // by a companion kernel enqueued before the loss kernel (else by the loss kernel's first warp)
+};
+WsPlan ws_plan(long long tiles, long long grid, size_t tile_bytes, int in_flight, bool allow_companion) {
+    WsPlan pl;
+    const long long per_block = (tiles + grid - 1) / grid;
+    const long long budget = option(IMPACT_OPT_PREFETCH_BYTES);
+    long long pf = budget / (grid * (long long)tile_bytes);
+    // Asking L2 for tiles ahead of time goes through the copy engine like the tiles themselves, so it pays only
+    // where requests are large (measured: with 18 KB tiles a short launch gains half a microsecond from its
+    // companion and a third from asking itself; with 3-9 KB tiles either costs 5-15 %).  The companion pays where a
+    // launch is short: a block has a handful of tiles, all within the budget.  A long launch is bound by HBM either
+    // way, and asking for many tiles far ahead of their use only competes with the tiles that are needed now.
+    // Without a companion the loss kernel's first warp asks for the tiles it is about to request anyway (more than
+    // that sits in the copy engine's queue ahead of the requests themselves).
+    const bool large_tiles = tile_bytes >= 16 * 1024;
+    pl.companion = allow_companion && large_tiles && option(IMPACT_OPT_EARLY_PREFETCH) != 0 && pf >= per_block &&
+                   per_block <= 8 && tiles * (long long)tile_bytes >= (4ll << 20);
+    if (!large_tiles) pf = 0;
+    if (!pl.companion && pf > in_flight) pf = in_flight;
+    if (pf > per_block) pf = per_block;
+    pl.prefetch_tiles = (int)pf;
+    return pl;
+}
+
+int32_t launch_companion(const PrefetchList& pf, long long grid, cudaStream_t stream) {
+    IMPACT_CUDA_TRY(launch_serialized(impact_prefetch_kernel, dim3((unsigned)grid), dim3(32), 0, stream, pf));
+    return IMPACT_OK;
 }
 
 template <typename LT, typename GT, int A, bool kPlain, bool kLong>
@@ -2258,25 +2427,42 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     constexpr int C = A > 32 ? 6 : (!kPlain ? kWsGroups : (A <= 9 ? kWsGroups + 2 : kWsGroups + 1));
     auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong, NT>;
     const size_t stage = ws_stage_bytes<LT, GT, A, NT>();
-    int S = 0, W = 0;
-    ws_ring_shape(stage, 2 * (size_t)NT * A * sizeof(LT), C, di->max_smem_optin, &S, &W);
-    if (S < 2) return IMPACT_ERR_UNSUPPORTED;
-
-
-    const size_t smem = (size_t)S * stage;
-    static thread_local int configured_device = -1;
-    if (configured_device != di->device) {
-        IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured_device = di->device;
-    }
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
     long long grid = tiles < di->sm_count ? tiles : di->sm_count;
     if (grid > kMaxTaggedRows) grid = kMaxTaggedRows;  // one tagged row per block
+    int S = 0, W = 0;
+    ws_ring_shape(stage, 2 * (size_t)NT * A * sizeof(LT), C, di->max_smem_optin, (tiles + grid - 1) / grid, &S, &W);
+    if (S < 1 || W < 1) return IMPACT_ERR_UNSUPPORTED;
+
+    const size_t smem = (size_t)S * stage;
+    static thread_local int configured_device = -1;
+    if (configured_device != di->device) {  // once per device: room for the largest ring any window setting asks for
+        IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, di->max_smem_optin - 4096));
+        configured_device = di->device;
+    }
     const int lanes = (S - W) < 4 ? ((S - W) < 1 ? 1 : (S - W)) : 4;  // producer lanes that request tiles side by side
     CatParams q = p;
     // tile-major once every block has a trajectory of its own: the aggregates a tile needs are then a round old
     q.geo.tile_major = (kLong && p.geo.B >= grid) ? 1 : 0;
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * NT + 32), smem, stream, q, S, W, lanes));
+    const int rows_full = kLong ? NT : q.geo.G * (int)q.geo.T;
+    const WsPlan plan = ws_plan(tiles, grid, (size_t)rows_full * (2 * A * sizeof(LT) + 20), W, true);
+    if (plan.companion) {
+        PrefetchList pf = {};
+        const void* bases[7] = {p.learner_logits, p.target_logits, p.actions, p.worker_logp, p.rewards, p.discounts, p.values};
+        for (int i = 0; i < 7; ++i) {
+            pf.base[i] = bases[i];
+            pf.row_bytes[i] = i < 2 ? A * (int)sizeof(LT) : 4;
+        }
+        pf.n_arrays = 7;
+        pf.n_tiles_max = plan.prefetch_tiles;
+        pf.nt = NT;
+        pf.is_long = kLong ? 1 : 0;
+        pf.geo = q.geo;
+        const int32_t st = launch_companion(pf, grid, stream);
+        if (st != IMPACT_OK) return st;
+    }
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * NT + 32), smem, stream, q, S, W, lanes,
+                                      plan.companion ? 0 : plan.prefetch_tiles));
     return IMPACT_OK;
 }
 
@@ -2377,22 +2563,44 @@ template <int D, bool kLong>
 int32_t launch_gaussian_ws(const GaussParams& p, const DeviceInfo* di, cudaStream_t stream) {
     constexpr int C = kWsGroupsGaussian;
     auto kernel = impact_loss_gaussian_ws_kernel<D, C, kLong>;
-    const size_t stage = (size_t)5 * kRegTileRows * D * sizeof(float);
-    int S = 0, W = 0;
-    ws_ring_shape(stage, stage, C, di->max_smem_optin, &S, &W);
-    if (S < 2) return IMPACT_ERR_UNSUPPORTED;
-    const size_t smem = (size_t)S * stage;
-    static thread_local int configured_device = -1;
-    if (configured_device != di->device) {
-        IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        configured_device = di->device;
-    }
+    const size_t stage = gaussian_ws_stage_bytes<D>();
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
     long long grid = tiles < di->sm_count ? tiles : di->sm_count;
     if (grid > kMaxTaggedRows) grid = kMaxTaggedRows;  // one tagged row per block
+    int S = 0, W = 0;
+    ws_ring_shape(stage, stage, C, di->max_smem_optin, (tiles + grid - 1) / grid, &S, &W);
+    if (S < 1 || W < 1) return IMPACT_ERR_UNSUPPORTED;
+    const size_t smem = (size_t)S * stage;
+    static thread_local int configured_device = -1;
+    if (configured_device != di->device) {
+        IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, di->max_smem_optin - 4096));
+        configured_device = di->device;
+    }
+    const int lanes = (S - W) < 4 ? ((S - W) < 1 ? 1 : (S - W)) : 4;  // tiles the producer requests side by side
     GaussParams q = p;
     q.geo.tile_major = (kLong && p.geo.B >= grid) ? 1 : 0;
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, q, S, W));
+    const int rows_full = kLong ? 128 : q.geo.G * (int)q.geo.T;
+    // (no companion here: measured on B = 512, T = 128, D = 17 it costs more of the copy engine's time than the
+    // earlier start gains: 10.7 us per launch with it, 8.8 us without)
+    const WsPlan plan = ws_plan(tiles, grid, (size_t)rows_full * (5 * D * sizeof(float) + 16), W, false);
+    if (plan.companion) {
+        PrefetchList pf = {};
+        const void* bases[9] = {p.learner_mean, p.learner_logstd, p.target_mean, p.target_logstd, p.actions,
+                                p.worker_logp, p.rewards, p.discounts, p.values};
+        for (int i = 0; i < 9; ++i) {
+            pf.base[i] = bases[i];
+            pf.row_bytes[i] = i < 5 ? D * (int)sizeof(float) : 4;
+        }
+        pf.n_arrays = 9;
+        pf.n_tiles_max = plan.prefetch_tiles;
+        pf.nt = 128;
+        pf.is_long = kLong ? 1 : 0;
+        pf.geo = q.geo;
+        const int32_t st = launch_companion(pf, grid, stream);
+        if (st != IMPACT_OK) return st;
+    }
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * 128 + 32), smem, stream, q, S, W, lanes,
+                                      plan.companion ? 0 : plan.prefetch_tiles));
     return IMPACT_OK;
 }
 
@@ -2467,7 +2675,7 @@ static int32_t loss_fwd_bwd_impl(
         return IMPACT_ERR_UNSUPPORTED;
     if (workspace_bytes < kWorkspaceFixedBytes) return IMPACT_ERR_WORKSPACE_TOO_SMALL;
 
-    CatParams p;
+    CatParams p = {};
     int32_t st = fill_scalars(p.k, rho_bar, c_bar, clip_eps, coef, B, T);
     if (st != IMPACT_OK) return st;
     const DeviceInfo* di = current_device_info();
@@ -2651,7 +2859,7 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
         return IMPACT_ERR_INVALID_ARG;
     if (A > 64) return IMPACT_ERR_UNSUPPORTED;  // keeps the tile at 64 steps or more, which the limit below counts in
 
-    CatParams p;
+    CatParams p = {};
     int32_t st = fill_scalars(p.k, rho_bar, c_bar, clip_eps, coef, B, T);
     if (st != IMPACT_OK) return st;
     p.A = A;

@@ -14,8 +14,17 @@ import impact_inputs as ii
 
 RTOL_ELEM, ATOL_ELEM = 1e-5, 1e-6
 RTOL_SCALAR, ATOL_SCALAR = 1e-4, 1e-7
-RTOL_BF16, ATOL_BF16 = 2e-2, 2e-3
-COND_ADV = 4e-6  # ~64 fp32 unit roundoffs (2^-24) of the advantage's condition sum
+RTOL_BF16, ATOL_BF16 = 2e-2, 1e-5  # bf16-stored gradients: the stated 2e-2 relative; the floor only covers elements
+                                   # that cancel to (almost) nothing before they are rounded to bf16
+COND_ADV = 1e-6  # 16 fp32 unit roundoffs (2^-24) of the advantage's condition sum: twice the worst case measured
+                 # over every parity case (5.5e-7, a Gaussian batch; categorical batches stay below 2.5e-7)
+
+
+def min_literal_share(n: int) -> float:
+    """Share of an output's elements that must meet the stated 1e-5 / 1e-6 bar with no allowance for the advantage's
+    conditioning.  Measured: large batches keep 99.95 % and more inside it (named configs: all but 0-6 of 130 000
+    steps); batches of a few hundred elements can hold a handful of strongly cancelling steps, hence 99 % there."""
+    return 0.9995 if n >= 50_000 else 0.99
 
 
 def f32_hyper(h: ii.LossHyper) -> ii.LossHyper:
@@ -92,7 +101,7 @@ def logp_scale(batch):
 
 
 def compare(gpu, ref, ref_flipped, near, M, grad_keys, kl_coef, sens, vf_coef, rtol=RTOL_ELEM, atol=ATOL_ELEM,
-            rtol_scalar=RTOL_SCALAR, atol_scalar=ATOL_SCALAR, cond=COND_ADV, min_literal=0.995, scale_l=1.0,
+            rtol_scalar=RTOL_SCALAR, atol_scalar=ATOL_SCALAR, cond=COND_ADV, min_literal=None, scale_l=1.0,
             kl_always=False, term_tol=None):
     """Element-by-element comparison.
 
@@ -101,7 +110,7 @@ def compare(gpu, ref, ref_flipped, near, M, grad_keys, kl_coef, sens, vf_coef, r
     values of the terms A_t is made of (the oracle's `adv_cond`), `cond` a few dozen fp32
     unit roundoffs, and s = |d output / d A_t|.  Without it, steps where A_t cancels to
     much less than its terms could not meet a purely relative bound in fp32 arithmetic.
-    At least `min_literal` of the elements must meet the bar without that term.
+    At least `min_literal` of the elements (default: min_literal_share) must meet the bar without that term.
     """
     report = {}
     rtol, cond = rtol * scale_l, cond * scale_l
@@ -131,12 +140,21 @@ def compare(gpu, ref, ref_flipped, near, M, grad_keys, kl_coef, sens, vf_coef, r
             literal = literal | (near[..., None] & alt)
         else:
             bad = ~ok
-        report[key] = dict(max_abs=float(err.max()), literal_frac=float(literal.mean()))
+        # how far the worst element is from the stated bar (in units of it), and what multiple of the condition sum
+        # S_t the part beyond the stated bar amounts to (the bar allows `cond`)
+        over = err / (rtol * np.abs(want) + atol)
+        unit = extra / cond if cond > 0 else np.zeros_like(err)
+        beyond = np.maximum(err - (rtol * np.abs(want) + atol), 0.0)
+        with np.errstate(divide="ignore", invalid="ignore"):
+            cond_used = np.where(unit > 0, beyond / unit, 0.0)
+        report[key] = dict(max_abs=float(err.max()), literal_frac=float(literal.mean()), n=int(literal.size),
+                           n_outside=int((~literal).sum()), worst_over_bar=float(over.max()),
+                           cond_used=float(cond_used.max()))
         assert not bad.any(), (f"{key}: {int(bad.sum())} mismatches, worst abs {err[bad].max():.3e} "
                                f"at {np.argwhere(bad)[0]} got {got[bad].ravel()[0]:.8e} want {want[bad].ravel()[0]:.8e}")
-        n_outside = int((~literal).sum())  # small batches: one or two cancelling steps are not a trend
-        assert n_outside <= max(2, (1.0 - min_literal) * literal.size), (
-            f"{key}: only {literal.mean():.5f} of elements within rtol/atol")
+        need = min_literal if min_literal is not None else min_literal_share(literal.size)
+        assert int((~literal).sum()) <= (1.0 - need) * literal.size, (
+            f"{key}: only {literal.mean():.5f} of {literal.size} elements within rtol/atol (need {need})")
     lt_g, lt_r = gpu["loss_terms"].copy(), ref["loss_terms"]
     if kl_coef == 0.0 and not kl_always:
         # the library evaluates the KL term only when it enters the loss, and reports 0 otherwise
@@ -148,7 +166,18 @@ def compare(gpu, ref, ref_flipped, near, M, grad_keys, kl_coef, sens, vf_coef, r
         ok = ok | _close(lt_g, ref_flipped["loss_terms"], rtol_scalar, atol_scalar)
     assert ok.all(), f"loss_terms: gpu {lt_g} vs oracle {lt_r}"
     report["loss_terms"] = float(np.max(np.abs(lt_g - lt_r) / (np.abs(lt_r) + 1e-12)))
+    _log_report(report)
     return report
+
+
+def _log_report(report):
+    """With IMPACT_PARITY_REPORT=<file> every comparison appends one JSON line (test id + per-output figures): the
+    table of measured margins in the design doc is made from it."""
+    import json, os
+    path = os.environ.get("IMPACT_PARITY_REPORT")
+    if path:
+        with open(path, "a") as f:
+            f.write(json.dumps({"test": os.environ.get("PYTEST_CURRENT_TEST", ""), **report}) + "\n")
 
 
 def _policy_sensitivity(loss_fn, batch, h, keys, M, flip):

@@ -31,7 +31,7 @@ def test_every_declared_symbol_is_exported(lib):
 
 
 def test_housekeeping_calls(lib):
-    assert lib.impact_version() == 200
+    assert lib.impact_version() == 300
     assert lib.impact_status_string(0) == b"ok"
     assert b"full" in lib.impact_status_string(-5)
     assert b"empty" in lib.impact_status_string(-4)
