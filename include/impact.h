@@ -205,7 +205,10 @@ int32_t impact_loss_workspace_status(const void* workspace, size_t workspace_byt
  * workspace: device scratch of at least impact_loss_workspace_bytes(B,T) bytes, cleared
  *   once with impact_loss_workspace_init.
  * Limits: 1 <= A <= 512; B*T*A < 2^40.  No input is clamped or sanitised: NaN/Inf inputs
- * give NaN/Inf outputs wherever the arithmetic above carries them.
+ * give NaN/Inf outputs wherever the arithmetic above carries them -- and, because trajectories
+ * shorter than 128 steps are worked on several to a tile with the recursion cut between them by
+ * a factor of zero, possibly also in the trajectories that precede the affected one within its
+ * tile (floor(128 / T) consecutive trajectories).  No wait depends on a value: nothing hangs.
  * Errors: INVALID_ARG, UNSUPPORTED, WORKSPACE_TOO_SMALL, CUDA (launch failure).
  */
 int32_t impact_loss_fwd_bwd(
@@ -301,6 +304,8 @@ int32_t impact_loss_fwd_bwd_gaussian(
  * previous call left.  All calls on a device share the one array: two calls whose kernels
  * may run at the same time (different streams, or different host threads without ordering)
  * corrupt each other's sums.  Keep them on one stream or order them with events.
+ * The array's error word (see impact_loss_workspace_status) is sticky across calls: read it,
+ * and clear it, with impact_loss_static_scratch_status.
  */
 int32_t impact_loss_fwd_bwd_static_scratch(
     const void* learner_logits, const void* target_logits, const float* worker_logp,
@@ -309,6 +314,14 @@ int32_t impact_loss_fwd_bwd_static_scratch(
     const impact_coefficients* coef, int64_t B, int64_t T, int32_t A, int32_t logits_dtype,
     float* loss_terms, void* dlogits, float* dvalues, float* vtarget, float* advantage,
     void* stream);
+
+/*
+ * The error word of the built-in scratch of impact_loss_fwd_bwd_static_scratch on the current device, into
+ * *flag_out (HOST): 0 = no call through that entry point has given up a bounded wait since the word was last
+ * cleared; non-zero = at least one did, and the outputs of such a call are not to be trusted.  clear != 0 also
+ * resets the word.  Synchronises `stream`; allocates nothing.  (No counterpart in the paper.)
+ */
+int32_t impact_loss_static_scratch_status(int32_t* flag_out, int32_t clear, void* stream);
 
 /* ---- circular buffer C(N, K) ---------------------------------------------------------- */
 

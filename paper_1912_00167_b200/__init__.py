@@ -6,7 +6,7 @@ library is loaded on first use and its absence is an error.
 from .binding import (  # noqa: F401
     Coefficients, ImpactBuffer, ImpactError, PreparedCall, TERM_NAMES,
     impact_gather_rows, impact_loss_fwd_bwd, impact_loss_fwd_bwd_gaussian,
-    impact_get_option, impact_loss_fwd_bwd_static_scratch, impact_set_option,
+    impact_get_option, impact_loss_fwd_bwd_static_scratch, impact_loss_static_scratch_status, impact_set_option,
     impact_loss_workspace_bytes, impact_loss_workspace_init, impact_loss_workspace_status, impact_status_string,
     impact_version, load_library, new_workspace, prepare_loss_fwd_bwd,
     prepare_loss_fwd_bwd_gaussian,

@@ -34,7 +34,7 @@ EXPORTS = (
     "impact_buffer_slot_ptr", "impact_buffer_live", "impact_buffer_state_bytes",
     "impact_buffer_export_state", "impact_buffer_import_state", "impact_gather_rows",
     "impact_loss_fwd_bwd_static_scratch", "impact_loss_fwd_bwd_call", "impact_loss_workspace_status",
-    "impact_set_option", "impact_get_option",
+    "impact_set_option", "impact_get_option", "impact_loss_static_scratch_status",
 )
 OPT_EARLY_PREFETCH, OPT_PREFETCH_BYTES, OPT_WINDOW_BYTES = 0, 1, 2
 
@@ -122,6 +122,8 @@ def load_library() -> ctypes.CDLL:
     lib.impact_buffer_import_state.argtypes = [_vp, _vp, _sz]
     lib.impact_gather_rows.restype = _i32
     lib.impact_gather_rows.argtypes = [_vp, _vp, _i64, _i64, _sz, _vp, _vp]
+    lib.impact_loss_static_scratch_status.restype = _i32
+    lib.impact_loss_static_scratch_status.argtypes = [ctypes.POINTER(_i32), _i32, _vp]
     lib.impact_set_option.restype = _i32
     lib.impact_set_option.argtypes = [_i32, _i64]
     lib.impact_get_option.restype = _i64
@@ -307,6 +309,14 @@ def impact_loss_fwd_bwd_static_scratch(learner_logits, target_logits, worker_log
         _dev(dvalues, f32, bt, "dvalues"), _dev(vtarget, f32, bt, "vtarget", True),
         _dev(advantage, f32, bt, "advantage", True), _stream(stream))
     _check(st, "impact_loss_fwd_bwd_static_scratch")
+
+
+def impact_loss_static_scratch_status(clear: bool = False, stream=None) -> int:
+    """Error word of the built-in scratch on the current device (0 = every bounded wait completed); synchronises."""
+    flag = _i32(-1)
+    _check(load_library().impact_loss_static_scratch_status(ctypes.byref(flag), 1 if clear else 0, _stream(stream)),
+           "impact_loss_static_scratch_status")
+    return flag.value
 
 
 def prepare_loss_fwd_bwd_gaussian(learner_mean, learner_logstd, target_mean, target_logstd, worker_logp, actions,

@@ -2874,11 +2874,11 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     st = static_scratch_address(di, &scratch);
     if (st != IMPACT_OK) return st;
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    // the scratch keeps whatever the previous call left; the completion counter and the error word are
-    // what has to start at zero (the launch number next to them must live on: it is what tells this call's
-    // rows from the previous call's)
+    // the scratch keeps whatever the previous call left; the completion counter is what has to start at zero.  The
+    // error word next to it stays as it is (it is sticky until impact_loss_static_scratch_status clears it), and so
+    // does the launch number, which is what tells this call's rows from the previous call's.
     unsigned char* counter = scratch + (size_t)kStaticMaxBlocks * 8 * sizeof(float);
-    IMPACT_CUDA_TRY(cudaMemsetAsync(counter, 0, 2 * sizeof(unsigned int), s));
+    IMPACT_CUDA_TRY(cudaMemsetAsync(counter, 0, sizeof(unsigned int), s));
 
     p.learner_logits = learner_logits;
     p.target_logits = target_logits;
@@ -2901,4 +2901,21 @@ extern "C" int32_t impact_loss_fwd_bwd_static_scratch(
     // the same kernels, chosen the same way, as impact_loss_fwd_bwd
     return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
                            di, s);
+}
+
+extern "C" int32_t impact_loss_static_scratch_status(int32_t* flag_out, int32_t clear, void* stream) {
+    if (!flag_out) return IMPACT_ERR_INVALID_ARG;
+    const DeviceInfo* di = current_device_info();
+    if (!di) return IMPACT_ERR_CUDA;
+    unsigned char* scratch = nullptr;
+    const int32_t st = static_scratch_address(di, &scratch);
+    if (st != IMPACT_OK) return st;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    unsigned char* word = scratch + (size_t)kStaticMaxBlocks * 8 * sizeof(float) + sizeof(unsigned int);
+    unsigned int flag = 0;
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(&flag, word, sizeof(flag), cudaMemcpyDeviceToHost, s));
+    IMPACT_CUDA_TRY(cudaStreamSynchronize(s));
+    if (clear && flag != 0) IMPACT_CUDA_TRY(cudaMemsetAsync(word, 0, sizeof(unsigned int), s));
+    *flag_out = (int32_t)flag;
+    return IMPACT_OK;
 }

@@ -42,23 +42,56 @@ def to_coef(h: ii.LossHyper):
                            is_source=h.is_source, ratio_mode=h.ratio_mode, objective=h.objective)
 
 
-def run_gpu_categorical(batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, extra=True):
+class Guarded:
+    """Output tensors with canary words on both sides (the compute sanitizer's stand-in): every output is a view into
+    a larger allocation whose 256 bytes before and after it hold a bit pattern that no kernel writes; `check()`
+    fails if a single one of those bytes changed."""
+
+    GUARD_BYTES = 256
+    PATTERN = 0xA5
+
+    def __init__(self, dev="cuda"):
+        self.dev, self._raw = dev, []
+
+    def full(self, shape, fill, dtype=torch.float32):
+        n = int(np.prod(shape)) * torch.empty((), dtype=dtype).element_size()
+        raw = torch.full((n + 2 * self.GUARD_BYTES,), self.PATTERN, dtype=torch.uint8, device=self.dev)
+        view = raw[self.GUARD_BYTES:self.GUARD_BYTES + n].view(dtype).view(*shape)
+        view.fill_(fill)
+        self._raw.append((raw, n))
+        return view
+
+    def check(self):
+        for raw, n in self._raw:
+            g = self.GUARD_BYTES
+            assert bool((raw[:g] == self.PATTERN).all()), "bytes BEFORE an output buffer were overwritten"
+            assert bool((raw[g + n:] == self.PATTERN).all()), "bytes AFTER an output buffer were overwritten"
+
+
+def run_gpu_categorical(batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, extra=True,
+                        target_copy=False):
     import paper_1912_00167_b200 as ip
     dev = "cuda"
     t = {k: torch.from_numpy(np.ascontiguousarray(v)).to(dev) for k, v in batch.items()}
     zl = t["learner_logits"].to(logits_dtype)
     zt = t["target_logits"].to(logits_dtype)
     B, T, A = zl.shape
-    out = dict(loss_terms=torch.full((8,), float("nan"), device=dev),
-               dlogits=torch.full((B, T, A), float("nan"), device=dev, dtype=dlogits_dtype),
-               dvalues=torch.full((B, T), float("nan"), device=dev))
+    g = Guarded(dev)
+    out = dict(loss_terms=g.full((8,), float("nan")),
+               dlogits=g.full((B, T, A), float("nan"), dlogits_dtype),
+               dvalues=g.full((B, T), float("nan")))
     if extra:
-        out["vtarget"] = torch.full((B, T), float("nan"), device=dev)
-        out["advantage"] = torch.full((B, T), float("nan"), device=dev)
+        out["vtarget"] = g.full((B, T), float("nan"))
+        out["advantage"] = g.full((B, T), float("nan"))
+    copy = g.full((B, T, A), -7.0, logits_dtype) if target_copy else None
     ws = ip.new_workspace(B, T)
     ip.impact_loss_fwd_bwd(zl, zt, t["worker_logp"], t["actions"], t["rewards"], t["discounts"], t["values"],
-                           t["bootstrap_values"], to_coef(h), workspace=ws, **out)
+                           t["bootstrap_values"], to_coef(h), workspace=ws, target_logits_copy=copy, **out)
     torch.cuda.synchronize()
+    g.check()
+    assert ip.impact_loss_workspace_status(ws) == 0
+    if target_copy:
+        assert torch.equal(copy.view(torch.uint8), zt.view(torch.uint8)), "the copy of the target logits differs"
     return {k: v.float().cpu().numpy().astype(np.float64) for k, v in out.items()}
 
 
@@ -67,18 +100,19 @@ def run_gpu_gaussian(batch, h, extra=True):
     dev = "cuda"
     t = {k: torch.from_numpy(np.ascontiguousarray(v)).to(dev) for k, v in batch.items()}
     B, T, D = t["learner_mean"].shape
-    out = dict(loss_terms=torch.full((8,), float("nan"), device=dev),
-               dmean=torch.full((B, T, D), float("nan"), device=dev),
-               dlogstd=torch.full((B, T, D), float("nan"), device=dev),
-               dvalues=torch.full((B, T), float("nan"), device=dev))
+    g = Guarded(dev)
+    out = dict(loss_terms=g.full((8,), float("nan")), dmean=g.full((B, T, D), float("nan")),
+               dlogstd=g.full((B, T, D), float("nan")), dvalues=g.full((B, T), float("nan")))
     if extra:
-        out["vtarget"] = torch.full((B, T), float("nan"), device=dev)
-        out["advantage"] = torch.full((B, T), float("nan"), device=dev)
+        out["vtarget"] = g.full((B, T), float("nan"))
+        out["advantage"] = g.full((B, T), float("nan"))
     ws = ip.new_workspace(B, T)
     ip.impact_loss_fwd_bwd_gaussian(t["learner_mean"], t["learner_logstd"], t["target_mean"], t["target_logstd"],
                                     t["worker_logp"], t["actions"], t["rewards"], t["discounts"], t["values"],
                                     t["bootstrap_values"], to_coef(h), workspace=ws, **out)
     torch.cuda.synchronize()
+    g.check()
+    assert ip.impact_loss_workspace_status(ws) == 0
     return {k: v.cpu().numpy().astype(np.float64) for k, v in out.items()}
 
 
@@ -203,7 +237,8 @@ def _vtrace_pg_bounds(ref, sens):
     return ref, sens
 
 
-def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, extra=True, **tol):
+def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtype=torch.float32, extra=True,
+                      target_copy=False, **tol):
     h = f32_hyper(h)
     if logits_dtype == torch.bfloat16:
         batch = dict(batch)
@@ -212,7 +247,7 @@ def check_categorical(oracle, batch, h, logits_dtype=torch.float32, dlogits_dtyp
     ref = oracle.loss_categorical(batch, h)
     near = near_clip_bound(ref, h)
     ref_flipped = oracle.loss_categorical(batch, h, flip=near.astype(np.int8)) if near.any() else None
-    gpu = run_gpu_categorical(batch, h, logits_dtype, dlogits_dtype, extra=extra)
+    gpu = run_gpu_categorical(batch, h, logits_dtype, dlogits_dtype, extra=extra, target_copy=target_copy)
     M = batch["rewards"].size
     if h.objective == 1:
         from scipy.special import softmax

@@ -77,6 +77,97 @@ def test_bf16_ragged(oracle, B, T, A):
     P.check_categorical(oracle, batch, h, torch.bfloat16, torch.float32)
 
 
+@pytest.mark.parametrize("B,T,A,dtype", [(301, 21, 9, torch.bfloat16), (77, 21, 6, torch.bfloat16),
+                                         (50, 25, 9, torch.float32), (1311, 50, 18, torch.bfloat16),
+                                         (2000, 21, 9, torch.bfloat16), (151, 127, 18, torch.bfloat16)])
+def test_tiles_that_start_and_end_inside_a_16_byte_granule(oracle, B, T, A, dtype):
+    """Row pitches that are no multiple of 16 bytes: every tile (or the last one) starts or ends inside a granule, so
+    the bulk copies are widened to the enclosing granules, the ends of the gradient rows and of the copied target
+    rows leave byte by byte, and the tensors' last partial granule comes by ordinary loads.  Few tiles per block
+    and more tiles than stages; the target logits are copied out as on a batch's first traversal."""
+    batch = ii.categorical_batch(B, T, A, seed=4100 + B + T + A, p_done=0.02)
+    plain = LossHyper(rho_bar=1.0, c_bar=1.0, clip_eps=0.3, vf_coef=0.5, ent_coef=0.01, kl_coef=0.0, rho_tw=1.0)
+    full = LossHyper(rho_bar=1.3, c_bar=1.1, clip_eps=0.25, vf_coef=0.7, ent_coef=0.02, kl_coef=0.1, lam=0.97, rho_tw=2.0)
+    if dtype == torch.bfloat16:
+        P.check_categorical(oracle, batch, plain, dtype, dtype, extra=False, target_copy=True, rtol=P.RTOL_BF16,
+                            atol=P.ATOL_BF16)
+        P.check_categorical(oracle, batch, full, dtype, torch.float32, target_copy=True)
+        P.check_categorical(oracle, batch, plain, torch.float32, dtype, extra=False, target_copy=True, rtol=P.RTOL_BF16,
+                            atol=P.ATOL_BF16)
+    else:
+        P.check_categorical(oracle, batch, plain, extra=False, target_copy=True)
+        P.check_categorical(oracle, batch, full, target_copy=True)
+
+
+@pytest.mark.parametrize("idx", [0, 1, 2])
+def test_named_configs_compare_the_kl_term_too(oracle, idx):
+    """The named configurations have kl_coef = 0, where the library does not evaluate the KL term (and reports 0,
+    which the other tests assert).  With a coefficient of 1e-20 the term is evaluated and weighs nothing: every
+    output including mean KL is compared with the oracle."""
+    cfg, batch = ii.make_config(idx)
+    P.check_categorical(oracle, batch, dataclasses.replace(cfg.hyper, kl_coef=1e-20))
+
+
+def test_nan_and_inf_inputs_propagate_and_nothing_hangs():
+    """No input is sanitised: a NaN logit or an infinite reward shows up in the outputs that depend on it (and in
+    the batch means), the gradients of the trajectories in other tiles are those of the clean batch, and no wait
+    gives up.  (Short trajectories share a 128-step tile, and the recursion's cut between them is a multiplication
+    by zero, which a non-finite value survives: it may also reach the trajectories before it in its own tile.)"""
+    import paper_1912_00167_b200 as ip
+    cfg, batch = ii.make_config(1)
+    B, T, A = cfg.B, cfg.T, cfg.A
+    clean = {k: torch.from_numpy(v).cuda() for k, v in batch.items()}
+    dirty = {k: v.clone() for k, v in clean.items()}
+    dirty["learner_logits"][3, 10, 2] = float("nan")
+    dirty["rewards"][7, 20] = float("inf")
+    dirty["target_logits"][9, 0, 0] = float("-inf")  # a target probability of exactly 0: legal
+    coef = P.to_coef(P.f32_hyper(cfg.hyper))
+    res = []
+    for t in (clean, dirty):
+        out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.zeros(B, T, A, device="cuda"),
+                   dvalues=torch.zeros(B, T, device="cuda"), advantage=torch.zeros(B, T, device="cuda"))
+        ws = ip.new_workspace(B, T)
+        ip.impact_loss_fwd_bwd(t["learner_logits"], t["target_logits"], t["worker_logp"], t["actions"], t["rewards"],
+                               t["discounts"], t["values"], t["bootstrap_values"], coef, workspace=ws, **out)
+        torch.cuda.synchronize()
+        assert ip.impact_loss_workspace_status(ws) == 0
+        res.append(out)
+    c, d = res
+    assert torch.isfinite(c["dlogits"]).all() and torch.isfinite(c["loss_terms"]).all()
+    assert torch.isnan(d["dlogits"][3, 10]).all()           # the row with the NaN logit
+    assert not torch.isfinite(d["advantage"][7, 20])        # the step with the infinite reward ...
+    assert not torch.isfinite(d["advantage"][7, :21]).any() or cfg.hyper.c_bar == 0  # ... and the steps before it
+    assert not torch.isfinite(d["loss_terms"][0])           # the batch means carry it
+    per_tile = 128 // T
+    hit = {b_ // per_tile for b_ in (3, 7)}
+    untouched = [b for b in range(B) if b // per_tile not in hit and b != 9]
+    assert torch.equal(d["dlogits"][untouched], c["dlogits"][untouched])
+    assert torch.equal(d["dvalues"][untouched], c["dvalues"][untouched])
+    assert torch.isfinite(d["dlogits"][9]).all()            # -inf target logit: probability 0, finite everything
+
+
+def test_out_of_range_actions_are_clamped():
+    """Actions outside [0, A) are clamped into range by the kernels (the oracle refuses them): the outputs are
+    those of the batch with the clamped actions, bit for bit."""
+    import paper_1912_00167_b200 as ip
+    for (B, T, A) in ((6, 40, 18), (5, 30, 33), (4, 200, 6)):
+        batch = ii.categorical_batch(B, T, A, seed=31 + A)
+        t = {k: torch.from_numpy(v).cuda() for k, v in batch.items()}
+        bad = t["actions"].clone()
+        bad[0, 0], bad[1, 5], bad[2, T - 1] = -3, A, A + 1000
+        outs = []
+        for act in (bad, bad.clamp(0, A - 1)):
+            out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.zeros(B, T, A, device="cuda"),
+                       dvalues=torch.zeros(B, T, device="cuda"))
+            ip.impact_loss_fwd_bwd(t["learner_logits"], t["target_logits"], t["worker_logp"], act, t["rewards"],
+                                   t["discounts"], t["values"], t["bootstrap_values"], ip.Coefficients(kl_coef=0.1),
+                                   workspace=ip.new_workspace(B, T), **out)
+            torch.cuda.synchronize()
+            outs.append(out)
+        for k in outs[0]:
+            assert torch.equal(outs[0][k], outs[1][k]), k
+
+
 @pytest.mark.parametrize("B,T,A", [(300, 64, 64), (7, 128, 64), (3, 200, 64), (1500, 20, 64), (33, 63, 64)])
 @pytest.mark.parametrize("dtype", [torch.float32, torch.bfloat16])
 def test_wide_rows_in_the_persistent_kernel(oracle, B, T, A, dtype):
