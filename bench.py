@@ -38,9 +38,33 @@ FALLBACK_HBM_GBS = 6650.0
 FIELD_NAMES = ["actions", "rewards", "discounts", "worker_logp", "target_logits"]
 N_DISTINCT = 4    # distinct synthetic batches generated on the host
 N_SETS = 16       # rotating learner-output / gradient buffer sets (footprint beyond L2)
-# dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel, from the ncu capture
-# summarised under profiles/ (None while the kernel has changed since the counters were taken)
-NCU_TRAFFIC_BYTES = 21567000  # dram read + write of one loss launch on config 2, from an ncu capture of this kernel
+TRAFFIC_RECORD = os.path.join(ROOT, "profiles", "loss_kernel_traffic.json")
+
+
+def kernel_sources_digest() -> str:
+    """SHA-256 over the library's CUDA sources and public header: what a traffic figure is valid for."""
+    import hashlib
+    h = hashlib.sha256()
+    csrc = os.path.join(ROOT, "paper_1912_00167_b200", "csrc")
+    files = sorted(os.path.join(csrc, f) for f in os.listdir(csrc) if f.endswith((".cu", ".cuh", ".h")))
+    files.append(os.path.join(ROOT, "include", "impact.h"))
+    for path in files:
+        with open(path, "rb") as f:
+            h.update(os.path.basename(path).encode() + b"\0" + f.read())
+    return h.hexdigest()
+
+
+def recorded_traffic():
+    """dram__bytes_read.sum + dram__bytes_write.sum of one launch of the timed kernel, from the ncu capture summarised
+    under profiles/ -- or None once a kernel source has changed since the counters were taken."""
+    try:
+        with open(TRAFFIC_RECORD) as f:
+            rec = json.load(f)
+        if rec.get("sources_sha256") == kernel_sources_digest():
+            return int(rec["dram_bytes_per_launch"])
+    except Exception:
+        pass
+    return None
 
 
 def algorithmic_bytes_per_step(A: int, logits_bytes: int = 4, grad_bytes: int = 4) -> int:
@@ -113,18 +137,43 @@ class ClockSampler:
                 "samples": len(sm), "reasons": sorted(reasons)}
 
 
-def time_oracle(batch, hyper, min_seconds: float, max_reps: int):
-    """Times the oracle, as it stands, on repeated full batches of the workload."""
+def host_cores() -> int:
+    try:
+        return max(1, len(os.sched_getaffinity(0)))
+    except AttributeError:
+        return max(1, os.cpu_count() or 1)
+
+
+def time_oracle(batch, hyper, min_seconds: float, max_reps: int, threads: int = 1):
+    """Times the oracle, as it stands, on repeated full batches of the workload.  With `threads` > 1 the batch's
+    trajectories (independent of one another) are cut into that many slices and the unchanged oracle runs on every
+    slice at once: its C routine is called through ctypes, which releases the interpreter lock."""
     import oracle
     oracle.build()
-    oracle.loss_categorical(batch, hyper)  # page in
+    B = batch["rewards"].shape[0]
+    threads = max(1, min(threads, B))
+    bounds = [(B * i // threads, B * (i + 1) // threads) for i in range(threads)]
+    slices = [{k: np.ascontiguousarray(v[lo:hi]) for k, v in batch.items()} for lo, hi in bounds]
+    pool = None
+    if threads > 1:
+        from concurrent.futures import ThreadPoolExecutor
+        pool = ThreadPoolExecutor(max_workers=threads)
+
+    def once():
+        if pool is None:
+            oracle.loss_categorical(slices[0], hyper)
+        else:
+            list(pool.map(lambda sl: oracle.loss_categorical(sl, hyper), slices))
+    once()  # page in
     reps, t0 = 0, time.perf_counter()
     while True:
-        oracle.loss_categorical(batch, hyper)
+        once()
         reps += 1
         el = time.perf_counter() - t0
         if el >= min_seconds or reps >= max_reps:
             break
+    if pool is not None:
+        pool.shutdown()
     M = batch["rewards"].size
     return reps * M / el, reps, el
 
@@ -149,25 +198,32 @@ def run_reference(args):
     cfg, batch = ii.make_config(WORKLOAD_IDX)
     import oracle
     oracle.build()
-    # each step is a bounded sample of the workload: the first 128 of its 1024 trajectories
+    # each step is a bounded sample of the workload: the first 128 of its 1024 trajectories, cut into one slice per
+    # host core (trajectories are independent), the unchanged oracle running on all slices at once
+    from concurrent.futures import ThreadPoolExecutor
     sample_B = min(128, cfg.B)
-    batch = {k: np.ascontiguousarray(v[:sample_B]) for k, v in batch.items()}
+    cores = min(host_cores(), sample_B)
+    bounds = [(sample_B * i // cores, sample_B * (i + 1) // cores) for i in range(cores)]
+    slices = [{k: np.ascontiguousarray(v[lo:hi]) for k, v in batch.items()} for lo, hi in bounds]
     M = sample_B * cfg.T
-    for _ in range(args.warmup):
-        oracle.loss_categorical(batch, cfg.hyper)
-    t0 = time.perf_counter()
-    for _ in range(args.steps):
-        oracle.loss_categorical(batch, cfg.hyper)
-    el = time.perf_counter() - t0
+    with ThreadPoolExecutor(max_workers=cores) as pool:
+        def step():
+            list(pool.map(lambda sl: oracle.loss_categorical(sl, cfg.hyper), slices))
+        for _ in range(args.warmup):
+            step()
+        t0 = time.perf_counter()
+        for _ in range(args.steps):
+            step()
+        el = time.perf_counter() - t0
     value = args.steps * M / el
     line = {
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
         "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * el / args.steps,
         "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64", "data": "synthetic",
         "config": {"workload": f"config 2: categorical B={cfg.B} T={cfg.T} A={cfg.A} fp32 (loss + gradients only)"},
-        "cpu_baseline": {"value": value, "unit": UNIT, "cores": 1, "kind": "oracle",
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": cores, "kind": "oracle",
                          "sample": f"{args.steps} steps of {sample_B} of the workload's {cfg.B} trajectories "
-                                   f"({M} timesteps each)"},
+                                   f"({M} timesteps each), one slice of trajectories per core"},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
         "gpu_launches": 0,
     }
@@ -333,6 +389,59 @@ def run_sweep(args):
             rows.append(dict(kind="ring+loss", A=A, T=T, B=B, timesteps=B * T, dtype="fp32", N=N, K=K,
                              us_per_launch=ms * 1e3, timesteps_per_s=B * T / (ms * 1e-3)))
             ring.close()
+    # the ring's own data movement at the config-2 slot size (11.5 MB per slot): bytes read + bytes written per second
+    fields0 = fields[0]
+    slot_bytes = sum(t.numel() * t.element_size() for t in fields0)
+    ring = ip.ImpactBuffer(8, 1000000, [t.numel() * t.element_size() for t in fields0], seed=3)
+    srcs = [[b[n] for n in FIELD_NAMES] for b in batches]
+    for i in range(8):
+        ring.push(srcs[i], sid)
+    gather_dst = [[torch.empty_like(t) for t in fields0] for _ in range(4)]
+
+    def time_op(fn, n=200):
+        for i in range(8):
+            fn(i)
+        torch.cuda.synchronize()
+        best = None
+        for _ in range(3):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(stream)
+            for i in range(n):
+                fn(i)
+            b.record(stream)
+            torch.cuda.synchronize()
+            ms = a.elapsed_time(b) / n
+            best = ms if best is None else min(best, ms)
+        return best
+
+    def ring_row(name, ms, moved):
+        rows.append(dict(kind=name, A=A, T=T, B=B, timesteps=B * T, dtype="bytes", us_per_launch=ms * 1e3,
+                         timesteps_per_s=B * T / (ms * 1e-3), gbs=2 * moved / (ms * 1e-3) / 1e9,
+                         frac_of_peak=2 * moved / (ms * 1e-3) / 1e9 / peak))
+    # push of a whole batch from device memory: every slot is live, so a slot is freed by hand first (host state only)
+    state0 = ring.export_state()
+
+    def push_op(i):
+        ring.import_state(state_free)
+        ring.push(srcs[i % 8], sid)
+    import struct
+    hdr = struct.calcsize("<IIiiiiiiQQ")
+    blob = bytearray(state0)
+    blob[hdr:hdr + 4] = struct.pack("<i", 0)  # slot 0 not valid: the next push lands there
+    state_free = bytes(blob)
+    ring_row("ring push (device source)", time_op(push_op), slot_bytes)
+    ring.import_state(state0)
+    tl = fields0[4]
+    ring_row("ring append (target logits)", time_op(lambda i: ring.append(i % 8, 4, batches[i % 8]["target_logits"], sid)),
+             tl.numel() * tl.element_size())
+    ring_row("ring sample + gather", time_op(lambda i: ring.sample(gather_dst[i % 4], sid)), slot_bytes)
+    # index gather of trajectory rows: B rows of T*A logits each, drawn from 8 B source rows
+    src_rows = torch.cat([b["target_logits"] for b in batches[:4]], 0)
+    idx = torch.randint(0, src_rows.shape[0], (B,), device="cuda", dtype=torch.int32)
+    dst_rows = [torch.empty(B, T, A, device="cuda") for _ in range(4)]
+    ring_row("gather_rows (B rows of T*A logits)", time_op(lambda i: ip.impact_gather_rows(src_rows, idx, dst_rows[i % 4])),
+             dst_rows[0].numel() * 4)
+    ring.close()
     out_path = args.sweep_out
     with open(out_path, "w") as f:
         json.dump({"peak_gbs": peak, "peak_kind": peak_kind, "rows": rows}, f, indent=1)
@@ -480,21 +589,37 @@ def main():
         barrier()
         return a.elapsed_time(b)
 
-    # ---- timed region: K learner iterations, whole-step throughput -----------------------------------------
+    # ---- timed region: blocks of K learner iterations, whole-step throughput ---------------------------------
+    # One block is exactly K steps between two events (barrier + synchronize on both sides).  Blocks are repeated
+    # until at least 0.2 s have been timed (at least three, at most 200), and the MEDIAN block is reported: a single
+    # 20-step block lasts a third of a millisecond, too short to carry a number.
     sampler = ClockSampler(local_rank)
     sampler.start()
     time.sleep(0.25)
     for c in counters:
         counters[c] = counters[c] if c == "pushed" else 0
-    t_wall0 = time.perf_counter()
+
+    def check_workspaces(where):
+        """A loss launch whose bounded wait gave up has untrustworthy outputs: no number is reported past one."""
+        for ws_ in (workspace, workspace2):
+            flag = ip.impact_loss_workspace_status(ws_)
+            if flag != 0:
+                raise SystemExit(f"bench.py: a loss kernel gave up a bounded wait ({where}); workspace error word {flag}")
 
     def run_steps():
         for _ in range(args.steps):
             step()
-    ms_total = time_on_stream(run_steps)
-    t_wall = time.perf_counter() - t_wall0
-    launches = counters["loss"] + counters["copy"]
-    loss_launches = counters["loss"]
+    block_ms, wall_s = [], []
+    while len(block_ms) < 3 or (sum(block_ms) < 200.0 and len(block_ms) < 200):
+        t_wall0 = time.perf_counter()
+        block_ms.append(time_on_stream(run_steps))
+        wall_s.append(time.perf_counter() - t_wall0)
+    check_workspaces("learner iterations")
+    ms_total = statistics.median(block_ms)
+    t_wall = statistics.median(wall_s)
+    n_blocks = len(block_ms)
+    launches = (counters["loss"] + counters["copy"]) // n_blocks
+    loss_launches = counters["loss"] // n_blocks
 
     # ---- the loss kernel alone: back-to-back launches over the rotating slots ---------------------------------
     # (a) issued from this host loop; (b) the same launches captured once in a CUDA graph, so that no host
@@ -532,6 +657,41 @@ def main():
     graph2.replay()
     dense_ms = min(time_on_stream(graph1.replay) for _ in range(5)) / n_dense
     overlap_ms = min(time_on_stream(graph2.replay) for _ in range(5)) / n_dense
+    check_workspaces("back-to-back loss launches")
+
+    # ---- what a batch of this size allows at all: the same bytes through plain 16-byte loads and stores (read the
+    # inputs' 21.5 MB, write the outputs' 10 MB), launched and timed exactly like the loss kernel above
+    per_in = (2 * A * 4 + 5 * 4) * M
+    per_out = (A * 4 + 4) * M
+    copy_src = [torch.empty(per_in, dtype=torch.uint8, device="cuda").random_(0, 255) for _ in range(N_SETS)]
+    copy_dst = [torch.empty(per_out, dtype=torch.uint8, device="cuda") for _ in range(N_SETS)]
+    copy_calls = [ip.prepare_stream_copy(copy_src[i], per_in, copy_dst[i], per_out) for i in range(N_SETS)]
+    graph3 = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        for c_ in copy_calls:
+            c_.on_stream(side.cuda_stream)
+        with torch.cuda.graph(graph3, stream=side):
+            for i in range(n_dense):
+                copy_calls[i % N_SETS].on_stream(side.cuda_stream)
+    torch.cuda.synchronize()
+    graph3.replay()
+    copy_ms = min(time_on_stream(graph3.replay) for _ in range(5)) / n_dense
+    del copy_calls, copy_src, copy_dst
+
+    # ---- one launch by itself: nothing before it on the device, L2 flushed (a 256 MB fill) before every launch
+    flush = torch.empty(256 << 20, dtype=torch.uint8, device="cuda")
+    iso = []
+    for i in range(12):
+        flush.fill_(i & 0xFF)
+        torch.cuda.synchronize()
+        a_, b_ = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a_.record(stream)
+        calls[i % N].on_stream(stream_id)
+        b_.record(stream)
+        torch.cuda.synchronize()
+        iso.append(a_.elapsed_time(b_))
+    iso_ms = statistics.median(iso[2:])
+    del flush
 
     # ---- the same kernel on a batch eight times as large (B*T = 1,048,576): start-up and drain amortised ----
     big = None
@@ -577,16 +737,21 @@ def main():
     dst = {k: torch.empty_like(v, device="cuda") for k, v in pinned.items()}
     out = out_sets[0]
     terms_host = torch.empty(8).pin_memory()
+    grads_host = {k_: torch.empty(out[k_].shape, dtype=out[k_].dtype).pin_memory() for k_ in ("dlogits", "dvalues")}
     e2e_call = ip.prepare_loss_fwd_bwd(dst["learner_logits"], dst["target_logits"], dst["worker_logp"],
                                        dst["actions"], dst["rewards"], dst["discounts"], dst["values"],
                                        dst["bootstrap_values"], coef, workspace=workspace, **out)
     h2d = sum(v.numel() * v.element_size() for v in pinned.values())
+    d2h = 32 + sum(v.numel() * v.element_size() for v in grads_host.values())
 
     def e2e_step():
+        # everything a caller without device-resident data pays: inputs in, loss terms AND gradients out
         for k_, v in pinned.items():
             dst[k_].copy_(v, non_blocking=True)
         e2e_call.on_stream(stream_id)
         terms_host.copy_(out["loss_terms"], non_blocking=True)
+        for k_, v in grads_host.items():
+            v.copy_(out[k_], non_blocking=True)
         stream.synchronize()
 
     for _ in range(3):
@@ -597,10 +762,11 @@ def main():
         e2e_step()
     barrier()
     e2e_s = time.perf_counter() - t0
+    check_workspaces("end-to-end steps")
 
     # ---- reduce over ranks: the slowest rank sets the time ---------------------------------------------------
-    (ms_total, e2e_s, loop_ms, dense_ms, overlap_ms), value = aggregate_over_ranks(
-        [ms_total, e2e_s, loop_ms, dense_ms, overlap_ms], args.steps, M, world, dist, "cuda")
+    (ms_total, e2e_s, loop_ms, dense_ms, overlap_ms, copy_ms, iso_ms), value = aggregate_over_ranks(
+        [ms_total, e2e_s, loop_ms, dense_ms, overlap_ms, copy_ms, iso_ms], args.steps, M, world, dist, "cuda")
     e2e_value = world * e2e_steps * M / e2e_s
 
     peak, peak_kind = peak_hbm_gbs()
@@ -610,13 +776,18 @@ def main():
     roofline = {
         "bound": "hbm", "kernel": "impact_loss_categorical_ws_kernel<float,float,18>",
         "achieved": achieved, "peak": peak, "unit": "GB/s", "frac": achieved / peak, "peak_kind": peak_kind,
-        "traffic": NCU_TRAFFIC_BYTES,
+        "traffic": recorded_traffic(),
         "algorithmic_bytes_per_launch": bytes_per_launch,
         "avg_launch_us": dense_ms * 1e3,
         "how": f"{n_dense} back-to-back loss launches over the rotating ring slots, captured in one CUDA graph; "
                "CUDA events on the launch stream around the replay, best of 5",
         "host_loop": {"avg_launch_us": loop_ms * 1e3, "achieved": gbs(loop_ms), "frac": gbs(loop_ms) / peak,
                       "how": "the same launches issued one by one from the Python loop"},
+        "copy_same_bytes": {"avg_launch_us": copy_ms * 1e3, "achieved": gbs(copy_ms), "frac": gbs(copy_ms) / peak,
+                            "how": "a plain 16-byte load/store kernel moving the same bytes (21.5 MB read, 10 MB "
+                                   "written per launch), same rotating footprint, same graph replay: what a batch of "
+                                   "this size allows with no arithmetic at all"},
+        "isolated_launch_us": iso_ms * 1e3,
         "two_streams": {"avg_launch_us": overlap_ms * 1e3, "achieved": gbs(overlap_ms), "frac": gbs(overlap_ms) / peak,
                         "how": "the same launches alternating between two streams (a workspace each): "
                                "throughput with two batches in flight, not one launch's duration"},
@@ -639,18 +810,26 @@ def main():
             "l2": f"inputs larger than L2: ring {ring.storage_bytes(N, field_bytes) >> 20} MiB + {N_SETS} "
                   f"learner-output sets + {N_SETS} gradient sets, rotated",
             "host_wall_ms_per_step": 1e3 * t_wall / args.steps,
+            "timing": f"median of {n_blocks} blocks of {args.steps} steps each (repeated until 0.2 s were timed)",
         },
+        "workspace_status": 0,
         "clocks": clocks,
-        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": 32,
-                "steps": e2e_steps},
+        "e2e": {"value": e2e_value, "unit": UNIT, "h2d_bytes_per_step": h2d, "d2h_bytes_per_step": d2h,
+                "steps": e2e_steps,
+                "what": "every input of the batch copied in from pinned host memory, the loss call, then the eight loss "
+                        "terms, dlogits and dvalues copied back to pinned host memory, each step"},
         "gpu_launches": launches,
         "gpu_launches_loss": loss_launches,
         "roofline": roofline,
     }
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        v, reps, el = time_oracle(host[0], h, min_seconds=10.0, max_reps=200)
-        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": 1, "kind": "oracle",
-                                "sample": f"{reps} full batches of {M} timesteps (loss + gradients), {el:.1f} s"}
+        cores = host_cores()
+        v1, reps1, el1 = time_oracle(host[0], h, min_seconds=5.0, max_reps=200)
+        v, reps, el = time_oracle(host[0], h, min_seconds=8.0, max_reps=4000, threads=cores)
+        line["cpu_baseline"] = {"value": v, "unit": UNIT, "cores": cores, "kind": "oracle",
+                                "sample": f"{reps} full batches of {M} timesteps (loss + gradients), {el:.1f} s, the "
+                                          f"batch's trajectories cut into one slice per core",
+                                "single_core": {"value": v1, "sample": f"{reps1} full batches, {el1:.1f} s"}}
     if rank == 0:
         print(json.dumps(line))
     ring.close()

@@ -415,6 +415,15 @@ int32_t impact_buffer_import_state(impact_buffer* h, const void* blob, size_t bl
 int32_t impact_gather_rows(const void* src, const int32_t* idx, int64_t n, int64_t n_src_rows,
                            size_t row_bytes, void* dst, void* stream);
 
+/*
+ * Measurement aid (no counterpart in the paper): reads read_bytes from src and writes the first write_bytes of
+ * them to dst with plain 16-byte loads and stores -- the byte mix of a loss launch with no arithmetic in between,
+ * launched the way the loss kernels are.  The benchmark times it beside the loss kernel to show what a batch of
+ * that size allows at all.  src, dst device, 16-byte aligned; sizes multiples of 16, 16 <= write_bytes <=
+ * read_bytes; the ranges must not overlap.
+ */
+int32_t impact_stream_copy(const void* src, size_t read_bytes, void* dst, size_t write_bytes, void* stream);
+
 #ifdef __cplusplus
 }
 #endif

@@ -34,7 +34,7 @@ EXPORTS = (
     "impact_buffer_slot_ptr", "impact_buffer_live", "impact_buffer_state_bytes",
     "impact_buffer_export_state", "impact_buffer_import_state", "impact_gather_rows",
     "impact_loss_fwd_bwd_static_scratch", "impact_loss_fwd_bwd_call", "impact_loss_workspace_status",
-    "impact_set_option", "impact_get_option", "impact_loss_static_scratch_status",
+    "impact_set_option", "impact_get_option", "impact_loss_static_scratch_status", "impact_stream_copy",
 )
 OPT_EARLY_PREFETCH, OPT_PREFETCH_BYTES, OPT_WINDOW_BYTES = 0, 1, 2
 
@@ -124,6 +124,8 @@ def load_library() -> ctypes.CDLL:
     lib.impact_gather_rows.argtypes = [_vp, _vp, _i64, _i64, _sz, _vp, _vp]
     lib.impact_loss_static_scratch_status.restype = _i32
     lib.impact_loss_static_scratch_status.argtypes = [ctypes.POINTER(_i32), _i32, _vp]
+    lib.impact_stream_copy.restype = _i32
+    lib.impact_stream_copy.argtypes = [_vp, _sz, _vp, _sz, _vp]
     lib.impact_set_option.restype = _i32
     lib.impact_set_option.argtypes = [_i32, _i64]
     lib.impact_get_option.restype = _i64
@@ -365,6 +367,16 @@ def impact_gather_rows(src: torch.Tensor, idx: torch.Tensor, dst: torch.Tensor, 
         raise ValueError("dst must hold one source row per index")
     _check(load_library().impact_gather_rows(src.data_ptr(), idx.data_ptr(), n, src.shape[0], row_bytes,
                                              dst.data_ptr(), _stream(stream)), "impact_gather_rows")
+
+
+def prepare_stream_copy(src: torch.Tensor, read_bytes: int, dst: torch.Tensor, write_bytes: int) -> PreparedCall:
+    """impact_stream_copy with its arguments marshalled once (a measurement aid: see include/impact.h)."""
+    if not (src.is_cuda and dst.is_cuda and src.is_contiguous() and dst.is_contiguous()):
+        raise ValueError("impact_stream_copy needs dense CUDA tensors")
+    if src.numel() * src.element_size() < read_bytes or dst.numel() * dst.element_size() < write_bytes:
+        raise ValueError("buffers smaller than the byte counts")
+    return PreparedCall(load_library().impact_stream_copy, [src.data_ptr(), read_bytes, dst.data_ptr(), write_bytes, 0],
+                        "impact_stream_copy", (src, dst))
 
 
 class ImpactBuffer:

@@ -85,6 +85,30 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const V* __restrict__ 
     }
 }
 
+// Reads `n_read` 16-byte units and writes `n_write` of them back out (n_write <= n_read): a loss launch's byte mix
+// with no arithmetic in between.  What is read but not written is folded into one word per thread that is stored
+// only if it has an impossible value, so that the loads cannot be dropped.
+__global__ void __launch_bounds__(256) stream_copy_kernel(const uint4* __restrict__ src, unsigned long long n_read,
+                                                          uint4* __restrict__ dst, unsigned long long n_write,
+                                                          unsigned int* __restrict__ sink) {
+    grid_dependency_wait();
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    unsigned int fold = 0;
+    constexpr int U = 4;
+    for (unsigned long long v = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; v < n_read; v += U * stride) {
+        uint4 x[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            x[u] = (v + u * stride < n_read) ? __ldcs(src + v + u * stride) : make_uint4(0u, 0u, 0u, 0u);
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            if (v + u * stride < n_write) dst[v + u * stride] = x[u];
+            else fold |= x[u].x ^ x[u].y ^ x[u].z ^ x[u].w;
+        }
+    }
+    if (fold == 0xFFFFFFFFu && n_read == 1) *sink = fold;  // (never: keeps the unwritten loads alive)
+}
+
 int blocks_for(unsigned long long work_items, int per_thread, const DeviceInfo* di) {
     unsigned long long blocks = (work_items + 256ull * per_thread - 1) / (256ull * per_thread);
     const unsigned long long cap = (unsigned long long)di->sm_count * 8ull;
@@ -375,5 +399,18 @@ extern "C" int32_t impact_gather_rows(const void* src, const int32_t* idx, int64
                                           static_cast<const unsigned char*>(src), idx, (long long)n, (long long)n_src_rows, units, static_cast<unsigned char*>(dst)));
     }
     IMPACT_CUDA_TRY(cudaGetLastError());
+    return IMPACT_OK;
+}
+
+extern "C" int32_t impact_stream_copy(const void* src, size_t read_bytes, void* dst, size_t write_bytes, void* stream) {
+    if (!src || !dst || !aligned16(src) || !aligned16(dst) || read_bytes == 0 || write_bytes > read_bytes ||
+        (read_bytes & 15u) != 0 || (write_bytes & 15u) != 0 || write_bytes < 16)
+        return IMPACT_ERR_INVALID_ARG;
+    const DeviceInfo* di = current_device_info();
+    if (!di) return IMPACT_ERR_CUDA;
+    const unsigned long long n_read = read_bytes / 16, n_write = write_bytes / 16;
+    IMPACT_CUDA_TRY(launch_serialized(stream_copy_kernel, dim3(blocks_for(n_read, 4, di)), dim3(256), 0,
+                                      static_cast<cudaStream_t>(stream), static_cast<const uint4*>(src), n_read,
+                                      static_cast<uint4*>(dst), n_write, reinterpret_cast<unsigned int*>(dst)));
     return IMPACT_OK;
 }
