@@ -621,6 +621,48 @@ def main():
     launches = (counters["loss"] + counters["copy"]) // n_blocks
     loss_launches = counters["loss"] // n_blocks
 
+    # ---- the same learner iteration with the ring's bookkeeping on the device, captured into a CUDA graph ------
+    # (push-if-a-slot-is-free, draw, loss with its inputs named by the draw's record; the host only replays)
+    ring_dev = ip.ImpactBuffer(N, K, field_bytes, seed=cfg.seed + 1)
+    n_cand = len(worker_batches)
+    table = torch.tensor([[wb[0].data_ptr(), wb[1].data_ptr(), wb[2].data_ptr(), wb[3].data_ptr(), 0, wb[4].data_ptr()]
+                          for wb in worker_batches], dtype=torch.int64, device="cuda")
+    record = ip.new_loss_inputs_record()
+    fmap = {n_: f_ for f_, n_ in enumerate(FIELD_NAMES)}
+    ls0 = learner_sets[0]
+    dev_step = ring_dev.prepare_device_step(fmap, ls0["learner_logits"], ls0["values"], ls0["bootstrap_values"],
+                                            push_sources=table, record=record)
+    dev_loss = ip.prepare_loss_fwd_bwd_from_record(record, B, T, A, torch.float32, coef, workspace=workspace,
+                                                   **out_sets[0])
+    ring_dev.device_begin()
+    dev_stream = torch.cuda.Stream()
+    n_graph = 64
+    with torch.cuda.stream(dev_stream):
+        for _ in range(2 * N):  # fills the ring (one push per iteration until every slot is live)
+            dev_step.on_stream(dev_stream.cuda_stream)
+            dev_loss.on_stream(dev_stream.cuda_stream)
+    torch.cuda.synchronize()
+    graph_dev = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(dev_stream):
+        with torch.cuda.graph(graph_dev, stream=dev_stream):
+            for _ in range(n_graph):
+                dev_step.on_stream(dev_stream.cuda_stream)
+                dev_loss.on_stream(dev_stream.cuda_stream)
+    torch.cuda.synchronize()
+    graph_dev.replay()
+    dev_ms, dev_wall = [], []
+    for _ in range(7):
+        t0_ = time.perf_counter()
+        dev_ms.append(time_on_stream(graph_dev.replay))
+        dev_wall.append(time.perf_counter() - t0_)
+    check_workspaces("device-bookkeeping iterations")
+    dev_events = ring_dev.device_events()
+    assert all(e[1] in (0, -5) for e in dev_events), "the device ring ran empty"
+    dev_iter_ms = statistics.median(dev_ms) / n_graph
+    dev_wall_ms = statistics.median(dev_wall) / n_graph * 1e3
+    ring_dev.device_end()
+    ring_dev.close()
+
     # ---- the loss kernel alone: back-to-back launches over the rotating slots ---------------------------------
     # (a) issued from this host loop; (b) the same launches captured once in a CUDA graph, so that no host
     # time sits between them; (c) alternating between two streams (a workspace each), so that one launch's
@@ -811,6 +853,12 @@ def main():
                   f"learner-output sets + {N_SETS} gradient sets, rotated",
             "host_wall_ms_per_step": 1e3 * t_wall / args.steps,
             "timing": f"median of {n_blocks} blocks of {args.steps} steps each (repeated until 0.2 s were timed)",
+            "device_bookkeeping": {
+                "ms_per_step": dev_iter_ms, "host_wall_ms_per_step": dev_wall_ms,
+                "how": f"the same iteration with the ring's bookkeeping in device memory (impact_buffer_device_step: "
+                       f"push if a slot is free, draw, loss with its inputs named by the draw's record), {n_graph} "
+                       f"iterations captured in one CUDA graph and replayed; learner outputs in one fixed set of "
+                       f"buffers, the ring's {N} slots in HBM"},
         },
         "workspace_status": 0,
         "clocks": clocks,

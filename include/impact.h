@@ -225,6 +225,7 @@ int32_t impact_loss_fwd_bwd(
  * address to impact_loss_fwd_bwd_call.  Field meanings, layouts, limits and errors are those
  * of impact_loss_fwd_bwd; `coef` is embedded by value.
  */
+struct impact_loss_inputs;
 typedef struct impact_loss_call {
     const void* learner_logits;
     const void* target_logits;
@@ -252,6 +253,13 @@ typedef struct impact_loss_call {
                                  the loss kernel itself, which has the rows in shared memory anyway, instead of by a
                                  copy of its own.  Typically a slot of the circular buffer
                                  (impact_buffer_slot_ptr).  Must not overlap any other argument. */
+    const struct impact_loss_inputs* inputs_on_device; /* optional (NULL = none): DEVICE pointer to a record written by
+                                 impact_buffer_device_step earlier on the same stream.  The kernel then takes its
+                                 eight input pointers and target_logits_copy from that record (read once the stream's
+                                 previous work is complete) instead of from the fields above, which are ignored and
+                                 may be NULL.  Shapes, types and outputs come from this struct as usual.  Served by
+                                 the persistent kernel only: A in {4, 6, 9, 18, 64} and T <= 128 (64 for A = 64);
+                                 else IMPACT_ERR_UNSUPPORTED. */
 } impact_loss_call;
 
 /* impact_loss_fwd_bwd with its arguments taken from `call` (Algorithm 1, gradient step). */
@@ -404,6 +412,64 @@ int32_t impact_buffer_live(const impact_buffer* h);
 size_t impact_buffer_state_bytes(const impact_buffer* h);
 int32_t impact_buffer_export_state(const impact_buffer* h, void* blob, size_t blob_bytes);
 int32_t impact_buffer_import_state(impact_buffer* h, const void* blob, size_t blob_bytes);
+
+/*
+ * ---- bookkeeping on the device -------------------------------------------------------------------------------
+ * Algorithm 1's "Obtain batch B ... traversed k times" / "If k = K, discard batch" and the workers' "Send B_i to
+ * C(N,K)" (Section 3.2) with the slot bookkeeping kept in device memory: a learner iteration is then enqueued --
+ * or captured into a CUDA graph and replayed -- without the host ever learning a slot number.  The protocol and the
+ * draw are exactly those of impact_buffer_push / impact_buffer_sample (same trace for the same seed).
+ *
+ *   impact_buffer_device_begin   uploads the handle's bookkeeping (allocating a few kilobytes of device memory the
+ *                                first time) and switches the handle to device mode: impact_buffer_push, _sample and
+ *                                _import_state are refused until impact_buffer_device_end, which brings the
+ *                                bookkeeping back to the host (synchronises `stream`).  impact_buffer_live and
+ *                                _export_state keep working (they fetch the device's copy; synchronising).
+ *   impact_buffer_device_step    one step on `stream`, in this order:
+ *     (1) if push_sources != NULL: the next of n_candidates worker batches goes into the first free slot at or after
+ *         the write cursor; with every slot live nothing happens (IMPACT_ERR_FULL in the event log).  push_sources is
+ *         a DEVICE array of n_candidates x (n_fields + 1) pointers: for each candidate its n_fields field sources
+ *         (NULL = leave the field for the append) and one extra pointer that is remembered with the slot -- the
+ *         target network's output for that batch.  Candidates are taken in turn (pushes so far mod n_candidates).
+ *         The copy itself is a second kernel enqueued by this call.
+ *     (2) if inputs_out != NULL: a live slot is drawn, its count goes up, after the K-th traversal it is discarded,
+ *         and *inputs_out (DEVICE memory, 16-byte aligned) receives the arguments of the loss call for that batch:
+ *         the slot's fields named by `map` (-1 = not kept in the ring: NULL), learner_logits / values /
+ *         bootstrap_values as passed here (the learner network's outputs for the batch), and for the target logits
+ *         either the slot's field or -- at the batch's first traversal, when an extra pointer came with the batch --
+ *         that pointer with the slot's field as target_logits_copy (Algorithm 1, "If k = 0, evaluate B on target,
+ *         append target output to B", done by the loss call).  With no live slot status is IMPACT_ERR_EMPTY and the
+ *         pointers of the previous draw stay in place.
+ *     A loss call reads the record through impact_loss_call.inputs_on_device.  All steps and the loss calls that
+ *     use their records belong on ONE stream.
+ *   impact_buffer_device_events  the most recent outcomes, oldest first, as (op, status, slot, k_before) quadruples
+ *                                of int32 (op 1 = push, 2 = sample; up to 4096 are kept); synchronises `stream`.
+ */
+typedef struct impact_ring_field_map {
+    int32_t actions, rewards, discounts, worker_logp, target_logits; /* index of the ring field, or -1 */
+} impact_ring_field_map;
+
+typedef struct impact_loss_inputs { /* lives in DEVICE memory */
+    const void* learner_logits;
+    const void* target_logits;
+    const float* worker_logp;
+    const int32_t* actions;
+    const float* rewards;
+    const float* discounts;
+    const float* values;
+    const float* bootstrap_values;
+    void* target_logits_copy;
+    int32_t status, slot, k_before, pad;
+} impact_loss_inputs;
+
+int32_t impact_buffer_device_begin(impact_buffer* h, void* stream);
+int32_t impact_buffer_device_end(impact_buffer* h, void* stream);
+int32_t impact_buffer_device_step(impact_buffer* h, const impact_ring_field_map* map, const void* learner_logits,
+                                  const float* values, const float* bootstrap_values,
+                                  const void* const* push_sources, int32_t n_candidates,
+                                  impact_loss_inputs* inputs_out, void* stream);
+int32_t impact_buffer_device_events(impact_buffer* h, int32_t* events_out, int32_t max_events, int32_t* n_out,
+                                    void* stream);
 
 /*
  * Index gather of rows: dst[i, :] = src[idx[i], :] for i in [0, n), rows of row_bytes

@@ -9,7 +9,7 @@ from .binding import (  # noqa: F401
     impact_get_option, impact_loss_fwd_bwd_static_scratch, impact_loss_static_scratch_status, impact_set_option,
     impact_loss_workspace_bytes, impact_loss_workspace_init, impact_loss_workspace_status, impact_status_string,
     impact_version, load_library, new_workspace, prepare_loss_fwd_bwd,
-    prepare_loss_fwd_bwd_gaussian, prepare_stream_copy,
+    new_loss_inputs_record, prepare_loss_fwd_bwd_from_record, prepare_loss_fwd_bwd_gaussian, prepare_stream_copy,
 )
 from . import binding  # noqa: F401
 from .kl_controller import AdaptiveKL  # noqa: F401

@@ -35,6 +35,8 @@ EXPORTS = (
     "impact_buffer_export_state", "impact_buffer_import_state", "impact_gather_rows",
     "impact_loss_fwd_bwd_static_scratch", "impact_loss_fwd_bwd_call", "impact_loss_workspace_status",
     "impact_set_option", "impact_get_option", "impact_loss_static_scratch_status", "impact_stream_copy",
+    "impact_buffer_device_begin", "impact_buffer_device_end", "impact_buffer_device_step",
+    "impact_buffer_device_events",
 )
 OPT_EARLY_PREFETCH, OPT_PREFETCH_BYTES, OPT_WINDOW_BYTES = 0, 1, 2
 
@@ -61,7 +63,19 @@ class impact_loss_call(ctypes.Structure):
                 ("B", ctypes.c_int64), ("T", ctypes.c_int64), ("loss_terms", ctypes.c_void_p),
                 ("dlogits", ctypes.c_void_p), ("dvalues", ctypes.c_void_p), ("vtarget", ctypes.c_void_p),
                 ("advantage", ctypes.c_void_p), ("workspace", ctypes.c_void_p), ("workspace_bytes", ctypes.c_size_t),
-                ("target_logits_copy", ctypes.c_void_p)]
+                ("target_logits_copy", ctypes.c_void_p), ("inputs_on_device", ctypes.c_void_p)]
+
+
+class impact_ring_field_map(ctypes.Structure):
+    _fields_ = [(n, ctypes.c_int32) for n in ("actions", "rewards", "discounts", "worker_logp", "target_logits")]
+
+
+class impact_loss_inputs(ctypes.Structure):
+    """Layout of the record impact_buffer_device_step writes (device memory; here only for its size and for
+    reading one back in tests)."""
+    _fields_ = [(n, ctypes.c_void_p) for n in ("learner_logits", "target_logits", "worker_logp", "actions", "rewards",
+                                               "discounts", "values", "bootstrap_values", "target_logits_copy")] + \
+               [(n, ctypes.c_int32) for n in ("status", "slot", "k_before", "pad")]
 
 
 _lib = None
@@ -124,6 +138,14 @@ def load_library() -> ctypes.CDLL:
     lib.impact_gather_rows.argtypes = [_vp, _vp, _i64, _i64, _sz, _vp, _vp]
     lib.impact_loss_static_scratch_status.restype = _i32
     lib.impact_loss_static_scratch_status.argtypes = [ctypes.POINTER(_i32), _i32, _vp]
+    lib.impact_buffer_device_begin.restype = _i32
+    lib.impact_buffer_device_begin.argtypes = [_vp, _vp]
+    lib.impact_buffer_device_end.restype = _i32
+    lib.impact_buffer_device_end.argtypes = [_vp, _vp]
+    lib.impact_buffer_device_step.restype = _i32
+    lib.impact_buffer_device_step.argtypes = [_vp, ctypes.POINTER(impact_ring_field_map), _vp, _vp, _vp, _vp, _i32, _vp, _vp]
+    lib.impact_buffer_device_events.restype = _i32
+    lib.impact_buffer_device_events.argtypes = [_vp, ctypes.POINTER(_i32), _i32, ctypes.POINTER(_i32), _vp]
     lib.impact_stream_copy.restype = _i32
     lib.impact_stream_copy.argtypes = [_vp, _sz, _vp, _sz, _vp]
     lib.impact_set_option.restype = _i32
@@ -271,8 +293,34 @@ def prepare_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, re
         _dev(dvalues, f32, bt, "dvalues"), _dev(vtarget, f32, bt, "vtarget", True),
         _dev(advantage, f32, bt, "advantage", True),
         _dev(workspace, torch.uint8, workspace.shape, "workspace"), workspace.numel(),
-        _dev(target_logits_copy, ldt, (B, T, A), "target_logits_copy", True))
+        _dev(target_logits_copy, ldt, (B, T, A), "target_logits_copy", True), None)
     return PreparedCall(lib.impact_loss_fwd_bwd_call, [ctypes.byref(call), 0], "impact_loss_fwd_bwd_call", (call,))
+
+
+def new_loss_inputs_record(device="cuda") -> torch.Tensor:
+    """Device memory for one impact_loss_inputs record (written by ImpactBuffer.device_step, read by the loss call)."""
+    return torch.zeros(ctypes.sizeof(impact_loss_inputs) + 8, dtype=torch.uint8, device=device)
+
+
+def prepare_loss_fwd_bwd_from_record(record: torch.Tensor, B: int, T: int, A: int, logits_dtype: torch.dtype,
+                                     coef: Coefficients, *, loss_terms, dlogits, dvalues, vtarget=None,
+                                     advantage=None, workspace) -> PreparedCall:
+    """The loss call whose inputs are named by a device record (impact_loss_call.inputs_on_device)."""
+    lib = load_library()
+    if logits_dtype not in _DTYPE_CODE or dlogits.dtype not in _DTYPE_CODE:
+        raise ValueError("logits must be float32 or bfloat16")
+    if not record.is_cuda or record.numel() * record.element_size() < ctypes.sizeof(impact_loss_inputs):
+        raise ValueError("record: device memory of at least sizeof(impact_loss_inputs) bytes")
+    f32, bt = torch.float32, (B, T)
+    cs = coef.c_struct(_DTYPE_CODE[dlogits.dtype])
+    call = impact_loss_call(
+        None, None, None, None, None, None, None, None,
+        coef.rho_bar, coef.c_bar, coef.clip_eps, _DTYPE_CODE[logits_dtype], cs, A, B, T,
+        _dev(loss_terms, f32, (NUM_TERMS,), "loss_terms"), _dev(dlogits, dlogits.dtype, (B, T, A), "dlogits"),
+        _dev(dvalues, f32, bt, "dvalues"), _dev(vtarget, f32, bt, "vtarget", True),
+        _dev(advantage, f32, bt, "advantage", True),
+        _dev(workspace, torch.uint8, workspace.shape, "workspace"), workspace.numel(), None, record.data_ptr())
+    return PreparedCall(lib.impact_loss_fwd_bwd_call, [ctypes.byref(call), 0], "impact_loss_fwd_bwd_call", (call, record))
 
 
 def impact_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
@@ -476,6 +524,43 @@ class ImpactBuffer:
 
     def import_state(self, blob: bytes) -> None:
         _check(self._lib.impact_buffer_import_state(self._h, blob, len(blob)), "impact_buffer_import_state")
+
+    # ---- bookkeeping on the device -------------------------------------------------------------------------
+    def device_begin(self, stream=None) -> None:
+        _check(self._lib.impact_buffer_device_begin(self._h, _stream(stream)), "impact_buffer_device_begin")
+
+    def device_end(self, stream=None) -> None:
+        _check(self._lib.impact_buffer_device_end(self._h, _stream(stream)), "impact_buffer_device_end")
+
+    def prepare_device_step(self, field_map=None, learner_logits=None, values=None, bootstrap_values=None,
+                            push_sources: torch.Tensor | None = None, record: torch.Tensor | None = None) -> PreparedCall:
+        """impact_buffer_device_step with its arguments marshalled once.  field_map: dict name -> ring field index
+        (missing = not in the ring); push_sources: int64 CUDA tensor [n_candidates, n_fields + 1] of device addresses
+        (0 = none); record: from new_loss_inputs_record()."""
+        fm = None
+        if record is not None:
+            m = field_map or {}
+            fm = impact_ring_field_map(*[int(m.get(n, -1)) for n in ("actions", "rewards", "discounts", "worker_logp",
+                                                                      "target_logits")])
+        ncand = 0
+        if push_sources is not None:
+            if not push_sources.is_cuda or push_sources.dtype != torch.int64 or push_sources.dim() != 2 or \
+                    push_sources.shape[1] != self.n_fields + 1 or not push_sources.is_contiguous():
+                raise ValueError("push_sources: contiguous int64 CUDA tensor [n_candidates, n_fields + 1]")
+            ncand = push_sources.shape[0]
+        ptr = lambda t: None if t is None else t.data_ptr()
+        args = [self._h, ctypes.byref(fm) if fm is not None else None, ptr(learner_logits), ptr(values),
+                ptr(bootstrap_values), ptr(push_sources), ncand, ptr(record), 0]
+        return PreparedCall(self._lib.impact_buffer_device_step, args, "impact_buffer_device_step",
+                            (fm, learner_logits, values, bootstrap_values, push_sources, record))
+
+    def device_events(self, max_events: int = 4096, stream=None):
+        """The most recent (op, status, slot, k_before) outcomes, oldest first (op 1 = push, 2 = sample)."""
+        buf = (_i32 * (4 * max_events))()
+        n = _i32(0)
+        _check(self._lib.impact_buffer_device_events(self._h, buf, max_events, ctypes.byref(n), _stream(stream)),
+               "impact_buffer_device_events")
+        return [tuple(buf[4 * i:4 * i + 4]) for i in range(n.value)]
 
     def close(self) -> None:
         if self._h:

@@ -47,6 +47,7 @@ struct CatParams {
     unsigned long long* tagged_rows;  // persistent kernel: rows of (value, launch tag) pairs, see dev::publish_tagged
     unsigned long long* tile_aggregates;  // persistent kernel, T > 128: two (value, launch tag) pairs per tile
     void* target_copy;  // persistent kernel: where the target logits are written as well (NULL = nowhere)
+    const impact_loss_inputs* indirect;  // persistent kernel: device record that overrides the nine pointers above (NULL = none)
     TileGeometry geo;
     LossScalars k;
     int A, As;
@@ -1000,6 +1001,35 @@ struct RowMath {
 // Rows wider than 32 actions are not held in registers: every pass streams the row from shared memory, the
 // gradient pass forms the exponentials again, and thread r starts its walk at pair r mod (A/2), because a row
 // pitch of 256 bytes would otherwise put all threads of a warp on the same banks.
+struct LossInputPointers {
+    const void* learner_logits;
+    const void* target_logits;
+    const float* worker_logp;
+    const int32_t* actions;
+    const float* rewards;
+    const float* discounts;
+    const float* values;
+    const float* bootstrap;
+    void* target_copy;
+};
+// The record of impact_buffer_device_step, read past L1 (an earlier launch may have left an older version there).
+__device__ __forceinline__ LossInputPointers fetch_loss_inputs(const impact_loss_inputs* rec) {
+    const ulonglong2* q = reinterpret_cast<const ulonglong2*>(rec);
+    const ulonglong2 a = __ldcg(q), b = __ldcg(q + 1), c = __ldcg(q + 2), d = __ldcg(q + 3);
+    const unsigned long long e = __ldcg(reinterpret_cast<const unsigned long long*>(q + 4));
+    LossInputPointers in;
+    in.learner_logits = reinterpret_cast<const void*>(a.x);
+    in.target_logits = reinterpret_cast<const void*>(a.y);
+    in.worker_logp = reinterpret_cast<const float*>(b.x);
+    in.actions = reinterpret_cast<const int32_t*>(b.y);
+    in.rewards = reinterpret_cast<const float*>(c.x);
+    in.discounts = reinterpret_cast<const float*>(c.y);
+    in.values = reinterpret_cast<const float*>(d.x);
+    in.bootstrap = reinterpret_cast<const float*>(d.y);
+    in.target_copy = reinterpret_cast<void*>(e);
+    return in;
+}
+
 // Barrier protocol of the persistent kernels (S stages, at most W tiles in flight, lanes <= S - W):
 //   full[s]     one arrival (a producer lane's, with the bytes the tile's two copies will deliver): stage s holds
 //               the rows of its current tile.
@@ -1019,7 +1049,7 @@ struct RowMath {
 // Without the in-order rule (lanes that found their own tile ready first went first) the first argument fails for
 // tiles of one round: a consumer could be handed a stage whose previous tile had not landed, read stale rows,
 // release the stage early, and the phases slipped until one of the bounded waits ran out.
-template <typename LT, typename GT, int A, int C, bool kPlain, bool kLong, int NT>
+template <typename LT, typename GT, int A, int C, bool kPlain, bool kLong, int NT, bool kIndirect>
 __global__ void __launch_bounds__(C * NT + 32, 1)
 impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W, const int lanes,
                                   const int n_prefetch) {
@@ -1048,6 +1078,12 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     const long long total_rows = g.B * g.T;
     const long long agg_stride = g.tile_major ? 2 * g.B : 2;  // slots between a tile's aggregate and that of the tile after it in time
     auto place_of = [&](int n) { return tile_place<kLong, NT>(g, n, rows_full, total_rows); };
+    // The tensors this launch reads: the call's own arguments (kernel parameters, read where they are used), or --
+    // kIndirect: the call names a record in device memory that an earlier kernel of the stream fills (the circular
+    // buffer's bookkeeping on the device) -- that record's, fetched by every thread once the stream dependency has
+    // resolved.
+    LossInputPointers in = {};
+#define IMPACT_IN(field) (kIndirect ? in.field : p.field)
 
     if (tid >= C * NT) {
         // ---- producer warp ----------------------------------------------------------------------------------
@@ -1058,13 +1094,13 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         if (n_prefetch > 0) {
             const void* base = nullptr;
             long long pitch = 4;
-            if (lane == 0) { base = p.learner_logits; pitch = kInRow; }
-            else if (lane == 1) { base = p.target_logits; pitch = kInRow; }
-            else if (lane == 2) base = p.actions;
-            else if (lane == 3) base = p.worker_logp;
-            else if (lane == 4) base = p.rewards;
-            else if (lane == 5) base = p.discounts;
-            else if (lane == 6) base = p.values;
+            if (lane == 0) { base = IMPACT_IN(learner_logits); pitch = kInRow; }
+            else if (lane == 1) { base = IMPACT_IN(target_logits); pitch = kInRow; }
+            else if (lane == 2) base = IMPACT_IN(actions);
+            else if (lane == 3) base = IMPACT_IN(worker_logp);
+            else if (lane == 4) base = IMPACT_IN(rewards);
+            else if (lane == 5) base = IMPACT_IN(discounts);
+            else if (lane == 6) base = IMPACT_IN(values);
             const int n_pf = n_tiles < n_prefetch ? n_tiles : n_prefetch;
             for (int n = 0; n < n_pf; ++n) {
                 const Place pc = place_of(n);
@@ -1097,8 +1133,8 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             const dev::WideRange w = dev::widen_range(pc.row0 * (long long)kInRow, (uint32_t)pc.nrows * kInRow, tensor_bytes);
             SlabRequest r;
             r.d0 = smem_raw + s * kStageBytes;  // the tile's first row starts (row0 * kInRow) mod 16 bytes in
-            r.gl = static_cast<const unsigned char*>(p.learner_logits) + w.first;
-            r.gt = static_cast<const unsigned char*>(p.target_logits) + w.first;
+            r.gl = static_cast<const unsigned char*>(IMPACT_IN(learner_logits)) + w.first;
+            r.gt = static_cast<const unsigned char*>(IMPACT_IN(target_logits)) + w.first;
             r.span = w.span;
             r.tail = w.tail;
             return r;
@@ -1131,10 +1167,14 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         const bool second = lane >= 16;
         // the first W tiles need no wait (tile n goes to stage n): their requests are worked out now and leave the
         // moment the stream's previous kernel is done, before the rest of the block has even started
-        const SlabRequest first = request_for(place_of(sub < n_first ? sub : 0), sub);
+        SlabRequest first = request_for(place_of(sub < n_first ? sub : 0), sub);
 
         grid_dependency_wait();
 
+        if (kIndirect) {  // (the addresses were not known before)
+            in = fetch_loss_inputs(p.indirect);
+            first = request_for(place_of(sub < n_first ? sub : 0), sub);
+        }
         if (sub < n_first) send_slab(first, sub, second);
         __syncthreads();  // the barriers are set up: the consumer warps may use them
         // The rest.  Tile n goes to stage n % S once that stage's previous tile has left (the "empty" phase before
@@ -1210,13 +1250,13 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         x.a = 0; x.l_worker = 0.0f; x.reward = 0.0f; x.discount = 0.0f; x.value = 0.0f; x.value_next = 0.0f;
         if (m.active) {
             const long long r = m.row;
-            const int a = p.actions[r];
+            const int a = IMPACT_IN(actions)[r];
             x.a = min(max(a, 0), A - 1);
-            x.l_worker = p.worker_logp[r];
-            x.reward = p.rewards[r];
-            x.discount = p.discounts[r];
-            x.value = p.values[r];
-            x.value_next = m.last_step ? p.bootstrap[m.traj] : p.values[r + 1];
+            x.l_worker = IMPACT_IN(worker_logp)[r];
+            x.reward = IMPACT_IN(rewards)[r];
+            x.discount = IMPACT_IN(discounts)[r];
+            x.value = IMPACT_IN(values)[r];
+            x.value_next = m.last_step ? IMPACT_IN(bootstrap)[m.traj] : IMPACT_IN(values)[r + 1];
         }
         return x;
     };
@@ -1234,6 +1274,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     int pending_stage = 0;
 
     grid_dependency_wait();
+    if (kIndirect) in = fetch_loss_inputs(p.indirect);
     Mine me = mine_in(grp);
     StepRaw cur = load_scalars(me);
     __syncthreads();  // the producer warp has set up the barriers
@@ -1277,10 +1318,10 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         bool stored = false;  // lane 0: a bulk store of this warp reads the stage
         // (first traversal of a batch) the target rows go to the circular buffer as well, each warp's 32 rows
         // straight from the stage, which nothing writes to
-        if (p.target_copy) {
+        if (IMPACT_IN(target_copy)) {
             const int left = me.pc.nrows - (gtid - lane);
             const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
-            unsigned char* const dst = static_cast<unsigned char*>(p.target_copy) + (me.row - lane) * (long long)kInRow;
+            unsigned char* const dst = static_cast<unsigned char*>(IMPACT_IN(target_copy)) + (me.row - lane) * (long long)kInRow;
             stored = dev::warp_send_bytes(dst, s1 + (gtid - lane) * kInRow, (uint32_t)wrows * kInRow, false);
         }
         const int a = cur.a;
@@ -1500,6 +1541,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             if (gtid == 0) atomicExch(p.counter + 1, 1u);
     }
     if (lane == 0) dev::bulk_store_wait_read();  // shared memory must outlive the stores' reads
+#undef IMPACT_IN
 }
 
 // ------------------------------------------------------------------------------------------
@@ -2425,7 +2467,11 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     // Wide rows (A = 64): tiles of 64 steps, six groups of 64 threads.
     constexpr int NT = ws_tile_rows(A);
     constexpr int C = A > 32 ? 6 : (!kPlain ? kWsGroups : (A <= 9 ? kWsGroups + 2 : kWsGroups + 1));
-    auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong, NT>;
+    // (inputs named by a device record: compiled for trajectories that fit a tile only)
+    if (p.indirect && kLong) return IMPACT_ERR_UNSUPPORTED;
+    auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong, NT, false>;
+    if constexpr (!kLong)
+        if (p.indirect) kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong, NT, true>;
     const size_t stage = ws_stage_bytes<LT, GT, A, NT>();
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
     long long grid = tiles < di->sm_count ? tiles : di->sm_count;
@@ -2435,17 +2481,20 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     if (S < 1 || W < 1) return IMPACT_ERR_UNSUPPORTED;
 
     const size_t smem = (size_t)S * stage;
-    static thread_local int configured_device = -1;
-    if (configured_device != di->device) {  // once per device: room for the largest ring any window setting asks for
+    static thread_local int configured_device[2] = {-1, -1};
+    int& configured = configured_device[p.indirect ? 1 : 0];
+    if (configured != di->device) {  // once per device: room for the largest ring any window setting asks for
         IMPACT_CUDA_TRY(cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, di->max_smem_optin - 4096));
-        configured_device = di->device;
+        configured = di->device;
     }
     const int lanes = (S - W) < 4 ? ((S - W) < 1 ? 1 : (S - W)) : 4;  // producer lanes that request tiles side by side
     CatParams q = p;
     // tile-major once every block has a trajectory of its own: the aggregates a tile needs are then a round old
     q.geo.tile_major = (kLong && p.geo.B >= grid) ? 1 : 0;
     const int rows_full = kLong ? NT : q.geo.G * (int)q.geo.T;
-    const WsPlan plan = ws_plan(tiles, grid, (size_t)rows_full * (2 * A * sizeof(LT) + 20), W, true);
+    WsPlan plan_ = ws_plan(tiles, grid, (size_t)rows_full * (2 * A * sizeof(LT) + 20), W, true);
+    if (p.indirect) { plan_.companion = false; plan_.prefetch_tiles = 0; }  // (addresses unknown on the host)
+    const WsPlan plan = plan_;
     if (plan.companion) {
         PrefetchList pf = {};
         const void* bases[7] = {p.learner_logits, p.target_logits, p.actions, p.worker_logp, p.rewards, p.discounts, p.values};
@@ -2486,6 +2535,7 @@ int32_t launch_categorical_reg(const CatParams& p, const DeviceInfo* di, cudaStr
         // with trajectories for every consumer group of the device the sweep inside a block is a little faster still
         if (p.tile_aggregates && p.geo.B < (long long)kWsGroups * di->sm_count)
             return launch_categorical_ws<LT, GT, A, false, true>(p, di, stream);
+        if (p.indirect) return IMPACT_ERR_UNSUPPORTED;  // the sweeping kernel takes its pointers from the call only
         auto kernel = impact_loss_categorical_reg_kernel<LT, GT, A>;
         const size_t smem = reg_kernel_smem<LT, GT, A>();
         int grid = 0;
@@ -2533,6 +2583,7 @@ int32_t run_categorical(CatParams& p, int64_t B, int64_t T, bool logits_bf16, bo
         if (logits_bf16 && !grads_bf16) return dispatch_reg<__nv_bfloat16, float>(p, di, s);
         return dispatch_reg<__nv_bfloat16, __nv_bfloat16>(p, di, s);
     }
+    if (p.indirect) return IMPACT_ERR_UNSUPPORTED;  // inputs named by a device record: the persistent kernel only
     p.As = p.A;
     const int nt = categorical_tile_rows(p.A, logits_bf16, grads_bf16, long_without_aggregates);
     p.geo = make_geometry(B, T, nt);
@@ -2655,10 +2706,18 @@ static int32_t loss_fwd_bwd_impl(
     const float* bootstrap_values, float rho_bar, float c_bar, float clip_eps,
     const impact_coefficients* coef, int64_t B, int64_t T, int32_t A, int32_t logits_dtype,
     float* loss_terms, void* dlogits, float* dvalues, float* vtarget, float* advantage,
-    void* workspace, size_t workspace_bytes, void* target_logits_copy, void* stream) {
-    if (!learner_logits || !target_logits || !worker_logp || !actions || !rewards || !discounts ||
-        !values || !bootstrap_values || !coef || !loss_terms || !dlogits || !dvalues || !workspace)
+    void* workspace, size_t workspace_bytes, void* target_logits_copy, const impact_loss_inputs* indirect, void* stream) {
+    if (!coef || !loss_terms || !dlogits || !dvalues || !workspace) return IMPACT_ERR_INVALID_ARG;
+    if (indirect) {  // the inputs come from a record in device memory: the pointers passed here are not looked at
+        if (!aligned16(indirect)) return IMPACT_ERR_INVALID_ARG;
+        learner_logits = target_logits = nullptr;
+        worker_logp = rewards = discounts = values = bootstrap_values = nullptr;
+        actions = nullptr;
+        target_logits_copy = nullptr;
+    } else if (!learner_logits || !target_logits || !worker_logp || !actions || !rewards || !discounts || !values ||
+               !bootstrap_values) {
         return IMPACT_ERR_INVALID_ARG;
+    }
     if (B <= 0 || T <= 0 || A <= 0) return IMPACT_ERR_INVALID_ARG;
     const void* ptrs[] = {learner_logits, target_logits, worker_logp, actions, rewards, discounts,
                           values, bootstrap_values, loss_terms, dlogits, dvalues, workspace};
@@ -2704,6 +2763,7 @@ static int32_t loss_fwd_bwd_impl(
                             ? reinterpret_cast<unsigned long long*>(static_cast<char*>(workspace) + kWorkspaceFixedBytes)
                             : nullptr;
     p.target_copy = target_logits_copy;
+    p.indirect = indirect;
     p.A = A;
     return run_categorical(p, B, T, logits_dtype == IMPACT_DTYPE_BF16, coef->dlogits_dtype == IMPACT_DTYPE_BF16,
                            di, static_cast<cudaStream_t>(stream));
@@ -2718,7 +2778,7 @@ extern "C" int32_t impact_loss_fwd_bwd(
     void* workspace, size_t workspace_bytes, void* stream) {
     return loss_fwd_bwd_impl(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
                              bootstrap_values, rho_bar, c_bar, clip_eps, coef, B, T, A, logits_dtype, loss_terms,
-                             dlogits, dvalues, vtarget, advantage, workspace, workspace_bytes, nullptr, stream);
+                             dlogits, dvalues, vtarget, advantage, workspace, workspace_bytes, nullptr, nullptr, stream);
 }
 
 extern "C" int32_t impact_loss_fwd_bwd_call(const impact_loss_call* c, void* stream) {
@@ -2727,7 +2787,7 @@ extern "C" int32_t impact_loss_fwd_bwd_call(const impact_loss_call* c, void* str
                              c->discounts, c->values, c->bootstrap_values, c->rho_bar, c->c_bar, c->clip_eps,
                              &c->coef, c->B, c->T, c->A, c->logits_dtype, c->loss_terms, c->dlogits,
                              c->dvalues, c->vtarget, c->advantage, c->workspace, c->workspace_bytes,
-                             c->target_logits_copy, stream);
+                             c->target_logits_copy, c->inputs_on_device, stream);
 }
 
 extern "C" int32_t impact_loss_fwd_bwd_gaussian(

@@ -109,6 +109,192 @@ __global__ void __launch_bounds__(256) stream_copy_kernel(const uint4* __restric
     if (fold == 0xFFFFFFFFu && n_read == 1) *sink = fold;  // (never: keeps the unwritten loads alive)
 }
 
+// ---- bookkeeping resident on the device ---------------------------------------------------------------------
+// The same few integers per slot as on the host, in device memory, so that a learner iteration -- push a worker
+// batch into a free slot, obtain a batch, loss and gradients -- can be enqueued (or captured into a CUDA graph)
+// without the host ever seeing a slot number.  One warp does the bookkeeping; it is the protocol of
+// impact_buffer_push / impact_buffer_sample statement by statement (docs/ring_protocol.md), so both modes give the
+// same trace for the same seed.
+struct RingDeviceHeader {
+    int32_t write_cursor, read_cursor;
+    uint32_t n_events, pad;
+    uint64_t draws, pushes;
+};
+constexpr int kEventLog = 4096;  // the most recent push / sample outcomes, for the host to read back
+constexpr int kMaxDeviceSlots = 1024;  // slots a buffer may have for its bookkeeping to go to the device
+
+struct RingDeviceView {
+    RingDeviceHeader* hd;
+    int32_t* valid;
+    int32_t* count;
+    uint64_t* fresh;   // per slot: the extra pointer that came with the batch pushed into it
+    int4* events;      // (op, status, slot, k_before); op 1 = push, 2 = sample
+    CopySegments* plan;
+    char* storage;
+    unsigned long long slot_stride;
+    unsigned long long field_offset[kMaxFields], field_bytes[kMaxFields];
+    int32_t N, K, n_fields, mode;
+    uint64_t seed;
+};
+
+__device__ __forceinline__ uint64_t splitmix64_at_dev(uint64_t seed, uint64_t n) {
+    uint64_t z = seed + (n + 1) * 0x9E3779B97F4A7C15ull;
+    z ^= z >> 30; z *= 0xBF58476D1CE4E5B9ull;
+    z ^= z >> 27; z *= 0x94D049BB133111EBull;
+    z ^= z >> 31;
+    return z;
+}
+
+// One learner-side step of the bookkeeping: (1) if `sources` is given, the next candidate batch goes into the
+// first free slot at or after the write cursor (none free: nothing happens, the event says FULL), and the copy
+// that the following kernel performs is written to `plan`; (2) a live slot is drawn and the inputs of the loss
+// call are resolved into `inputs`.
+__global__ void __launch_bounds__(32) ring_step_kernel(const RingDeviceView v, const impact_ring_field_map map,
+                                                       const void* learner_logits, const float* values,
+                                                       const float* bootstrap_values, const void* const* sources,
+                                                       int32_t n_candidates, int32_t do_sample,
+                                                       impact_loss_inputs* inputs) {
+    grid_dependency_wait();
+    // the slots' flags and counts are staged in shared memory by the whole warp (one trip to L2 instead of one per
+    // slot); lane 0 then walks them exactly as the host code does and writes back what it changed
+    __shared__ int32_t valid_s[kMaxDeviceSlots], count_s[kMaxDeviceSlots];
+    for (int32_t i = threadIdx.x; i < v.N; i += 32) {
+        valid_s[i] = v.valid[i];
+        count_s[i] = v.count[i];
+    }
+    RingDeviceHeader hd = *v.hd;
+    // (the candidate's pointers too: lane f fetches the f-th, all at once)
+    __shared__ const void* cand_s[kMaxFields + 1];
+    if (sources && (int)threadIdx.x <= v.n_fields)
+        cand_s[threadIdx.x] = sources[(size_t)(hd.pushes % (uint64_t)n_candidates) * (size_t)(v.n_fields + 1) + threadIdx.x];
+    __syncwarp();
+    if (threadIdx.x != 0) return;
+    v.plan->n = 0;
+    if (sources) {
+        int32_t slot = -1;
+        for (int32_t i = 0; i < v.N; ++i) {
+            const int32_t s = (hd.write_cursor + i) % v.N;
+            if (!valid_s[s]) { slot = s; break; }
+        }
+        if (slot >= 0) {
+            const void* const* cand = cand_s;
+            int n = 0;
+            unsigned long long units = 0;
+            for (int f = 0; f < v.n_fields; ++f) {
+                if (!cand[f]) continue;
+                v.plan->src[n] = static_cast<const char*>(cand[f]);
+                v.plan->dst[n] = v.storage + (unsigned long long)slot * v.slot_stride + v.field_offset[f];
+                v.plan->bytes[n] = v.field_bytes[f];
+                units += (v.field_bytes[f] + 15ull) / 16ull;
+                v.plan->vec_end[n] = units;
+                ++n;
+            }
+            v.plan->n = n;
+            v.fresh[slot] = reinterpret_cast<uint64_t>(cand[v.n_fields]);
+            valid_s[slot] = 1;
+            count_s[slot] = 0;
+            v.valid[slot] = 1;
+            v.count[slot] = 0;
+            hd.write_cursor = (slot + 1) % v.N;
+            hd.pushes += 1;
+        }
+        v.events[hd.n_events++ % kEventLog] = make_int4(1, slot >= 0 ? IMPACT_OK : IMPACT_ERR_FULL, slot, 0);
+    }
+    if (do_sample) {
+        int32_t live = 0;
+        for (int32_t s = 0; s < v.N; ++s) live += valid_s[s] ? 1 : 0;
+        int32_t pick = -1;
+        if (live > 0) {
+            if (v.mode == IMPACT_SAMPLE_UNIFORM) {
+                const uint64_t u = splitmix64_at_dev(v.seed, hd.draws++);
+                uint64_t j = __umul64hi(u, (uint64_t)live);  // floor(u * live / 2^64)
+                for (int32_t s = 0; s < v.N; ++s) {
+                    if (!valid_s[s]) continue;
+                    if (j == 0) { pick = s; break; }
+                    --j;
+                }
+            } else {
+                for (int32_t i = 0; i < v.N; ++i) {
+                    const int32_t s = (hd.read_cursor + i) % v.N;
+                    if (valid_s[s]) { pick = s; break; }
+                }
+                hd.read_cursor = (pick + 1) % v.N;
+            }
+        }
+        int32_t k_before = 0;
+        if (pick >= 0) {
+            k_before = count_s[pick];
+            v.count[pick] = k_before + 1;
+            if (k_before + 1 >= v.K) v.valid[pick] = 0;
+            auto field = [&](int32_t f) -> const void* {
+                return f >= 0 ? v.storage + (unsigned long long)pick * v.slot_stride + v.field_offset[f] : nullptr;
+            };
+            impact_loss_inputs in;
+            in.learner_logits = learner_logits;
+            in.values = values;
+            in.bootstrap_values = bootstrap_values;
+            in.actions = static_cast<const int32_t*>(field(map.actions));
+            in.rewards = static_cast<const float*>(field(map.rewards));
+            in.discounts = static_cast<const float*>(field(map.discounts));
+            in.worker_logp = static_cast<const float*>(field(map.worker_logp));
+            const void* in_slot = field(map.target_logits);
+            const void* fresh = reinterpret_cast<const void*>(v.fresh[pick]);
+            if (k_before == 0 && fresh && in_slot) {  // first traversal: the target network's output is appended now
+                in.target_logits = fresh;
+                in.target_logits_copy = const_cast<void*>(in_slot);
+            } else {
+                in.target_logits = in_slot;
+                in.target_logits_copy = nullptr;
+            }
+            in.status = IMPACT_OK;
+            in.slot = pick;
+            in.k_before = k_before;
+            in.pad = 0;
+            *inputs = in;
+        } else {
+            inputs->status = IMPACT_ERR_EMPTY;  // the pointers of the previous draw stay in place
+        }
+        v.events[hd.n_events++ % kEventLog] = make_int4(2, pick >= 0 ? IMPACT_OK : IMPACT_ERR_EMPTY, pick, k_before);
+    }
+    *v.hd = hd;
+}
+
+// multi_copy_kernel with its segments read from device memory (an empty plan copies nothing).
+__global__ void __launch_bounds__(256) multi_copy_planned_kernel(const CopySegments* plan) {
+    grid_dependency_wait();
+    const int n = plan->n;
+    if (n == 0) return;
+    const unsigned long long total = plan->vec_end[n - 1];
+    const unsigned long long stride = (unsigned long long)gridDim.x * blockDim.x;
+    constexpr int U = 4;
+    for (unsigned long long v0 = (unsigned long long)blockIdx.x * blockDim.x + threadIdx.x; v0 < total; v0 += U * stride) {
+        uint4 x[U];
+        char* out[U];
+#pragma unroll
+        for (int u = 0; u < U; ++u) {
+            const unsigned long long vu = v0 + u * stride;
+            out[u] = nullptr;
+            if (vu < total) {
+                int f = 0;
+                while (vu >= plan->vec_end[f]) ++f;
+                const unsigned long long off = (vu - (f ? plan->vec_end[f - 1] : 0ull)) * 16ull;
+                const char* src = plan->src[f] + off;
+                char* dst = plan->dst[f] + off;
+                if (off + 16ull <= plan->bytes[f]) {
+                    x[u] = __ldcs(reinterpret_cast<const uint4*>(src));
+                    out[u] = dst;
+                } else {
+                    const int tail = (int)(plan->bytes[f] - off);
+                    for (int i = 0; i < tail; ++i) dst[i] = src[i];
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < U; ++u)
+            if (out[u]) __stcs(reinterpret_cast<uint4*>(out[u]), x[u]);
+    }
+}
+
 int blocks_for(unsigned long long work_items, int per_thread, const DeviceInfo* di) {
     unsigned long long blocks = (work_items + 256ull * per_thread - 1) / (256ull * per_thread);
     const unsigned long long cap = (unsigned long long)di->sm_count * 8ull;
@@ -152,6 +338,31 @@ struct impact_buffer {
     size_t slot_stride = 0;
     char* storage = nullptr;
     bool owns_storage = false;
+    // bookkeeping on the device (impact_buffer_device_begin): one allocation, laid out as
+    // [header | valid N | count N | fresh N | events | copy plan]
+    char* device_state = nullptr;
+    bool device_mode = false;
+    size_t device_state_bytes() const {
+        return align_up16(sizeof(RingDeviceHeader)) + align_up16(sizeof(int32_t) * (size_t)N) * 2 +
+               align_up16(sizeof(uint64_t) * (size_t)N) + sizeof(int4) * (size_t)kEventLog + align_up16(sizeof(CopySegments));
+    }
+    static size_t align_up16(size_t x) { return (x + 15) / 16 * 16; }
+    RingDeviceView view() const {
+        RingDeviceView v;
+        char* p = device_state;
+        v.hd = reinterpret_cast<RingDeviceHeader*>(p); p += align_up16(sizeof(RingDeviceHeader));
+        v.valid = reinterpret_cast<int32_t*>(p); p += align_up16(sizeof(int32_t) * (size_t)N);
+        v.count = reinterpret_cast<int32_t*>(p); p += align_up16(sizeof(int32_t) * (size_t)N);
+        v.fresh = reinterpret_cast<uint64_t*>(p); p += align_up16(sizeof(uint64_t) * (size_t)N);
+        v.events = reinterpret_cast<int4*>(p); p += sizeof(int4) * (size_t)kEventLog;
+        v.plan = reinterpret_cast<CopySegments*>(p);
+        v.storage = storage;
+        v.slot_stride = slot_stride;
+        for (int f = 0; f < kMaxFields; ++f) { v.field_offset[f] = field_offset[f]; v.field_bytes[f] = field_bytes[f]; }
+        v.N = N; v.K = K; v.n_fields = n_fields; v.mode = mode;
+        v.seed = seed;
+        return v;
+    }
 
     char* field_ptr(int32_t slot, int32_t f) const {
         return storage + (size_t)slot * slot_stride + field_offset[f];
@@ -207,9 +418,10 @@ extern "C" int32_t impact_buffer_create(int32_t N, int32_t K, int32_t n_fields, 
 extern "C" int32_t impact_buffer_destroy(impact_buffer* h) {
     if (!h) return IMPACT_ERR_INVALID_ARG;
     int32_t st = IMPACT_OK;
-    if (h->owns_storage) {
+    if (h->owns_storage || h->device_state) {
         cudaError_t e = cudaDeviceSynchronize();
-        if (e == cudaSuccess) e = cudaFree(h->storage);
+        if (e == cudaSuccess && h->owns_storage) e = cudaFree(h->storage);
+        if (e == cudaSuccess && h->device_state) e = cudaFree(h->device_state);
         if (e != cudaSuccess) st = record_cuda_error(e);
     }
     delete h;
@@ -236,7 +448,7 @@ static void add_segment(CopySegments& s, const void* src, void* dst, size_t byte
 
 extern "C" int32_t impact_buffer_push(impact_buffer* h, const void* const* field_src, int32_t src_location,
                                       int32_t* slot_out, void* stream) {
-    if (!h || !field_src || !slot_out) return IMPACT_ERR_INVALID_ARG;
+    if (!h || !field_src || !slot_out || h->device_mode) return IMPACT_ERR_INVALID_ARG;
     if (src_location != IMPACT_SRC_DEVICE && src_location != IMPACT_SRC_HOST) return IMPACT_ERR_INVALID_ARG;
     if (src_location == IMPACT_SRC_DEVICE)
         for (int f = 0; f < h->n_fields; ++f)
@@ -270,7 +482,7 @@ extern "C" int32_t impact_buffer_push(impact_buffer* h, const void* const* field
 
 extern "C" int32_t impact_buffer_sample(impact_buffer* h, int32_t* slot_out, int32_t* k_before_out,
                                         void* const* gather_dst, void* stream) {
-    if (!h || !slot_out || !k_before_out) return IMPACT_ERR_INVALID_ARG;
+    if (!h || !slot_out || !k_before_out || h->device_mode) return IMPACT_ERR_INVALID_ARG;
     if (gather_dst)
         for (int f = 0; f < h->n_fields; ++f)
             if (gather_dst[f] && !aligned16(gather_dst[f])) return IMPACT_ERR_INVALID_ARG;
@@ -328,8 +540,112 @@ extern "C" void* impact_buffer_slot_ptr(impact_buffer* h, int32_t slot, int32_t 
     return h->field_ptr(slot, field);
 }
 
+// Brings the host copy of the bookkeeping up to date with the device's (device mode only); synchronises `stream`.
+static int32_t download_state(impact_buffer* h, cudaStream_t cs) {
+    const RingDeviceView v = h->view();
+    RingDeviceHeader hd;
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(&hd, v.hd, sizeof(hd), cudaMemcpyDeviceToHost, cs));
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(h->valid.data(), v.valid, sizeof(int32_t) * (size_t)h->N, cudaMemcpyDeviceToHost, cs));
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(h->count.data(), v.count, sizeof(int32_t) * (size_t)h->N, cudaMemcpyDeviceToHost, cs));
+    IMPACT_CUDA_TRY(cudaStreamSynchronize(cs));
+    h->write_cursor = hd.write_cursor;
+    h->read_cursor = hd.read_cursor;
+    h->draws = hd.draws;
+    return IMPACT_OK;
+}
+
+extern "C" int32_t impact_buffer_device_begin(impact_buffer* h, void* stream) {
+    if (!h || h->device_mode) return IMPACT_ERR_INVALID_ARG;
+    if (h->N > kMaxDeviceSlots) return IMPACT_ERR_UNSUPPORTED;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    if (!h->device_state) {
+        void* mem = nullptr;
+        IMPACT_CUDA_TRY(cudaMalloc(&mem, h->device_state_bytes()));
+        h->device_state = static_cast<char*>(mem);
+    }
+    IMPACT_CUDA_TRY(cudaMemsetAsync(h->device_state, 0, h->device_state_bytes(), cs));
+    const RingDeviceView v = h->view();
+    RingDeviceHeader hd = {};
+    hd.write_cursor = h->write_cursor;
+    hd.read_cursor = h->read_cursor;
+    hd.draws = h->draws;
+    // (pageable sources: the copies have read them when the calls return)
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(v.hd, &hd, sizeof(hd), cudaMemcpyHostToDevice, cs));
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(v.valid, h->valid.data(), sizeof(int32_t) * (size_t)h->N, cudaMemcpyHostToDevice, cs));
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(v.count, h->count.data(), sizeof(int32_t) * (size_t)h->N, cudaMemcpyHostToDevice, cs));
+    h->device_mode = true;
+    return IMPACT_OK;
+}
+
+extern "C" int32_t impact_buffer_device_end(impact_buffer* h, void* stream) {
+    if (!h || !h->device_mode) return IMPACT_ERR_INVALID_ARG;
+    const int32_t st = download_state(h, static_cast<cudaStream_t>(stream));
+    if (st != IMPACT_OK) return st;
+    h->device_mode = false;
+    return IMPACT_OK;
+}
+
+extern "C" int32_t impact_buffer_device_step(impact_buffer* h, const impact_ring_field_map* map,
+                                             const void* learner_logits, const float* values,
+                                             const float* bootstrap_values, const void* const* push_sources,
+                                             int32_t n_candidates, impact_loss_inputs* inputs_out, void* stream) {
+    if (!h || !h->device_mode) return IMPACT_ERR_INVALID_ARG;
+    if (push_sources && (n_candidates < 1 || (reinterpret_cast<uintptr_t>(push_sources) & 7u) != 0)) return IMPACT_ERR_INVALID_ARG;
+    impact_ring_field_map m = {-1, -1, -1, -1, -1};
+    if (inputs_out) {
+        if (!map || !aligned16(inputs_out)) return IMPACT_ERR_INVALID_ARG;
+        m = *map;
+        const int32_t* fs = &m.actions;
+        for (int i = 0; i < 5; ++i)
+            if (fs[i] < -1 || fs[i] >= h->n_fields) return IMPACT_ERR_INVALID_ARG;
+    } else if (!push_sources) {
+        return IMPACT_ERR_INVALID_ARG;  // nothing to do
+    }
+    const DeviceInfo* di = current_device_info();
+    if (!di) return IMPACT_ERR_CUDA;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const RingDeviceView v = h->view();
+    IMPACT_CUDA_TRY(launch_serialized(ring_step_kernel, dim3(1), dim3(32), 0, cs, v, m, learner_logits, values,
+                                      bootstrap_values, push_sources, n_candidates, inputs_out ? 1 : 0, inputs_out));
+    if (push_sources) {
+        unsigned long long units = 0;
+        for (int f = 0; f < h->n_fields; ++f) units += (h->field_bytes[f] + 15) / 16;
+        // (a grid of two blocks per SM: most steps find every slot live and copy nothing, and an empty launch should
+        // cost as little as possible)
+        int blocks = blocks_for(units, 4, di);
+        if (blocks > 2 * di->sm_count) blocks = 2 * di->sm_count;
+        IMPACT_CUDA_TRY(launch_serialized(multi_copy_planned_kernel, dim3(blocks), dim3(256), 0, cs,
+                                          static_cast<const CopySegments*>(v.plan)));
+    }
+    return IMPACT_OK;
+}
+
+extern "C" int32_t impact_buffer_device_events(impact_buffer* h, int32_t* events_out, int32_t max_events,
+                                               int32_t* n_out, void* stream) {
+    if (!h || !h->device_mode || !events_out || !n_out || max_events < 1) return IMPACT_ERR_INVALID_ARG;
+    cudaStream_t cs = static_cast<cudaStream_t>(stream);
+    const RingDeviceView v = h->view();
+    RingDeviceHeader hd;
+    std::vector<int4> log((size_t)kEventLog);
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(&hd, v.hd, sizeof(hd), cudaMemcpyDeviceToHost, cs));
+    IMPACT_CUDA_TRY(cudaMemcpyAsync(log.data(), v.events, sizeof(int4) * (size_t)kEventLog, cudaMemcpyDeviceToHost, cs));
+    IMPACT_CUDA_TRY(cudaStreamSynchronize(cs));
+    uint32_t have = hd.n_events < (uint32_t)kEventLog ? hd.n_events : (uint32_t)kEventLog;
+    if (have > (uint32_t)max_events) have = (uint32_t)max_events;
+    for (uint32_t i = 0; i < have; ++i) {  // oldest first
+        const int4 e = log[(hd.n_events - have + i) % kEventLog];
+        events_out[4 * i + 0] = e.x; events_out[4 * i + 1] = e.y; events_out[4 * i + 2] = e.z; events_out[4 * i + 3] = e.w;
+    }
+    *n_out = (int32_t)have;
+    return IMPACT_OK;
+}
+
 extern "C" int32_t impact_buffer_live(const impact_buffer* h) {
     if (!h) return IMPACT_ERR_INVALID_ARG;
+    if (h->device_mode) {
+        const int32_t st = download_state(const_cast<impact_buffer*>(h), nullptr);
+        if (st != IMPACT_OK) return st;
+    }
     int32_t live = 0;
     for (int32_t s = 0; s < h->N; ++s) live += h->valid[s] ? 1 : 0;
     return live;
@@ -342,6 +658,10 @@ extern "C" size_t impact_buffer_state_bytes(const impact_buffer* h) {
 
 extern "C" int32_t impact_buffer_export_state(const impact_buffer* h, void* blob, size_t blob_bytes) {
     if (!h || !blob || blob_bytes < impact_buffer_state_bytes(h)) return IMPACT_ERR_INVALID_ARG;
+    if (h->device_mode) {  // the device holds the truth: fetch it (default stream; synchronises)
+        const int32_t st = download_state(const_cast<impact_buffer*>(h), nullptr);
+        if (st != IMPACT_OK) return st;
+    }
     StateHeader hd;
     memset(&hd, 0, sizeof(hd));
     hd.magic = kStateMagic; hd.version = 1;
@@ -356,7 +676,7 @@ extern "C" int32_t impact_buffer_export_state(const impact_buffer* h, void* blob
 }
 
 extern "C" int32_t impact_buffer_import_state(impact_buffer* h, const void* blob, size_t blob_bytes) {
-    if (!h || !blob || blob_bytes < impact_buffer_state_bytes(h)) return IMPACT_ERR_INVALID_ARG;
+    if (!h || !blob || blob_bytes < impact_buffer_state_bytes(h) || h->device_mode) return IMPACT_ERR_INVALID_ARG;
     StateHeader hd;
     const char* in = static_cast<const char*>(blob);
     memcpy(&hd, in, sizeof(hd));

@@ -169,3 +169,160 @@ def test_gathered_trajectories_give_the_same_loss(oracle):
     for k in b:
         np.testing.assert_array_equal(dev[k].cpu().numpy(), gathered[k])
     P.check_categorical(oracle, {k: v.cpu().numpy() for k, v in dev.items()}, cfg.hyper)
+
+
+def _ring_with_candidates(cfg_idx, n_cand, N, K, mode, seed):
+    """A ring plus `n_cand` candidate worker batches on the device and their address table for device_step."""
+    import paper_1912_00167_b200 as ip
+    names = ["actions", "rewards", "discounts", "worker_logp", "target_logits"]
+    cands = []
+    for i in range(n_cand):
+        cfg, b = ii.make_config(cfg_idx, seed=700 + i)
+        cands.append({k: torch.from_numpy(np.ascontiguousarray(v)).cuda() for k, v in b.items()})
+    fb = [cands[0][n].numel() * cands[0][n].element_size() for n in names]
+    ring = ip.ImpactBuffer(N, K, fb, seed=seed, sample_mode=mode)
+    # per candidate: the four per-step fields (the slot's target-logits field is left for the first traversal), and
+    # the candidate's fresh target logits as the pointer that is remembered with the slot
+    table = torch.tensor([[c["actions"].data_ptr(), c["rewards"].data_ptr(), c["discounts"].data_ptr(),
+                           c["worker_logp"].data_ptr(), 0, c["target_logits"].data_ptr()] for c in cands],
+                         dtype=torch.int64, device="cuda")
+    return cfg, ring, cands, table, names
+
+
+@pytest.mark.parametrize("cfg_idx,mode,N,K", [(0, 0, 2, 2), (1, 0, 16, 2), (1, 1, 5, 3), (0, 0, 7, 1)])
+def test_device_resident_bookkeeping_gives_the_oracles_trace(oracle, cfg_idx, mode, N, K):
+    """The same script of pushes and draws, the bookkeeping on the device: every outcome (FULL, EMPTY, slot,
+    traversal count) equals the oracle ring's, the slots hold the pushed bytes, the state survives the way back
+    to the host, and a host-mode continuation agrees with the oracle as well."""
+    import paper_1912_00167_b200 as ip
+    seed = 90 + N
+    cfg, ring, cands, table, names = _ring_with_candidates(cfg_idx, 3, N, K, mode, seed)
+    ref = oracle.Ring(N, K, mode, seed=seed)
+    record = ip.new_loss_inputs_record()
+    fmap = {n: f for f, n in enumerate(names)}
+    push_only = ring.prepare_device_step(push_sources=table)
+    draw_only = ring.prepare_device_step(fmap, cands[0]["learner_logits"], cands[0]["values"],
+                                         cands[0]["bootstrap_values"], record=record)
+    both = ring.prepare_device_step(fmap, cands[0]["learner_logits"], cands[0]["values"], cands[0]["bootstrap_values"],
+                                    push_sources=table, record=record)
+    ring.device_begin()
+    rng = np.random.default_rng(seed)
+    want, where, pushes = [], {}, 0
+    for step in range(120):
+        u = rng.random()
+        if u < 0.35:
+            push_only()
+            ops = ["push"]
+        elif u < 0.75:
+            draw_only()
+            ops = ["draw"]
+        else:
+            both()
+            ops = ["push", "draw"]
+        for op in ops:
+            if op == "push":
+                st, slot = ref.push()
+                want.append((1, -5 if st == ref.FULL else 0, -1 if st == ref.FULL else slot, 0))
+                if st != ref.FULL:
+                    where[slot] = pushes % 3
+                    pushes += 1
+            else:
+                st, slot, k = ref.sample()
+                want.append((2, -4, -1, 0) if st == ref.EMPTY else (2, 0, slot, k))
+    got = ring.device_events()
+    assert got == want
+    assert ring.live() == ref.live()
+    # the last successful draw's record names the slot's fields (and the fresh target logits at k = 0)
+    last = [e for e in want if e[0] == 2 and e[1] == 0][-1]
+    rec = ip.binding.impact_loss_inputs.from_buffer_copy(bytes(record.cpu().numpy())[:ip.binding.ctypes.sizeof(ip.binding.impact_loss_inputs)])
+    assert (rec.status, rec.slot, rec.k_before) == (0, last[2], last[3])
+    assert rec.actions == ring.slot_ptr(last[2], 0) and rec.worker_logp == ring.slot_ptr(last[2], 3)
+    if last[3] == 0:
+        assert rec.target_logits == cands[where[last[2]]]["target_logits"].data_ptr()
+        assert rec.target_logits_copy == ring.slot_ptr(last[2], 4)
+    else:
+        assert rec.target_logits == ring.slot_ptr(last[2], 4) and not rec.target_logits_copy
+    # payload: every live slot holds its candidate's bytes
+    torch.cuda.synchronize()
+    for slot, c in where.items():
+        for f in range(4):
+            view = ring.slot_view(slot, f, torch.uint8, (ring.field_bytes[f],))
+            assert torch.equal(view, cands[c][names[f]].view(torch.uint8).reshape(-1))
+    # back on the host the two rings keep agreeing
+    ring.device_end()
+    for _ in range(3 * N):
+        got_h = ring.sample()
+        st, slot, k = ref.sample()
+        assert (got_h is None) == (st == ref.EMPTY)
+        if got_h is not None:
+            assert got_h == (slot, k)
+    ring.close()
+
+
+def test_learner_iterations_from_a_cuda_graph_with_device_bookkeeping(oracle):
+    """Push-if-free, draw, loss with the inputs named by the draw's record: captured once into a CUDA graph and
+    replayed.  Every iteration's loss terms equal those of the ordinary call on the batch the oracle ring says was
+    drawn, and after a batch's first traversal its slot holds the target logits."""
+    import paper_1912_00167_b200 as ip
+    N, K, seed = 4, 2, 17
+    cfg, ring, cands, table, names = _ring_with_candidates(1, 3, N, K, 0, seed)
+    B, T, A = cfg.B, cfg.T, cfg.A
+    ref = oracle.Ring(N, K, 0, seed=seed)
+    learner = cands[0]  # the learner network's outputs: one fixed set of buffers
+    coef = ip.Coefficients(clip_eps=0.3)
+    ws = ip.new_workspace(B, T)
+    record = ip.new_loss_inputs_record()
+    out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
+               dvalues=torch.empty(B, T, device="cuda"))
+    fmap = {n: f for f, n in enumerate(names)}
+    step = ring.prepare_device_step(fmap, learner["learner_logits"], learner["values"], learner["bootstrap_values"],
+                                    push_sources=table, record=record)
+    loss = ip.prepare_loss_fwd_bwd_from_record(record, B, T, A, torch.float32, coef, workspace=ws, **out)
+    ring.device_begin()
+    side = torch.cuda.Stream()
+    with torch.cuda.stream(side):
+        step.on_stream(side.cuda_stream)   # (warm-up outside the capture: first-use set-up of the kernels)
+        loss.on_stream(side.cuda_stream)
+    torch.cuda.synchronize()
+    seen = [out["loss_terms"].clone()]
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(side):
+        with torch.cuda.graph(graph, stream=side):
+            step.on_stream(side.cuda_stream)
+            loss.on_stream(side.cuda_stream)
+    for _ in range(11):
+        graph.replay()
+        torch.cuda.synchronize()
+        seen.append(out["loss_terms"].clone())
+    assert ip.impact_loss_workspace_status(ws) == 0
+    # the oracle's trace for 12 iterations of push-then-draw, and the ordinary call on each drawn batch
+    where, pushes = {}, 0
+    want_out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
+                    dvalues=torch.empty(B, T, device="cuda"))
+    for it in range(12):
+        st, slot = ref.push()
+        if st != ref.FULL:
+            where[slot] = pushes % 3
+            pushes += 1
+        st, slot, k = ref.sample()
+        assert st != ref.EMPTY
+        c = cands[where[slot]]
+        ip.impact_loss_fwd_bwd(learner["learner_logits"], c["target_logits"], c["worker_logp"], c["actions"],
+                               c["rewards"], c["discounts"], learner["values"], learner["bootstrap_values"], coef,
+                               workspace=ip.new_workspace(B, T), **want_out)
+        torch.cuda.synchronize()
+        assert torch.equal(seen[it], want_out["loss_terms"]), it
+    events = ring.device_events()
+    assert len(events) == 24 and all(e[1] in (0, -5) for e in events)
+    # a slot whose current batch has been drawn holds that batch's target logits (appended by the loss call)
+    drawn_since_push = {}
+    for op, status, slot, k in events:
+        if status != 0:
+            continue
+        drawn_since_push[slot] = (op == 2) if op == 2 else False
+    for slot, was_drawn in drawn_since_push.items():
+        if was_drawn:
+            view = ring.slot_view(slot, 4, torch.float32, (B, T, A))
+            assert torch.equal(view, cands[where[slot]]["target_logits"])
+    ring.device_end()
+    ring.close()
