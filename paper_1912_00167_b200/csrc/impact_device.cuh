@@ -204,6 +204,15 @@ __device__ __forceinline__ void prefetch_range_l2(const void* base, long long by
 // whether a bulk store was issued (its group is committed; see bulk_store_wait_read).
 __device__ __forceinline__ bool warp_send_bytes(unsigned char* dst, const unsigned char* src, uint32_t bytes, bool wrote) {
     const uint32_t lane = threadIdx.x & 31u;
+    if ((((uint32_t)reinterpret_cast<uintptr_t>(dst) | bytes) & 15u) == 0u) {  // whole granules only: the usual case
+        if (wrote) fence_async_shared();
+        __syncwarp();
+        if (lane == 0 && bytes) {
+            bulk_store(dst, src, bytes);
+            return true;
+        }
+        return false;
+    }
     uint32_t head = (16u - ((uint32_t)reinterpret_cast<uintptr_t>(dst) & 15u)) & 15u;
     if (head > bytes) head = bytes;
     const uint32_t body = (bytes - head) & ~15u;

@@ -1179,8 +1179,10 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         __syncthreads();  // the barriers are set up: the consumer warps may use them
         // The rest.  Tile n goes to stage n % S once that stage's previous tile has left (the "empty" phase before
         // this one) and tile n - W has landed (at most W tiles in flight).  The owners look at their barriers side by
-        // side, but a tile is sent only when every earlier tile of the round has been sent or is sent in the same
-        // instruction: tiles leave in order.
+        // side (one thread taking tile after tile through blocking waits costs a third of a microsecond per tile, too
+        // much for small tiles: measured 33 us against 25 us on a million steps of six actions), but a tile is sent
+        // only when every earlier tile of the round has been sent or is sent in the same instruction: tiles leave in
+        // order.
         for (int base = n_first; base < n_tiles; base += lanes) {
             const int n = base + sub;
             bool pending = sub < lanes && n < n_tiles;
@@ -1224,39 +1226,45 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     // (short trajectories) the thread's place in a tile never changes: step ts of trajectory q of the tile
     int q = 0, ts = gtid;
     if (!kLong && g.G > 1) { q = gtid / (int)g.T; ts = gtid - q * (int)g.T; }
-    // this thread's row, trajectory, whether it has a row at all and whether that row ends its trajectory,
-    // in the block's n-th tile
-    struct Mine {
-        long long row, traj;
-        bool active, last_step;
-        Place pc;
+    // Where the group's next tile sits: short trajectories advance by a fixed number of rows and trajectories
+    // (C tiles of the block further on), long ones are placed tile by tile.
+    const long long group_row_stride = (long long)C * gridDim.x * rows_full;
+    const long long group_traj_stride = (long long)C * gridDim.x * g.G;
+    auto place_after = [&](const Place& pc, int n_next) {
+        if constexpr (kLong) {
+            return place_of(n_next < n_tiles ? n_next : 0);
+        } else {
+            Place pn;
+            pn.row0 = pc.row0 + group_row_stride;
+            pn.traj = pc.traj + group_traj_stride;
+            const long long left = total_rows - pn.row0;
+            pn.nrows = left < rows_full ? (left > 0 ? (int)left : 0) : rows_full;
+            pn.r = 0;
+            return pn;
+        }
     };
-    auto mine_in = [&](int n) {
-        Mine m;
-        m.pc = place_of(n < n_tiles ? n : 0);
-        m.row = m.pc.row0 + gtid;
-        m.traj = m.pc.traj + q;
-        m.active = n < n_tiles && gtid < m.pc.nrows;
-        m.last_step = kLong ? (m.pc.r == 0 && gtid == m.pc.nrows - 1) : (ts == (int)g.T - 1);
-        return m;
+    // does this thread's row end its trajectory (in the tile at `pc`)?
+    auto ends_trajectory = [&](const Place& pc) {
+        return kLong ? (pc.r == 0 && gtid == pc.nrows - 1) : (ts == (int)g.T - 1);
     };
 
     struct StepRaw {
         int a;
         float l_worker, reward, discount, value, value_next;
     };
-    auto load_scalars = [&](const Mine& m) {
+    // the per-step scalars of this thread's row in the tile at `pc` (`has`: the block has such a tile)
+    auto load_scalars = [&](const Place& pc, bool has) {
         StepRaw x;
         x.a = 0; x.l_worker = 0.0f; x.reward = 0.0f; x.discount = 0.0f; x.value = 0.0f; x.value_next = 0.0f;
-        if (m.active) {
-            const long long r = m.row;
+        if (has && gtid < pc.nrows) {
+            const long long r = pc.row0 + gtid;
             const int a = IMPACT_IN(actions)[r];
             x.a = min(max(a, 0), A - 1);
             x.l_worker = IMPACT_IN(worker_logp)[r];
             x.reward = IMPACT_IN(rewards)[r];
             x.discount = IMPACT_IN(discounts)[r];
             x.value = IMPACT_IN(values)[r];
-            x.value_next = m.last_step ? IMPACT_IN(bootstrap)[m.traj] : IMPACT_IN(values)[r + 1];
+            x.value_next = ends_trajectory(pc) ? IMPACT_IN(bootstrap)[pc.traj + q] : IMPACT_IN(values)[r + 1];
         }
         return x;
     };
@@ -1266,8 +1274,8 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     // The group's sums, once final: a butterfly per warp into `red`, then one arrival per warp tells the
     // producer warp that the row can be published (fixed order throughout).
     auto hand_over_sums = [&]() {
-        dev::hand_over_group_sums(t_surr, t_val, t_ent, t_ratio, t_kl, want_kl, n_clip, n_trunc, red[grp][gwarp],
-                                  &sums_bar[grp]);
+        dev::hand_over_group_sums(t_surr, t_val, t_ent, t_ratio, t_kl, want_kl, __reduce_add_sync(0xffffffffu, n_clip),
+                                  __reduce_add_sync(0xffffffffu, n_trunc), red[grp][gwarp], &sums_bar[grp]);
     };
 
     bool pending = false;  // lane 0 of each warp: a store of this warp may still be reading its stage
@@ -1275,18 +1283,18 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
 
     grid_dependency_wait();
     if (kIndirect) in = fetch_loss_inputs(p.indirect);
-    Mine me = mine_in(grp);
-    StepRaw cur = load_scalars(me);
+    Place pc = place_of(grp < n_tiles ? grp : 0);
+    StepRaw cur = load_scalars(pc, grp < n_tiles);
     __syncthreads();  // the producer warp has set up the barriers
     int s = grp % S;
     uint32_t ph = (uint32_t)(grp / S) & 1u;
 
     for (int n = grp; n < n_tiles; n += C) {
         // the next tile's scalars travel while this tile is worked on
-        const Mine me_next = mine_in(n + C);
-        const StepRaw nxt = load_scalars(me_next);
-        const bool active = me.active;
-        const long long row = me.row;
+        const Place pc_next = place_after(pc, n + C);
+        const StepRaw nxt = load_scalars(pc_next, n + C < n_tiles);
+        const bool active = gtid < pc.nrows;
+        const long long row = pc.row0 + gtid;
         // this warp's previous rows have left shared memory: hand the stage back.  (Only where stages are used
         // more than once: the wait for the store's reads sits between two tiles of the warp, and a block with no
         // more tiles than stages never needs a stage back.)
@@ -1301,27 +1309,27 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         // many trajectories they were published a round ago, and reading them now keeps that trip to L2 off the
         // path between this tile's scan and its gradients
         // (only where tiles are numbered tile-major; the values are first looked at after the scan)
-        const bool peeked = kLong && g.tile_major && gwarp == 0 && me.pc.r > lane;
+        const bool peeked = kLong && g.tile_major && gwarp == 0 && pc.r > lane;
         unsigned long long early_a = 0, early_b = 0;
         if (peeked)
             dev::load_aggregate(p.tile_aggregates + 2 * ((long long)blockIdx.x + (long long)n * gridDim.x), agg_stride,
-                                me.pc.r - lane, early_a, early_b);
+                                pc.r - lane, early_a, early_b);
         if (!dev::mbarrier_wait(&full_bar[s], ph, &abort_s)) atomicExch(p.counter + 1, 1u);
 
         // rows keep their place inside their 16-byte granule: the tile's first row starts (row0 * pitch) mod 16
         // bytes into the slab
         unsigned char* const stage = smem_raw + s * kStageBytes;
-        const uint32_t m_in = (uint32_t)(me.pc.row0 * kInRow) & 15u;
+        const uint32_t m_in = (uint32_t)(pc.row0 * kInRow) & 15u;
         unsigned char* const s0 = stage + m_in;     // learner logits
         unsigned char* const s1 = s0 + kInPitch;    // target logits
-        unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : stage + 2 * kInPitch + ((uint32_t)(me.pc.row0 * kOutRow) & 15u);
+        unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : stage + 2 * kInPitch + ((uint32_t)(pc.row0 * kOutRow) & 15u);
         bool stored = false;  // lane 0: a bulk store of this warp reads the stage
         // (first traversal of a batch) the target rows go to the circular buffer as well, each warp's 32 rows
         // straight from the stage, which nothing writes to
         if (IMPACT_IN(target_copy)) {
-            const int left = me.pc.nrows - (gtid - lane);
+            const int left = pc.nrows - (gtid - lane);
             const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
-            unsigned char* const dst = static_cast<unsigned char*>(IMPACT_IN(target_copy)) + (me.row - lane) * (long long)kInRow;
+            unsigned char* const dst = static_cast<unsigned char*>(IMPACT_IN(target_copy)) + (row - lane) * (long long)kInRow;
             stored = dev::warp_send_bytes(dst, s1 + (gtid - lane) * kInRow, (uint32_t)wrows * kInRow, false);
         }
         const int a = cur.a;
@@ -1331,7 +1339,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         st.discount = cur.discount;
         st.value = cur.value;
         st.value_next = cur.value_next;
-        st.last_step = me.last_step;
+        st.last_step = ends_trajectory(pc);
 
         // ---- row passes (every thread; rows beyond the tile hold stale bytes and are masked)
         float2 e[kStream ? 1 : NP];
@@ -1422,9 +1430,9 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             const long long gtile = (long long)blockIdx.x + (long long)n * gridDim.x;
             if (gtid == 0) dev::publish_tile_aggregate(p.tile_aggregates + 2 * gtile, ma, mb, dev::launch_tag(p.counter));
             float carry = 0.0f;
-            if (me.pc.r > 0) {  // uniform over the group
+            if (pc.r > 0) {  // uniform over the group
                 if (gwarp == 0) {
-                    const float c = dev::compose_later_aggregates(p.tile_aggregates + 2 * gtile, agg_stride, me.pc.r,
+                    const float c = dev::compose_later_aggregates(p.tile_aggregates + 2 * gtile, agg_stride, pc.r,
                                                                   dev::launch_tag(p.counter), &abort_s, peeked,
                                                                   early_a, early_b);
                     if (lane == 0) carry_s[grp] = c;
@@ -1447,8 +1455,8 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             t_ratio += ratio;
             if (!kPlain) t_kl += kl;
         }
-        n_clip += __popc(__ballot_sync(0xffffffffu, active && clipped));
-        n_trunc += __popc(__ballot_sync(0xffffffffu, active && truncated));
+        n_clip += (active && clipped) ? 1 : 0;    // (per thread; added up over the warp when the sums are handed over)
+        n_trunc += (active && truncated) ? 1 : 0;
         // the group's sums are final after its last tile's scan: handed over here, they are published while
         // that tile's gradient pass runs
         if (n + C >= n_tiles) hand_over_sums();
@@ -1510,7 +1518,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         // ---- each warp sends its own 32 rows: no barrier across the group
         {
             const long long wrow0 = row - lane;  // first row of this warp
-            const int left = me.pc.nrows - (gtid - lane);
+            const int left = pc.nrows - (gtid - lane);
             const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
             unsigned char* const gd = static_cast<unsigned char*>(p.dlogits) + wrow0 * (long long)kOutRow;
             if (dev::warp_send_bytes(gd, so + (gtid - lane) * kOutRow, (uint32_t)wrows * kOutRow, true)) stored = true;
@@ -1524,7 +1532,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             }
         }
         cur = nxt;
-        me = me_next;
+        pc = pc_next;
         s += C;
         while (s >= S) { s -= S; ph ^= 1u; }
     }
