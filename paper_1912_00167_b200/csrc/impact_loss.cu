@@ -2447,13 +2447,13 @@ WsPlan ws_plan(long long tiles, long long grid, size_t tile_bytes, int in_flight
     const long long budget = option(IMPACT_OPT_PREFETCH_BYTES);
     long long pf = budget / (grid * (long long)tile_bytes);
     // Asking L2 for tiles ahead of time goes through the copy engine like the tiles themselves, so it pays only
-    // where requests are large (measured: with 18 KB tiles a short launch gains half a microsecond from its
+    // where requests are large (measured: with 12-21 KB tiles a short launch gains half a microsecond from its
     // companion and a third from asking itself; with 3-9 KB tiles either costs 5-15 %).  The companion pays where a
     // launch is short: a block has a handful of tiles, all within the budget.  A long launch is bound by HBM either
     // way, and asking for many tiles far ahead of their use only competes with the tiles that are needed now.
     // Without a companion the loss kernel's first warp asks for the tiles it is about to request anyway (more than
     // that sits in the copy engine's queue ahead of the requests themselves).
-    const bool large_tiles = tile_bytes >= 16 * 1024;
+    const bool large_tiles = tile_bytes >= 10 * 1024;
     pl.companion = allow_companion && large_tiles && option(IMPACT_OPT_EARLY_PREFETCH) != 0 && pf >= per_block &&
                    per_block <= 8 && tiles * (long long)tile_bytes >= (4ll << 20);
     if (!large_tiles) pf = 0;

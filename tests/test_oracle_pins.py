@@ -496,3 +496,45 @@ def test_bf16_rounding_helper_is_round_to_nearest_even():
     np.testing.assert_array_equal(r, expect)
     big = np.random.default_rng(0).standard_normal(10000).astype(np.float32)
     np.testing.assert_array_equal(ii.round_to_bf16(big), torch.tensor(big).to(torch.bfloat16).float().numpy())
+
+
+def test_the_two_test_hooks_of_the_oracle_are_what_the_tests_take_them_for(oracle):
+    """`adv_cond` and `flip` are not part of the loss; the GPU parity tests take their tolerance and their "other
+    valid branch" from them, so both are pinned here against evaluations that do not go through the oracle's
+    recursion: adv_cond against the defining double sum over |terms|, flip against the difference it must make
+    (the policy term of exactly the marked steps, present in one run and absent in the other)."""
+    cfg, batch = ii.make_config(0)
+    h = dataclasses.replace(cfg.hyper, lam=0.97, rho_bar=1.3, c_bar=1.1, clip_eps=0.25, kl_coef=0.0)
+    ref = oracle.loss_categorical(batch, h)
+    B, T = batch["rewards"].shape
+    lp_t = log_softmax(batch["target_logits"].astype(np.float64), axis=-1)
+    l_t = np.take_along_axis(lp_t, batch["actions"][..., None], -1)[..., 0]
+    w = np.exp(l_t - batch["worker_logp"].astype(np.float64))
+    rho, c = np.minimum(w, h.rho_bar), np.minimum(w, h.c_bar)
+    r, g, v = (batch[k].astype(np.float64) for k in ("rewards", "discounts", "values"))
+    v_next = np.concatenate([v[:, 1:], batch["bootstrap_values"].astype(np.float64)[:, None]], 1)
+    term = rho * (np.abs(r) + np.abs(g * v_next) + np.abs(v))
+    want = np.zeros((B, T))
+    for b in range(B):
+        for t in range(T):
+            prod = 1.0
+            for i in range(t, T):  # sum_i |prod_{j<i} lambda gamma_j c_j| * |terms of delta_i|
+                want[b, t] += prod * term[b, i]
+                prod *= abs(h.lam * g[b, i] * c[b, i])
+    np.testing.assert_allclose(ref["adv_cond"], want, rtol=1e-12, atol=0)
+    assert (ref["adv_cond"] >= np.abs(ref["advantage"]) * (1 - 1e-12)).all()
+
+    flip = np.zeros((B, T), np.int8)
+    flip[1, 3] = flip[2, 7] = 1
+    other = oracle.loss_categorical(batch, h, flip=flip)
+    changed = np.abs(other["dlogits"] - ref["dlogits"]).max(-1) > 0
+    assert (changed == (flip == 1)).all()
+    for key in ("advantage", "vtarget", "dvalues", "ratio"):
+        np.testing.assert_array_equal(other[key], ref[key])
+    # the difference is the policy term of the marked steps: -A R (onehot - pi) / M, present on one side only
+    pi = np.exp(log_softmax(batch["learner_logits"].astype(np.float64), axis=-1))
+    onehot = np.eye(pi.shape[-1])[batch["actions"]]
+    term_pg = -(ref["advantage"] * ref["ratio"])[..., None] * (onehot - pi) / (B * T)
+    for (b, t) in ((1, 3), (2, 7)):
+        diff = other["dlogits"][b, t] - ref["dlogits"][b, t]
+        assert np.allclose(diff, term_pg[b, t], rtol=1e-10, atol=1e-18) or np.allclose(diff, -term_pg[b, t], rtol=1e-10, atol=1e-18)
