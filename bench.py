@@ -453,6 +453,81 @@ def run_sweep(args):
               f"{r['us_per_launch']:9.2f} us {r['timesteps_per_s'] / 1e9:7.3f} G/s{gb}")
 
 
+def run_case(spec: str):
+    """A handful of plain launches of one kernel on seeded data, for profiler captures (`ncu ... python bench.py --case
+    ...`): `cat:B:T:A[:bf16]` categorical loss, `gauss:B:T:D` Gaussian loss, `ring` the ring's copy / gather / device
+    bookkeeping kernels at the config-2 slot size.  Prints nothing but a final status line."""
+    import torch
+    import paper_1912_00167_b200 as ip
+    torch.cuda.set_device(0)
+    parts = spec.split(":")
+    kind = parts[0]
+    if kind == "cat":
+        B, T, A = (int(x) for x in parts[1:4])
+        dtype = torch.bfloat16 if parts[4:] == ["bf16"] else torch.float32
+        ws = ip.new_workspace(B, T)
+        coef = ip.Coefficients(clip_eps=0.4)
+        calls = []
+        for i in range(6):
+            d = synth_categorical_device(B, T, A, 900 + i, 0.005, 0.99, dtype)
+            out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda", dtype=dtype),
+                       dvalues=torch.empty(B, T, device="cuda"))
+            calls.append(ip.prepare_loss_fwd_bwd(d["learner_logits"], d["target_logits"], d["worker_logp"], d["actions"],
+                                                 d["rewards"], d["discounts"], d["values"], d["bootstrap_values"], coef,
+                                                 workspace=ws, **out))
+        torch.cuda.synchronize()
+        for c in calls:
+            c()
+        torch.cuda.synchronize()
+        print("case", spec, "status", ip.impact_loss_workspace_status(ws))
+    elif kind == "gauss":
+        B, T, D = (int(x) for x in parts[1:4])
+        ws = ip.new_workspace(B, T)
+        calls = []
+        for i in range(6):
+            hb = ii.gaussian_batch(B, T, D, 300 + i, p_done=0.001)
+            d = {k: torch.from_numpy(v).cuda() for k, v in hb.items()}
+            out = dict(loss_terms=torch.zeros(8, device="cuda"), dmean=torch.empty(B, T, D, device="cuda"),
+                       dlogstd=torch.empty(B, T, D, device="cuda"), dvalues=torch.empty(B, T, device="cuda"))
+            calls.append(ip.prepare_loss_fwd_bwd_gaussian(
+                d["learner_mean"], d["learner_logstd"], d["target_mean"], d["target_logstd"], d["worker_logp"],
+                d["actions"], d["rewards"], d["discounts"], d["values"], d["bootstrap_values"],
+                ip.Coefficients(ent_coef=0.0), workspace=ws, **out))
+        torch.cuda.synchronize()
+        for c in calls:
+            c()
+        torch.cuda.synchronize()
+        print("case", spec, "status", ip.impact_loss_workspace_status(ws))
+    elif kind == "ring":
+        cfg, b = ii.make_config(WORKLOAD_IDX)
+        t = {k: torch.from_numpy(v).cuda() for k, v in b.items()}
+        src = [t[n] for n in FIELD_NAMES]
+        ring = ip.ImpactBuffer(8, 4, [x.numel() * x.element_size() for x in src], seed=1)
+        for _ in range(6):
+            ring.push(src)
+        dst = [torch.empty_like(x) for x in src]
+        for _ in range(4):
+            ring.sample(dst)
+        ring.append(0, 4, t["target_logits"])
+        idx = torch.randint(0, cfg.B, (cfg.B,), device="cuda", dtype=torch.int32)
+        rows = torch.empty_like(t["target_logits"])
+        for _ in range(3):
+            ip.impact_gather_rows(t["target_logits"], idx, rows)
+        table = torch.tensor([[x.data_ptr() for x in src[:4]] + [0, src[4].data_ptr()]], dtype=torch.int64, device="cuda")
+        rec = ip.new_loss_inputs_record()
+        step = ring.prepare_device_step({n: f for f, n in enumerate(FIELD_NAMES)}, t["learner_logits"], t["values"],
+                                        t["bootstrap_values"], push_sources=table, record=rec)
+        ring.device_begin()
+        for _ in range(6):
+            step()
+        torch.cuda.synchronize()
+        print("case ring, last events", ring.device_events()[-2:])
+        ring.device_end()
+        ring.close()
+    else:
+        raise SystemExit(f"unknown case {spec!r}")
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -462,7 +537,12 @@ def main():
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--sweep", action="store_true", help="run the throughput sweep instead of the benchmark line")
     ap.add_argument("--sweep-out", default="sweep.json")
+    ap.add_argument("--case", default=None, help="run a few plain launches of one kernel (for profiler captures); "
+                                                 "cat:B:T:A[:bf16] | gauss:B:T:D | ring")
     args = ap.parse_args()
+    if args.case:
+        run_case(args.case)
+        return
     if args.sweep:
         run_sweep(args)
         return
@@ -526,11 +606,11 @@ def main():
     counters = {"loss": 0, "copy": 0, "pushed": 0}
     slot_batch = [0] * N  # which synthetic worker batch sits in each slot
 
-    def push_one():
+    def push_one(sid_=None):
         idx = counters["pushed"] % len(worker_batches)
         src = list(worker_batches[idx])
         src[4] = None  # the target network's output is appended at the first traversal
-        slot = ring.push(src, stream_id)
+        slot = ring.push(src, stream_id if sid_ is None else sid_)
         if slot is not None:
             slot_batch[slot] = idx
             counters["pushed"] += 1
@@ -556,18 +636,19 @@ def main():
         for i_ in range(len(worker_batches)):
             first_call(s_, i_)
 
-    def step():
-        got = ring.sample(None, stream_id)
+    def step(sid_=None):
+        sid_ = stream_id if sid_ is None else sid_
+        got = ring.sample(None, sid_)
         if got is None:
             raise RuntimeError("ring ran empty")
         slot, k = got
         if k == 0:
-            first_call(slot, slot_batch[slot]).on_stream(stream_id)
+            first_call(slot, slot_batch[slot]).on_stream(sid_)
         else:
-            calls[slot].on_stream(stream_id)
+            calls[slot].on_stream(sid_)
         counters["loss"] += 1
         if k == K - 1:
-            push_one()
+            push_one(sid_)
 
     while push_one() is not None:
         pass
@@ -606,20 +687,48 @@ def main():
             if flag != 0:
                 raise SystemExit(f"bench.py: a loss kernel gave up a bounded wait ({where}); workspace error word {flag}")
 
+    # The ring's bookkeeping is host arithmetic that depends on nothing the GPU computes, so the host may run ahead of
+    # the device: the K iterations of a block are enqueued into a CUDA graph first (bookkeeping done, kernels
+    # recorded; outside the timed region) and the timed region replays that graph once -- K learner iterations, each
+    # its sample, its loss launch (with the target logits stored into the slot at a first traversal) and, when a
+    # batch is discarded, the push of a new one.  Every block captures K NEW iterations: the ring moves on.
+    cap_stream = torch.cuda.Stream()
+
+    def capture_block():
+        g_ = torch.cuda.CUDAGraph()
+        with torch.cuda.stream(cap_stream):
+            with torch.cuda.graph(g_, stream=cap_stream):
+                for _ in range(args.steps):
+                    step(cap_stream.cuda_stream)
+        return g_
+
     def run_steps():
         for _ in range(args.steps):
             step()
     block_ms, wall_s = [], []
     while len(block_ms) < 3 or (sum(block_ms) < 200.0 and len(block_ms) < 200):
+        graph_block = capture_block()
+        graph_block.replay()  # untimed: the first launch of a new graph also uploads it to the device
+        torch.cuda.synchronize()
         t_wall0 = time.perf_counter()
-        block_ms.append(time_on_stream(run_steps))
+        block_ms.append(time_on_stream(graph_block.replay))
         wall_s.append(time.perf_counter() - t_wall0)
+        del graph_block
+    # the same iterations issued one by one from this Python loop (host-bound: what the interpreter and the driver
+    # need per launch, not what the device needs)
+    for c in counters:
+        counters[c] = counters[c] if c == "pushed" else 0
+    host_loop_ms = statistics.median(time_on_stream(run_steps) for _ in range(3)) / args.steps
+    n_blocks_counted = 3
     check_workspaces("learner iterations")
     ms_total = statistics.median(block_ms)
     t_wall = statistics.median(wall_s)
     n_blocks = len(block_ms)
-    launches = (counters["loss"] + counters["copy"]) // n_blocks
-    loss_launches = counters["loss"] // n_blocks
+    # kernels of this library per timed block: a loss call on this batch is two launches while the early prefetch is
+    # on (its one-warp-per-block companion, then the loss kernel), a push is one copy kernel
+    per_loss_call = 2 if ip.impact_get_option(ip.binding.OPT_EARLY_PREFETCH) else 1
+    loss_launches = counters["loss"] // n_blocks_counted
+    launches = per_loss_call * loss_launches + counters["copy"] // n_blocks_counted
 
     # ---- the same learner iteration with the ring's bookkeeping on the device, captured into a CUDA graph ------
     # (push-if-a-slot-is-free, draw, loss with its inputs named by the draw's record; the host only replays)
@@ -852,7 +961,10 @@ def main():
             "l2": f"inputs larger than L2: ring {ring.storage_bytes(N, field_bytes) >> 20} MiB + {N_SETS} "
                   f"learner-output sets + {N_SETS} gradient sets, rotated",
             "host_wall_ms_per_step": 1e3 * t_wall / args.steps,
-            "timing": f"median of {n_blocks} blocks of {args.steps} steps each (repeated until 0.2 s were timed)",
+            "timing": f"median of {n_blocks} blocks of {args.steps} steps each (repeated until 0.2 s were timed); a "
+                      f"block's iterations are enqueued into a CUDA graph ahead of time (the ring's bookkeeping is "
+                      f"host arithmetic independent of the device's results), replayed once untimed (upload) and once timed",
+            "host_loop_ms_per_step": host_loop_ms,
             "device_bookkeeping": {
                 "ms_per_step": dev_iter_ms, "host_wall_ms_per_step": dev_wall_ms,
                 "how": f"the same iteration with the ring's bookkeeping in device memory (impact_buffer_device_step: "

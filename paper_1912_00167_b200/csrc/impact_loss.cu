@@ -1081,9 +1081,11 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     // The tensors this launch reads: the call's own arguments (kernel parameters, read where they are used), or --
     // kIndirect: the call names a record in device memory that an earlier kernel of the stream fills (the circular
     // buffer's bookkeeping on the device) -- that record's, fetched by every thread once the stream dependency has
-    // resolved.
-    LossInputPointers in = {};
-#define IMPACT_IN(field) (kIndirect ? in.field : p.field)
+    // resolved
+    // (kept in shared memory, not in registers: every warp's lane 0 fetches the record and stores the same nine
+    // pointers there)
+    __shared__ LossInputPointers in_s;
+#define IMPACT_IN(field) (kIndirect ? in_s.field : p.field)
 
     if (tid >= C * NT) {
         // ---- producer warp ----------------------------------------------------------------------------------
@@ -1172,7 +1174,8 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         grid_dependency_wait();
 
         if (kIndirect) {  // (the addresses were not known before)
-            in = fetch_loss_inputs(p.indirect);
+            if (lane == 0) in_s = fetch_loss_inputs(p.indirect);
+            __syncwarp();
             first = request_for(place_of(sub < n_first ? sub : 0), sub);
         }
         if (sub < n_first) send_slab(first, sub, second);
@@ -1282,7 +1285,10 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     int pending_stage = 0;
 
     grid_dependency_wait();
-    if (kIndirect) in = fetch_loss_inputs(p.indirect);
+    if (kIndirect) {
+        if (lane == 0) in_s = fetch_loss_inputs(p.indirect);
+        __syncwarp();
+    }
     Place pc = place_of(grp < n_tiles ? grp : 0);
     StepRaw cur = load_scalars(pc, grp < n_tiles);
     __syncthreads();  // the producer warp has set up the barriers
