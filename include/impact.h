@@ -126,8 +126,9 @@ int32_t impact_last_cuda_error(void);
  *       previous kernel, so stream order is kept exactly; the loss kernel finds its first tiles in L2 instead of
  *       waiting for HBM.  0: no companion; the loss kernel asks for its first tiles itself when it starts.
  *   IMPACT_OPT_PREFETCH_BYTES  upper bound on the bytes one call asks L2 for ahead of time (default 48 MiB).
- *   IMPACT_OPT_WINDOW_BYTES    bytes of tiles a block keeps in flight from global to shared memory (default
- *       72 KiB; 16 KiB .. 160 KiB).
+ *   IMPACT_OPT_WINDOW_BYTES    bytes of tiles a block keeps in flight from global to shared memory: 0 (default)
+ *       lets each launch choose (48 KiB where a block has eight tiles or fewer, 72 KiB beyond), else
+ *       16 KiB .. 160 KiB.
  * impact_set_option returns IMPACT_ERR_INVALID_ARG for an unknown option or a value out of range;
  * impact_get_option returns -1 for an unknown option.
  */

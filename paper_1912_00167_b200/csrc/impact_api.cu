@@ -41,7 +41,7 @@ const DeviceInfo* current_device_info() {
 static std::atomic<int64_t> g_options[IMPACT_NUM_OPTIONS] = {
     {1},           // IMPACT_OPT_EARLY_PREFETCH
     {48ll << 20},  // IMPACT_OPT_PREFETCH_BYTES
-    {72ll << 10},  // IMPACT_OPT_WINDOW_BYTES
+    {0},           // IMPACT_OPT_WINDOW_BYTES: chosen per launch
 };
 int64_t option(int32_t which) { return g_options[which].load(std::memory_order_relaxed); }
 
@@ -49,7 +49,7 @@ int64_t option(int32_t which) { return g_options[which].load(std::memory_order_r
 
 extern "C" int32_t impact_set_option(int32_t option, int64_t value) {
     if (option < 0 || option >= IMPACT_NUM_OPTIONS || value < 0) return IMPACT_ERR_INVALID_ARG;
-    if (option == IMPACT_OPT_WINDOW_BYTES && (value < 16 * 1024 || value > 160 * 1024)) return IMPACT_ERR_INVALID_ARG;
+    if (option == IMPACT_OPT_WINDOW_BYTES && value != 0 && (value < 16 * 1024 || value > 160 * 1024)) return IMPACT_ERR_INVALID_ARG;
     impact::g_options[option].store(value, std::memory_order_relaxed);
     return IMPACT_OK;
 }

@@ -129,17 +129,17 @@ __device__ __forceinline__ bool mbarrier_test(uint64_t* bar, uint32_t parity) {
 // runs out ends every other wait of the block instead of each running out in turn.
 __device__ __forceinline__ bool mbarrier_wait(uint64_t* bar, uint32_t parity, int* abort_flag) {
     const uint32_t addr = smem_addr(bar);
-    constexpr uint32_t kSuspendHintNs = 1000;
-    for (uint32_t tries = 0; tries < (1u << 20); ++tries) {
+    // (no suspend hint and no sleep between tries: the wait sits between a tile's landing and the first
+    // instruction that uses it, and a hinted try followed by a 64 ns sleep measured 0.1 us per launch slower)
+    for (uint32_t tries = 0; tries < (1u << 24); ++tries) {
         uint32_t done;
         asm volatile(
             "{\n\t.reg .pred p;\n\t"
-            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2, %3;\n\t"
+            "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
             "selp.u32 %0, 1, 0, p;\n\t}"
-            : "=r"(done) : "r"(addr), "r"(parity), "r"(kSuspendHintNs) : "memory");
+            : "=r"(done) : "r"(addr), "r"(parity) : "memory");
         if (done) return true;
         if (*reinterpret_cast<volatile int*>(abort_flag)) return false;
-        __nanosleep(64);
     }
     *reinterpret_cast<volatile int*>(abort_flag) = 1;
     return false;
@@ -428,6 +428,54 @@ __device__ __forceinline__ float suffix_affine_scan_group(float a, float b, floa
     const float below = __shfl_down_sync(0xffffffffu, result, 1);
     next = (lane == 31) ? x : below;
     return result;
+}
+
+// The same scan with R rows per thread: a group of NTH threads covers NTH * R consecutive steps, warp w the steps
+// [32 R w, 32 R (w + 1)), lane l of it the steps 32 R w + 32 i + l for i < R (a lane's rows are 32 apart, which
+// keeps its accesses to rows of shared memory on the banks a single row per lane would use).  a[i], b[i] are the
+// rows' maps; res[i] receives A of row i, next[i] the value row i's map was applied to (0 after the last step).
+template <int NTH, int R>
+__device__ __forceinline__ void suffix_affine_scan_rows(float (&a)[R], float (&b)[R], float2* warp_agg, float (&res)[R],
+                                                        float (&next)[R], int bar_id) {
+    const int lane = threadIdx.x & 31, warp = (threadIdx.x & (NTH - 1)) >> 5;
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+#pragma unroll
+        for (int off = 1; off < 32; off <<= 1) {
+            const float a2 = __shfl_down_sync(0xffffffffu, a[i], off);
+            const float b2 = __shfl_down_sync(0xffffffffu, b[i], off);
+            if (lane + off < 32) {
+                b[i] = fmaf(a[i], b2, b[i]);
+                a[i] = a[i] * a2;
+            }
+        }
+    }
+    // inside the warp: the maps of the later sub-segments follow those of the earlier ones
+#pragma unroll
+    for (int i = R - 2; i >= 0; --i) {
+        const float ta = __shfl_sync(0xffffffffu, a[i + 1], 0), tb = __shfl_sync(0xffffffffu, b[i + 1], 0);
+        b[i] = fmaf(a[i], tb, b[i]);
+        a[i] = a[i] * ta;
+    }
+    float x = 0.0f;
+    if constexpr (NTH > 32) {
+        if (lane == 0) warp_agg[warp] = make_float2(a[0], b[0]);
+        asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NTH) : "memory");
+#pragma unroll
+        for (int w = NTH / 32 - 1; w > 0; --w) {
+            const float2 g = warp_agg[w];
+            if (w > warp) x = fmaf(g.x, x, g.y);
+        }
+    }
+#pragma unroll
+    for (int i = 0; i < R; ++i) res[i] = fmaf(a[i], x, b[i]);
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        const float below = __shfl_down_sync(0xffffffffu, res[i], 1);
+        float first_after = x;  // what follows this sub-segment's last row
+        if (i + 1 < R) first_after = __shfl_sync(0xffffffffu, res[i + 1], 0);
+        next[i] = (lane == 31) ? first_after : below;
+    }
 }
 
 // The scan as maps, for tiles that do not know yet what enters their last step: (ma, mb) is the

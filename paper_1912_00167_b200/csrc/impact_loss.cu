@@ -1049,11 +1049,15 @@ __device__ __forceinline__ LossInputPointers fetch_loss_inputs(const impact_loss
 // Without the in-order rule (lanes that found their own tile ready first went first) the first argument fails for
 // tiles of one round: a consumer could be handed a stage whose previous tile had not landed, read stale rows,
 // release the stage early, and the phases slipped until one of the bounded waits ran out.
-template <typename LT, typename GT, int A, int C, bool kPlain, bool kLong, int NT, bool kIndirect>
-__global__ void __launch_bounds__(C * NT + 32, 1)
+template <typename LT, typename GT, int A, int C, bool kPlain, bool kLong, int NT, bool kIndirect, int R>
+__global__ void __launch_bounds__(C * (NT / R) + 32, 1)
 impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int S, const int W, const int lanes,
                                   const int n_prefetch) {
     constexpr int NP = (A + 1) / 2;
+    constexpr int NTH = NT / R;  // threads of a consumer group: R steps of a tile each
+    constexpr int WR = 32 * R;   // rows of a tile that one warp works on
+    static_assert(R == 1 || (!kLong && A <= 32), "several steps per thread: trajectories within a tile, rows in registers");
+    static_assert(NTH % 32 == 0 && NTH >= 32, "whole warps");
     constexpr bool kStream = (A > 32);
     static_assert(!kStream || (A % 2 == 0 && (NP & (NP - 1)) == 0), "streamed rows: an even, power-of-two pair count");
     constexpr int kInRow = A * (int)sizeof(LT), kOutRow = A * (int)sizeof(GT);
@@ -1064,8 +1068,8 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kWsMaxStages], empty_bar[kWsMaxStages];
     __shared__ __align__(8) uint64_t sums_bar[C];  // a group's final sums are in `red`
-    __shared__ float2 warp_agg[C][NT / 32];
-    __shared__ __align__(16) float red[C][NT / 32][8];
+    __shared__ float2 warp_agg[C][2][NTH / 32];  // (two sets, used in turn: a tile's scan has one barrier)
+    __shared__ __align__(16) float red[C][NTH / 32][8];
     __shared__ int abort_s;
     __shared__ float carry_s[C];
 
@@ -1087,7 +1091,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     __shared__ LossInputPointers in_s;
 #define IMPACT_IN(field) (kIndirect ? in_s.field : p.field)
 
-    if (tid >= C * NT) {
+    if (tid >= C * NTH) {
         // ---- producer warp ----------------------------------------------------------------------------------
         const int n_first = n_tiles < W ? n_tiles : W;
         // First of all, while the kernel before this one on the stream is still finishing, the warp asks L2 for
@@ -1112,9 +1116,9 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         // then the barriers
         if (lane < S) {
             dev::mbarrier_init_nofence(&full_bar[lane], 1);
-            dev::mbarrier_init_nofence(&empty_bar[lane], NT / 32);  // one arrival per consumer warp
+            dev::mbarrier_init_nofence(&empty_bar[lane], NTH / 32);  // one arrival per consumer warp
         }
-        if (lane < C) dev::mbarrier_init_nofence(&sums_bar[lane], NT / 32);
+        if (lane < C) dev::mbarrier_init_nofence(&sums_bar[lane], NTH / 32);
         if (lane == 0) abort_s = 0;
         dev::fence_mbarrier_init();
         __syncwarp();
@@ -1216,19 +1220,33 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         }
         __syncwarp();
         // ---- then it publishes the block's sums, once every group's are final
-        if (!dev::publish_block_row<C, NT>(sums_bar, red, &abort_s, p.counter, p.tagged_rows, n_tiles > kWsFewTiles) && lane == 0)
+        if (!dev::publish_block_row<C, NTH>(sums_bar, red, &abort_s, p.counter, p.tagged_rows, n_tiles > kWsFewTiles) && lane == 0)
             atomicExch(p.counter + 1, 1u);  // a group never delivered its sums
         return;
     }
 
     // ---- consumer groups ------------------------------------------------------------------
-    const int grp = tid / NT, gtid = tid & (NT - 1), gwarp = gtid >> 5;
+    // A group of NTH threads works on a tile of NT steps, R steps per thread: warp w of the group on the tile's
+    // rows [WR w, WR (w + 1)), lane l of it on rows WR w + 32 i + l (i < R).  Everything a tile costs per thread
+    // and not per step -- the waits, the placement, the hand-over of the stage, the stores' bookkeeping -- is paid
+    // once for R steps, and a thread has R independent rows in flight.
+    const int grp = tid / NTH, gtid = tid & (NTH - 1), gwarp = gtid >> 5;
     const int bar_id = grp + 1;
+    const int wrow = gwarp * WR;  // the warp's first row in a tile
     const bool want_kl = !kPlain && (k.kl_coef != 0.0f);
 
-    // (short trajectories) the thread's place in a tile never changes: step ts of trajectory q of the tile
-    int q = 0, ts = gtid;
-    if (!kLong && g.G > 1) { q = gtid / (int)g.T; ts = gtid - q * (int)g.T; }
+    // (short trajectories) a thread's places in a tile never change: row tr[i] is step ts of trajectory q[i] of
+    // the tile
+    int tr[R], q[R];
+    bool ends_short[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) {
+        tr[i] = wrow + 32 * i + lane;
+        q[i] = 0;
+        int ts = tr[i];
+        if (!kLong && g.G > 1) { q[i] = tr[i] / (int)g.T; ts = tr[i] - q[i] * (int)g.T; }
+        ends_short[i] = ts == (int)g.T - 1;
+    }
     // Where the group's next tile sits: short trajectories advance by a fixed number of rows and trajectories
     // (C tiles of the block further on), long ones are placed tile by tile.
     const long long group_row_stride = (long long)C * gridDim.x * rows_full;
@@ -1246,28 +1264,28 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             return pn;
         }
     };
-    // does this thread's row end its trajectory (in the tile at `pc`)?
-    auto ends_trajectory = [&](const Place& pc) {
-        return kLong ? (pc.r == 0 && gtid == pc.nrows - 1) : (ts == (int)g.T - 1);
+    // does the thread's i-th row end its trajectory (in the tile at `pc`)?
+    auto ends_trajectory = [&](const Place& pc, int i) {
+        return kLong ? (pc.r == 0 && tr[i] == pc.nrows - 1) : ends_short[i];
     };
 
     struct StepRaw {
         int a;
         float l_worker, reward, discount, value, value_next;
     };
-    // the per-step scalars of this thread's row in the tile at `pc` (`has`: the block has such a tile)
-    auto load_scalars = [&](const Place& pc, bool has) {
+    // the per-step scalars of the thread's i-th row in the tile at `pc` (`has`: the block has such a tile)
+    auto load_scalars = [&](const Place& pc, bool has, int i) {
         StepRaw x;
         x.a = 0; x.l_worker = 0.0f; x.reward = 0.0f; x.discount = 0.0f; x.value = 0.0f; x.value_next = 0.0f;
-        if (has && gtid < pc.nrows) {
-            const long long r = pc.row0 + gtid;
+        if (has && tr[i] < pc.nrows) {
+            const long long r = pc.row0 + tr[i];
             const int a = IMPACT_IN(actions)[r];
             x.a = min(max(a, 0), A - 1);
             x.l_worker = IMPACT_IN(worker_logp)[r];
             x.reward = IMPACT_IN(rewards)[r];
             x.discount = IMPACT_IN(discounts)[r];
             x.value = IMPACT_IN(values)[r];
-            x.value_next = ends_trajectory(pc) ? IMPACT_IN(bootstrap)[pc.traj + q] : IMPACT_IN(values)[r + 1];
+            x.value_next = ends_trajectory(pc, i) ? IMPACT_IN(bootstrap)[pc.traj + q[i]] : IMPACT_IN(values)[r + 1];
         }
         return x;
     };
@@ -1290,17 +1308,20 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         __syncwarp();
     }
     Place pc = place_of(grp < n_tiles ? grp : 0);
-    StepRaw cur = load_scalars(pc, grp < n_tiles);
+    StepRaw cur[R];
+#pragma unroll
+    for (int i = 0; i < R; ++i) cur[i] = load_scalars(pc, grp < n_tiles, i);
     __syncthreads();  // the producer warp has set up the barriers
     int s = grp % S;
     uint32_t ph = (uint32_t)(grp / S) & 1u;
+    int turn = 0;  // which of the group's two sets of warp aggregates this tile uses
 
     for (int n = grp; n < n_tiles; n += C) {
         // the next tile's scalars travel while this tile is worked on
         const Place pc_next = place_after(pc, n + C);
-        const StepRaw nxt = load_scalars(pc_next, n + C < n_tiles);
-        const bool active = gtid < pc.nrows;
-        const long long row = pc.row0 + gtid;
+        StepRaw nxt[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) nxt[i] = load_scalars(pc_next, n + C < n_tiles, i);
         // this warp's previous rows have left shared memory: hand the stage back.  (Only where stages are used
         // more than once: the wait for the store's reads sits between two tiles of the warp, and a block with no
         // more tiles than stages never needs a stage back.)
@@ -1330,109 +1351,119 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         unsigned char* const s1 = s0 + kInPitch;    // target logits
         unsigned char* const so = (sizeof(LT) == sizeof(GT)) ? s0 : stage + 2 * kInPitch + ((uint32_t)(pc.row0 * kOutRow) & 15u);
         bool stored = false;  // lane 0: a bulk store of this warp reads the stage
-        // (first traversal of a batch) the target rows go to the circular buffer as well, each warp's 32 rows
+        // the warp's rows of this tile
+        const int wleft = pc.nrows - wrow;
+        const int wrows = wleft > WR ? WR : (wleft > 0 ? wleft : 0);
+        const long long wrow0 = pc.row0 + wrow;
+        // (first traversal of a batch) the target rows go to the circular buffer as well, each warp's rows
         // straight from the stage, which nothing writes to
         if (IMPACT_IN(target_copy)) {
-            const int left = pc.nrows - (gtid - lane);
-            const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
-            unsigned char* const dst = static_cast<unsigned char*>(IMPACT_IN(target_copy)) + (row - lane) * (long long)kInRow;
-            stored = dev::warp_send_bytes(dst, s1 + (gtid - lane) * kInRow, (uint32_t)wrows * kInRow, false);
+            unsigned char* const dst = static_cast<unsigned char*>(IMPACT_IN(target_copy)) + wrow0 * (long long)kInRow;
+            stored = dev::warp_send_bytes(dst, s1 + wrow * kInRow, (uint32_t)wrows * kInRow, false);
         }
-        const int a = cur.a;
-        dev::StepIn st;
-        st.l_worker = cur.l_worker;
-        st.reward = cur.reward;
-        st.discount = cur.discount;
-        st.value = cur.value;
-        st.value_next = cur.value_next;
-        st.last_step = ends_trajectory(pc);
 
         // ---- row passes (every thread; rows beyond the tile hold stale bytes and are masked)
-        float2 e[kStream ? 1 : NP];
-        float lse2_t, lse2_l, inv_s, ent, m2_l = 0.0f;
-        float kl = 0.0f;
-        if constexpr (!kStream) {
-            float m2_t, sum_t, unused, sum_l, sez;
-            lse2_t = RM::template lse2<false>(s1, gtid, e, m2_t, sum_t, unused);
-            lse2_l = RM::template lse2<true>(s0, gtid, e, m2_l, sum_l, sez);
-            inv_s = dev::rcp_fast(sum_l);
-            // H = -sum_j pi_j lp_j = (m + ln S) - sum_j e_j z_j / S
-            ent = fmaf(lse2_l, kLn2, -sez * inv_s);
-            if (want_kl) {
+        dev::StepIn st[R];
+        float2 e[R][kStream ? 1 : NP];
+        float lse2_t[R], lse2_l[R], inv_s[R], ent[R], m2_l[R], kl[R];
+        float fa[R], fb[R];
+        bool active[R], truncated[R];
 #pragma unroll
-                for (int j = 0; j < A; ++j) {
-                    const float lpt2 = fmaf(RowIO<LT, A>::at(s1, gtid, j), kLog2e, -lse2_t);
-                    const float lpl2 = fmaf(RowIO<LT, A>::at(s0, gtid, j), kLog2e, -lse2_l);
-                    kl = fmaf(dev::exp2_fast(lpt2), (lpt2 - lpl2) * kLn2, kl);
+        for (int i = 0; i < R; ++i) {
+            const int row = tr[i];
+            active[i] = row < pc.nrows;
+            st[i].l_worker = cur[i].l_worker;
+            st[i].reward = cur[i].reward;
+            st[i].discount = cur[i].discount;
+            st[i].value = cur[i].value;
+            st[i].value_next = cur[i].value_next;
+            st[i].last_step = ends_trajectory(pc, i);
+            m2_l[i] = 0.0f;
+            kl[i] = 0.0f;
+            if constexpr (!kStream) {
+                float m2_t, sum_t, unused, sum_l, sez;
+                lse2_t[i] = RM::template lse2<false>(s1, row, e[i], m2_t, sum_t, unused);
+                lse2_l[i] = RM::template lse2<true>(s0, row, e[i], m2_l[i], sum_l, sez);
+                inv_s[i] = dev::rcp_fast(sum_l);
+                // H = -sum_j pi_j lp_j = (m + ln S) - sum_j e_j z_j / S
+                ent[i] = fmaf(lse2_l[i], kLn2, -sez * inv_s[i]);
+                if (want_kl) {
+#pragma unroll
+                    for (int j = 0; j < A; ++j) {
+                        const float lpt2 = fmaf(RowIO<LT, A>::at(s1, row, j), kLog2e, -lse2_t[i]);
+                        const float lpl2 = fmaf(RowIO<LT, A>::at(s0, row, j), kLog2e, -lse2_l[i]);
+                        kl[i] = fmaf(dev::exp2_fast(lpt2), (lpt2 - lpl2) * kLn2, kl[i]);
+                    }
+                }
+            } else {
+                const int skew = row & (NP - 1);
+                const float2 log2e2 = make_float2(kLog2e, kLog2e);
+                auto row_max2 = [&](const unsigned char* slab) {
+                    float2 mx = RowIO<LT, A>::load_pair(slab, row, skew);
+#pragma unroll 8
+                    for (int j = 1; j < NP; ++j) {
+                        const float2 v = RowIO<LT, A>::load_pair(slab, row, (j + skew) & (NP - 1));
+                        mx.x = fmaxf(mx.x, v.x);
+                        mx.y = fmaxf(mx.y, v.y);
+                    }
+                    return fmaxf(mx.x, mx.y) * kLog2e;
+                };
+                {   // target row: its log-sum-exp
+                    const float m2 = row_max2(s1);
+                    const float2 neg_m2 = make_float2(-m2, -m2);
+                    float2 sum2 = make_float2(0.0f, 0.0f);
+#pragma unroll 8
+                    for (int j = 0; j < NP; ++j) {
+                        const float2 t2 = __ffma2_rn(RowIO<LT, A>::load_pair(s1, row, (j + skew) & (NP - 1)), log2e2, neg_m2);
+                        sum2 = __fadd2_rn(sum2, make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y)));
+                    }
+                    lse2_t[i] = m2 + dev::log2_fast(sum2.x + sum2.y);
+                }
+                {   // learner row: log-sum-exp and sum_j e_j z_j
+                    m2_l[i] = row_max2(s0);
+                    const float2 neg_m2 = make_float2(-m2_l[i], -m2_l[i]);
+                    float2 sum2 = make_float2(0.0f, 0.0f), sez2 = make_float2(0.0f, 0.0f);
+#pragma unroll 8
+                    for (int j = 0; j < NP; ++j) {
+                        const float2 z = RowIO<LT, A>::load_pair(s0, row, (j + skew) & (NP - 1));
+                        const float2 t2 = __ffma2_rn(z, log2e2, neg_m2);
+                        const float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
+                        sum2 = __fadd2_rn(sum2, ex);
+                        sez2 = __ffma2_rn(ex, z, sez2);
+                    }
+                    const float sum_l = sum2.x + sum2.y;
+                    lse2_l[i] = m2_l[i] + dev::log2_fast(sum_l);
+                    inv_s[i] = dev::rcp_fast(sum_l);
+                    ent[i] = fmaf(lse2_l[i], kLn2, -(sez2.x + sez2.y) * inv_s[i]);
+                }
+                if (want_kl) {
+#pragma unroll 8
+                    for (int j = 0; j < NP; ++j) {
+                        const int jj = (j + skew) & (NP - 1);
+                        const float2 zt2 = RowIO<LT, A>::load_pair(s1, row, jj), zl2 = RowIO<LT, A>::load_pair(s0, row, jj);
+                        const float ax = fmaf(zt2.x, kLog2e, -lse2_t[i]), ay = fmaf(zt2.y, kLog2e, -lse2_t[i]);
+                        kl[i] = fmaf(dev::exp2_fast(ax), (ax - fmaf(zl2.x, kLog2e, -lse2_l[i])) * kLn2, kl[i]);
+                        kl[i] = fmaf(dev::exp2_fast(ay), (ay - fmaf(zl2.y, kLog2e, -lse2_l[i])) * kLn2, kl[i]);
+                    }
                 }
             }
-        } else {
-            const int skew = gtid & (NP - 1);
-            const float2 log2e2 = make_float2(kLog2e, kLog2e);
-            auto row_max2 = [&](const unsigned char* slab) {
-                float2 mx = RowIO<LT, A>::load_pair(slab, gtid, skew);
-#pragma unroll 8
-                for (int j = 1; j < NP; ++j) {
-                    const float2 v = RowIO<LT, A>::load_pair(slab, gtid, (j + skew) & (NP - 1));
-                    mx.x = fmaxf(mx.x, v.x);
-                    mx.y = fmaxf(mx.y, v.y);
-                }
-                return fmaxf(mx.x, mx.y) * kLog2e;
-            };
-            {   // target row: its log-sum-exp
-                const float m2 = row_max2(s1);
-                const float2 neg_m2 = make_float2(-m2, -m2);
-                float2 sum2 = make_float2(0.0f, 0.0f);
-#pragma unroll 8
-                for (int j = 0; j < NP; ++j) {
-                    const float2 t2 = __ffma2_rn(RowIO<LT, A>::load_pair(s1, gtid, (j + skew) & (NP - 1)), log2e2, neg_m2);
-                    sum2 = __fadd2_rn(sum2, make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y)));
-                }
-                lse2_t = m2 + dev::log2_fast(sum2.x + sum2.y);
-            }
-            {   // learner row: log-sum-exp and sum_j e_j z_j
-                m2_l = row_max2(s0);
-                const float2 neg_m2 = make_float2(-m2_l, -m2_l);
-                float2 sum2 = make_float2(0.0f, 0.0f), sez2 = make_float2(0.0f, 0.0f);
-#pragma unroll 8
-                for (int j = 0; j < NP; ++j) {
-                    const float2 z = RowIO<LT, A>::load_pair(s0, gtid, (j + skew) & (NP - 1));
-                    const float2 t2 = __ffma2_rn(z, log2e2, neg_m2);
-                    const float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
-                    sum2 = __fadd2_rn(sum2, ex);
-                    sez2 = __ffma2_rn(ex, z, sez2);
-                }
-                const float sum_l = sum2.x + sum2.y;
-                lse2_l = m2_l + dev::log2_fast(sum_l);
-                inv_s = dev::rcp_fast(sum_l);
-                ent = fmaf(lse2_l, kLn2, -(sez2.x + sez2.y) * inv_s);
-            }
-            if (want_kl) {
-#pragma unroll 8
-                for (int j = 0; j < NP; ++j) {
-                    const int jj = (j + skew) & (NP - 1);
-                    const float2 zt2 = RowIO<LT, A>::load_pair(s1, gtid, jj), zl2 = RowIO<LT, A>::load_pair(s0, gtid, jj);
-                    const float ax = fmaf(zt2.x, kLog2e, -lse2_t), ay = fmaf(zt2.y, kLog2e, -lse2_t);
-                    kl = fmaf(dev::exp2_fast(ax), (ax - fmaf(zl2.x, kLog2e, -lse2_l)) * kLn2, kl);
-                    kl = fmaf(dev::exp2_fast(ay), (ay - fmaf(zl2.y, kLog2e, -lse2_l)) * kLn2, kl);
-                }
-            }
+            st[i].l_target = fmaf(RowIO<LT, A>::at(s1, row, cur[i].a), kLog2e, -lse2_t[i]) * kLn2;
+            st[i].l_theta = fmaf(RowIO<LT, A>::at(s0, row, cur[i].a), kLog2e, -lse2_l[i]) * kLn2;
+            if (kPlain) truncated[i] = dev::recursion_map_plain(st[i], k, fa[i], fb[i]);
+            else truncated[i] = dev::recursion_map(st[i], k, fa[i], fb[i]);
+            if (!active[i]) { fa[i] = 1.0f; fb[i] = 0.0f; }
         }
-        st.l_target = fmaf(RowIO<LT, A>::at(s1, gtid, a), kLog2e, -lse2_t) * kLn2;
-        st.l_theta = fmaf(RowIO<LT, A>::at(s0, gtid, a), kLog2e, -lse2_l) * kLn2;
-        float fa, fb;
-        bool truncated;
-        if (kPlain) truncated = dev::recursion_map_plain(st, k, fa, fb);
-        else truncated = dev::recursion_map(st, k, fa, fb);
-        if (!active) { fa = 1.0f; fb = 0.0f; }
-        float adv;
-        if (!kLong) {
-            adv = dev::suffix_affine_scan_group<NT>(fa, fb, warp_agg[grp], st.adv_next, bar_id);
+        float adv[R];
+        if constexpr (!kLong) {
+            float adv_next[R];
+            dev::suffix_affine_scan_rows<NTH, R>(fa, fb, warp_agg[grp][turn], adv, adv_next, bar_id);
+#pragma unroll
+            for (int i = 0; i < R; ++i) st[i].adv_next = adv_next[i];
         } else {
             // maps instead of values: (ma, mb) takes the value that enters the tile's last step to A of this
             // step, (la, lb) to A of the step after this warp's last
             float ma, mb, la, lb;
-            dev::suffix_affine_maps_group<NT>(fa, fb, warp_agg[grp], ma, mb, la, lb, bar_id);
+            dev::suffix_affine_maps_group<NT>(fa[0], fb[0], warp_agg[grp][turn], ma, mb, la, lb, bar_id);
             const long long gtile = (long long)blockIdx.x + (long long)n * gridDim.x;
             if (gtid == 0) dev::publish_tile_aggregate(p.tile_aggregates + 2 * gtile, ma, mb, dev::launch_tag(p.counter));
             float carry = 0.0f;
@@ -1446,88 +1477,94 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
                 asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory");
                 carry = carry_s[grp];
             }
-            adv = fmaf(ma, carry, mb);
-            const float below = __shfl_down_sync(0xffffffffu, adv, 1);
-            st.adv_next = (lane == 31) ? fmaf(la, carry, lb) : below;
+            adv[0] = fmaf(ma, carry, mb);
+            const float below = __shfl_down_sync(0xffffffffu, adv[0], 1);
+            st[0].adv_next = (lane == 31) ? fmaf(la, carry, lb) : below;
         }
+        turn ^= 1;
 
-        float surr, ratio;
-        bool clipped;
-        const float wpg = kPlain ? dev::surrogate_plain(st, k, adv, surr, ratio, clipped) : dev::surrogate(st, k, adv, surr, ratio, clipped);
-        if (active) {
-            t_surr += surr;
-            t_val = fmaf(0.5f * adv, adv, t_val);
-            t_ent += ent;
-            t_ratio += ratio;
-            if (!kPlain) t_kl += kl;
+        float wpg[R];
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            float surr, ratio;
+            bool clipped;
+            wpg[i] = kPlain ? dev::surrogate_plain(st[i], k, adv[i], surr, ratio, clipped)
+                            : dev::surrogate(st[i], k, adv[i], surr, ratio, clipped);
+            if (active[i]) {
+                t_surr += surr;
+                t_val = fmaf(0.5f * adv[i], adv[i], t_val);
+                t_ent += ent[i];
+                t_ratio += ratio;
+                if (!kPlain) t_kl += kl[i];
+            }
+            n_clip += (active[i] && clipped) ? 1 : 0;  // (per thread; added up over the warp when the sums are handed over)
+            n_trunc += (active[i] && truncated[i]) ? 1 : 0;
         }
-        n_clip += (active && clipped) ? 1 : 0;    // (per thread; added up over the warp when the sums are handed over)
-        n_trunc += (active && truncated) ? 1 : 0;
         // the group's sums are final after its last tile's scan: handed over here, they are published while
         // that tile's gradient pass runs
         if (n + C >= n_tiles) hand_over_sums();
 
         // ---- gradients: row_j = e_j (ga z_j + gb) [- kl_coef pi_target_j / M], then the taken action's entry
-        {
-            const float w1 = wpg * k.inv_M, ce = k.ent_coef * k.inv_M, ck = kPlain ? 0.0f : k.kl_coef * k.inv_M;
-            const float h_off = fmaf(-lse2_l, kLn2, ent);
-            const float ga = ce * inv_s, gb = (fmaf(ce, h_off, w1) + ck) * inv_s;
+#pragma unroll
+        for (int i = 0; i < R; ++i) {
+            const int row = tr[i];
+            const float w1 = wpg[i] * k.inv_M, ce = k.ent_coef * k.inv_M, ck = kPlain ? 0.0f : k.kl_coef * k.inv_M;
+            const float h_off = fmaf(-lse2_l[i], kLn2, ent[i]);
+            const float ga = ce * inv_s[i], gb = (fmaf(ce, h_off, w1) + ck) * inv_s[i];
             const float2 ga2 = make_float2(ga, ga), gb2 = make_float2(gb, gb);
             if constexpr (!kStream) {
                 if (!want_kl) {
 #pragma unroll
                     for (int j = 0; j < NP; ++j) {
-                        const float2 z = RowIO<LT, A>::load_pair(s0, gtid, j);
-                        RowIO<GT, A>::store_pair(so, gtid, j, __fmul2_rn(e[j], __ffma2_rn(z, ga2, gb2)));
+                        const float2 z = RowIO<LT, A>::load_pair(s0, row, j);
+                        RowIO<GT, A>::store_pair(so, row, j, __fmul2_rn(e[i][j], __ffma2_rn(z, ga2, gb2)));
                     }
                 } else {
-                    const float2 neg_lse2 = make_float2(-lse2_t, -lse2_t), nck2 = make_float2(-ck, -ck);
+                    const float2 neg_lse2 = make_float2(-lse2_t[i], -lse2_t[i]), nck2 = make_float2(-ck, -ck);
                     const float2 log2e2 = make_float2(kLog2e, kLog2e);
 #pragma unroll
                     for (int j = 0; j < NP; ++j) {
-                        const float2 z = RowIO<LT, A>::load_pair(s0, gtid, j);
-                        const float2 tt = __ffma2_rn(RowIO<LT, A>::load_pair(s1, gtid, j), log2e2, neg_lse2);
+                        const float2 z = RowIO<LT, A>::load_pair(s0, row, j);
+                        const float2 tt = __ffma2_rn(RowIO<LT, A>::load_pair(s1, row, j), log2e2, neg_lse2);
                         const float2 pt = make_float2(dev::exp2_fast(tt.x), dev::exp2_fast(tt.y));
-                        RowIO<GT, A>::store_pair(so, gtid, j, __ffma2_rn(nck2, pt, __fmul2_rn(e[j], __ffma2_rn(z, ga2, gb2))));
+                        RowIO<GT, A>::store_pair(so, row, j, __ffma2_rn(nck2, pt, __fmul2_rn(e[i][j], __ffma2_rn(z, ga2, gb2))));
                     }
                 }
             } else {
-                const int skew = gtid & (NP - 1);
-                const float2 log2e2 = make_float2(kLog2e, kLog2e), neg_m2 = make_float2(-m2_l, -m2_l);
-                const float2 neg_lse2 = make_float2(-lse2_t, -lse2_t), nck2 = make_float2(-ck, -ck);
+                const int skew = row & (NP - 1);
+                const float2 log2e2 = make_float2(kLog2e, kLog2e), neg_m2 = make_float2(-m2_l[i], -m2_l[i]);
+                const float2 neg_lse2 = make_float2(-lse2_t[i], -lse2_t[i]), nck2 = make_float2(-ck, -ck);
 #pragma unroll 8
                 for (int j = 0; j < NP; ++j) {
                     const int jj = (j + skew) & (NP - 1);
-                    const float2 z = RowIO<LT, A>::load_pair(s0, gtid, jj);
+                    const float2 z = RowIO<LT, A>::load_pair(s0, row, jj);
                     const float2 t2 = __ffma2_rn(z, log2e2, neg_m2);
                     const float2 ex = make_float2(dev::exp2_fast(t2.x), dev::exp2_fast(t2.y));
                     float2 gr = __fmul2_rn(ex, __ffma2_rn(z, ga2, gb2));
                     if (want_kl) {
-                        const float2 tt = __ffma2_rn(RowIO<LT, A>::load_pair(s1, gtid, jj), log2e2, neg_lse2);
+                        const float2 tt = __ffma2_rn(RowIO<LT, A>::load_pair(s1, row, jj), log2e2, neg_lse2);
                         gr = __ffma2_rn(nck2, make_float2(dev::exp2_fast(tt.x), dev::exp2_fast(tt.y)), gr);
                     }
-                    RowIO<GT, A>::store_pair(so, gtid, jj, gr);
+                    RowIO<GT, A>::store_pair(so, row, jj, gr);
                 }
             }
-            const float pi_a = dev::exp2_fast(st.l_theta * kLog2e);
-            float g_a = fmaf(pi_a, fmaf(ce, st.l_theta + ent, w1), -w1);
-            if (want_kl) g_a = fmaf(ck, pi_a - dev::exp2_fast(st.l_target * kLog2e), g_a);
-            if (active) {
-                p.dvalues[row] = -k.vf_coef * k.inv_M * adv;  // V - Vhat = -A
+            const float pi_a = dev::exp2_fast(st[i].l_theta * kLog2e);
+            float g_a = fmaf(pi_a, fmaf(ce, st[i].l_theta + ent[i], w1), -w1);
+            if (want_kl) g_a = fmaf(ck, pi_a - dev::exp2_fast(st[i].l_target * kLog2e), g_a);
+            if (active[i]) {
+                const long long grow = pc.row0 + row;
+                p.dvalues[grow] = -k.vf_coef * k.inv_M * adv[i];  // V - Vhat = -A
                 if (!kPlain) {
-                    if (p.vtarget) p.vtarget[row] = st.value + adv;
-                    if (p.advantage) p.advantage[row] = adv;
+                    if (p.vtarget) p.vtarget[grow] = st[i].value + adv[i];
+                    if (p.advantage) p.advantage[grow] = adv[i];
                 }
             }
-            RowIO<GT, A>::put(so, gtid, a, g_a);
+            RowIO<GT, A>::put(so, row, cur[i].a, g_a);
         }
-        // ---- each warp sends its own 32 rows: no barrier across the group
+        // ---- each warp sends its own rows: no barrier across the group
         {
-            const long long wrow0 = row - lane;  // first row of this warp
-            const int left = pc.nrows - (gtid - lane);
-            const int wrows = left > 32 ? 32 : (left > 0 ? left : 0);
             unsigned char* const gd = static_cast<unsigned char*>(p.dlogits) + wrow0 * (long long)kOutRow;
-            if (dev::warp_send_bytes(gd, so + (gtid - lane) * kOutRow, (uint32_t)wrows * kOutRow, true)) stored = true;
+            if (dev::warp_send_bytes(gd, so + wrow * kOutRow, (uint32_t)wrows * kOutRow, true)) stored = true;
             if (lane == 0) {
                 if (stored) {  // the stage goes back once the stores have read it: before this warp's next tile
                     pending = n_tiles > S;
@@ -1537,7 +1574,8 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
                 }
             }
         }
-        cur = nxt;
+#pragma unroll
+        for (int i = 0; i < R; ++i) cur[i] = nxt[i];
         pc = pc_next;
         s += C;
         while (s >= S) { s -= S; ph ^= 1u; }
@@ -1549,9 +1587,9 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     // last rows appear) collects every block's row
     // as it appears and writes the loss terms
     if (blockIdx.x == 0 && grp == n_tiles % C) {
-        if (!dev::reduce_tagged_rows<NT>(p.tagged_rows, (int)gridDim.x, dev::launch_tag(p.counter), p.counter,
-                                         p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, k.steps_total,
-                                         gtid, bar_id, &abort_s))
+        if (!dev::reduce_tagged_rows<NTH>(p.tagged_rows, (int)gridDim.x, dev::launch_tag(p.counter), p.counter,
+                                          p.loss_terms, k.vf_coef, k.ent_coef, k.kl_coef, k.steps_total,
+                                          gtid, bar_id, &abort_s))
             if (gtid == 0) atomicExch(p.counter + 1, 1u);
     }
     if (lane == 0) dev::bulk_store_wait_read();  // shared memory must outlive the stores' reads
@@ -2431,7 +2469,10 @@ void ws_ring_shape(size_t stage_bytes, size_t tile_in_bytes, int groups, int max
     if (s > kWsMaxStages) s = kWsMaxStages;
     const int fit = (int)((size_t)(max_smem - 4096) / stage_bytes);  // 4 KB left for static shared memory
     if (s > fit) s = fit;
-    if (s > groups) {
+    if (tiles_per_block <= s) {
+        // no stage is used twice: every barrier sees one phase only, and any number of tiles may be in flight
+        if (w > s) w = s;
+    } else if (s > groups) {
         if (w > s - groups) w = s - groups;
     } else if (s == groups) {
         if (w > s) w = s;
@@ -2480,12 +2521,18 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     // registers, no spills); six there for small action sets, which are bound by arithmetic, not bytes, and fit 72.
     // Wide rows (A = 64): tiles of 64 steps, six groups of 64 threads.
     constexpr int NT = ws_tile_rows(A);
+    // One step of a tile per thread.  (Two -- groups of 64 threads, seven groups, 128 registers -- execute 18 %
+    // fewer instructions on 18 actions and 27 % fewer on 6, everything paid per thread and tile being paid half as
+    // often, but a launch takes 0.3 us longer on 131 072 steps and 7 % longer on a million, and small action sets
+    // lose 7-20 % with eight to twelve such groups: a tile's rows then wait on half as many warps, and what
+    // bounds a launch is how long a tile takes, not how many instructions the SM issues.)
+    constexpr int R = 1;
     constexpr int C = A > 32 ? 6 : (!kPlain ? kWsGroups : (A <= 9 ? kWsGroups + 2 : kWsGroups + 1));
     // (inputs named by a device record: compiled for trajectories that fit a tile only)
     if (p.indirect && kLong) return IMPACT_ERR_UNSUPPORTED;
-    auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong, NT, false>;
+    auto kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong, NT, false, R>;
     if constexpr (!kLong)
-        if (p.indirect) kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong, NT, true>;
+        if (p.indirect) kernel = impact_loss_categorical_ws_kernel<LT, GT, A, C, kPlain, kLong, NT, true, R>;
     const size_t stage = ws_stage_bytes<LT, GT, A, NT>();
     const long long tiles = kLong ? p.geo.nchunks * p.geo.ntiles : p.geo.nchunks;
     long long grid = tiles < di->sm_count ? tiles : di->sm_count;
@@ -2524,7 +2571,7 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
         const int32_t st = launch_companion(pf, grid, stream);
         if (st != IMPACT_OK) return st;
     }
-    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * NT + 32), smem, stream, q, S, W, lanes,
+    IMPACT_CUDA_TRY(launch_serialized(kernel, dim3((unsigned)grid), dim3(C * (NT / R) + 32), smem, stream, q, S, W, lanes,
                                       plan.companion ? 0 : plan.prefetch_tiles));
     return IMPACT_OK;
 }
