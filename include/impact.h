@@ -120,8 +120,9 @@ int32_t impact_last_cuda_error(void);
  * result.  (The paper prescribes no kernel design, so these have no counterpart there.)  A value set here is
  * used by every later loss call of the process; setting one while another thread is inside a loss call is safe
  * (that call uses the old or the new value).
- *   IMPACT_OPT_EARLY_PREFETCH  1 (default): a loss call on a batch of at least a few megabytes enqueues a
- *       one-warp-per-block companion kernel right before its loss kernel.  The companion runs beside whatever
+ *   IMPACT_OPT_EARLY_PREFETCH  1 (default): a loss call whose thread blocks have four to eight tiles each (of at
+ *       least 10 KB, rows of at most 32 actions: batches of roughly 75 000 to 150 000 steps of 18 actions) enqueues
+ *       a one-warp-per-block companion kernel right before its loss kernel.  The companion runs beside whatever
  *       kernel is still busy on the stream, asks L2 for the batch's first tiles, and then waits for the stream's
  *       previous kernel, so stream order is kept exactly; the loss kernel finds its first tiles in L2 instead of
  *       waiting for HBM.  0: no companion; the loss kernel asks for its first tiles itself when it starts.

@@ -254,7 +254,9 @@ _DTYPE_CODE = {torch.float32: DTYPE_F32, torch.bfloat16: DTYPE_BF16}
 
 
 class PreparedCall:
-    """A C call with its arguments marshalled once; `()` re-issues it on the given stream."""
+    """A C call with its arguments marshalled once; `()` re-issues it on the given stream.  `keep` holds whatever
+    the marshalled pointers point into (the C structs and every tensor of the call), so that the call can be
+    re-issued for as long as it exists."""
 
     def __init__(self, fn, args, what, keep):
         self._fn, self._args, self._what, self._keep = fn, list(args), what, keep
@@ -294,7 +296,10 @@ def prepare_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, re
         _dev(advantage, f32, bt, "advantage", True),
         _dev(workspace, torch.uint8, workspace.shape, "workspace"), workspace.numel(),
         _dev(target_logits_copy, ldt, (B, T, A), "target_logits_copy", True), None)
-    return PreparedCall(lib.impact_loss_fwd_bwd_call, [ctypes.byref(call), 0], "impact_loss_fwd_bwd_call", (call,))
+    return PreparedCall(lib.impact_loss_fwd_bwd_call, [ctypes.byref(call), 0], "impact_loss_fwd_bwd_call",
+                        (call, learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
+                         bootstrap_values, loss_terms, dlogits, dvalues, vtarget, advantage, workspace,
+                         target_logits_copy))
 
 
 def new_loss_inputs_record(device="cuda") -> torch.Tensor:
@@ -320,7 +325,8 @@ def prepare_loss_fwd_bwd_from_record(record: torch.Tensor, B: int, T: int, A: in
         _dev(dvalues, f32, bt, "dvalues"), _dev(vtarget, f32, bt, "vtarget", True),
         _dev(advantage, f32, bt, "advantage", True),
         _dev(workspace, torch.uint8, workspace.shape, "workspace"), workspace.numel(), None, record.data_ptr())
-    return PreparedCall(lib.impact_loss_fwd_bwd_call, [ctypes.byref(call), 0], "impact_loss_fwd_bwd_call", (call, record))
+    return PreparedCall(lib.impact_loss_fwd_bwd_call, [ctypes.byref(call), 0], "impact_loss_fwd_bwd_call",
+                        (call, record, loss_terms, dlogits, dvalues, vtarget, advantage, workspace))
 
 
 def impact_loss_fwd_bwd(learner_logits, target_logits, worker_logp, actions, rewards, discounts, values,
@@ -389,7 +395,10 @@ def prepare_loss_fwd_bwd_gaussian(learner_mean, learner_logstd, target_mean, tar
         _dev(vtarget, f32, bt, "vtarget", True), _dev(advantage, f32, bt, "advantage", True),
         _dev(workspace, torch.uint8, workspace.shape, "workspace"), workspace.numel(), 0,
     ]
-    return PreparedCall(lib.impact_loss_fwd_bwd_gaussian, args, "impact_loss_fwd_bwd_gaussian", (cs,))
+    return PreparedCall(lib.impact_loss_fwd_bwd_gaussian, args, "impact_loss_fwd_bwd_gaussian",
+                        (cs, learner_mean, learner_logstd, target_mean, target_logstd, worker_logp, actions, rewards,
+                         discounts, values, bootstrap_values, loss_terms, dmean, dlogstd, dvalues, vtarget, advantage,
+                         workspace))
 
 
 def impact_loss_fwd_bwd_gaussian(learner_mean, learner_logstd, target_mean, target_logstd, worker_logp, actions,

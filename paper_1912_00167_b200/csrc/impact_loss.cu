@@ -2501,8 +2501,10 @@ WsPlan ws_plan(long long tiles, long long grid, size_t tile_bytes, int in_flight
     // Without a companion the loss kernel's first warp asks for the tiles it is about to request anyway (more than
     // that sits in the copy engine's queue ahead of the requests themselves).
     const bool large_tiles = tile_bytes >= 10 * 1024;
+    // (measured on 18 actions: a gain from five tiles per block on -- 8.3 -> 7.6 us at seven --, nothing at three
+    // to four, a loss of a quarter of a microsecond at two)
     pl.companion = allow_companion && large_tiles && option(IMPACT_OPT_EARLY_PREFETCH) != 0 && pf >= per_block &&
-                   per_block <= 8 && tiles * (long long)tile_bytes >= (4ll << 20);
+                   per_block >= 4 && per_block <= 8;
     if (!large_tiles) pf = 0;
     if (!pl.companion && pf > in_flight) pf = in_flight;
     if (pf > per_block) pf = per_block;
@@ -2553,7 +2555,9 @@ int32_t launch_categorical_ws(const CatParams& p, const DeviceInfo* di, cudaStre
     // tile-major once every block has a trajectory of its own: the aggregates a tile needs are then a round old
     q.geo.tile_major = (kLong && p.geo.B >= grid) ? 1 : 0;
     const int rows_full = kLong ? NT : q.geo.G * (int)q.geo.T;
-    WsPlan plan_ = ws_plan(tiles, grid, (size_t)rows_full * (2 * A * sizeof(LT) + 20), W, true);
+    // (rows wider than 32 actions: the companion gains nothing with fp32 logits and doubles a launch with bf16 ones
+    // -- 27 against 14 us at 65 536 steps --, so such launches ask for their first tiles themselves)
+    WsPlan plan_ = ws_plan(tiles, grid, (size_t)rows_full * (2 * A * sizeof(LT) + 20), W, A <= 32);
     if (p.indirect) { plan_.companion = false; plan_.prefetch_tiles = 0; }  // (addresses unknown on the host)
     const WsPlan plan = plan_;
     if (plan.companion) {

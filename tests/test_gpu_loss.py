@@ -527,3 +527,36 @@ def test_batch_split_over_calls_adds_up_to_the_whole(oracle, B, T, A, parts):
                                dataclasses.replace(P.to_coef(h), global_steps=M - 1), workspace=ip.new_workspace(B, T),
                                loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
                                dvalues=torch.empty(B, T, device="cuda"))
+
+
+def test_prepared_calls_keep_their_tensors_alive():
+    """A prepared call holds raw device addresses; it must also hold the tensors they point into, or the call
+    outlives its memory as soon as the caller drops its own references."""
+    import paper_1912_00167_b200 as ip
+    B, T, A, D = 3, 7, 6, 3
+
+    def categorical():
+        t = {k: torch.from_numpy(v).cuda() for k, v in ii.categorical_batch(B, T, A, seed=1).items()}
+        out = dict(loss_terms=torch.zeros(8, device="cuda"), dlogits=torch.empty(B, T, A, device="cuda"),
+                   dvalues=torch.empty(B, T, device="cuda"))
+        ws = ip.new_workspace(B, T)
+        call = ip.prepare_loss_fwd_bwd(t["learner_logits"], t["target_logits"], t["worker_logp"], t["actions"],
+                                       t["rewards"], t["discounts"], t["values"], t["bootstrap_values"],
+                                       ip.Coefficients(), workspace=ws, **out)
+        return call, [t[k].data_ptr() for k in sorted(t)] + [v.data_ptr() for v in out.values()] + [ws.data_ptr()]
+
+    def gaussian():
+        t = {k: torch.from_numpy(v).cuda() for k, v in ii.gaussian_batch(B, T, D, seed=2).items()}
+        out = dict(loss_terms=torch.zeros(8, device="cuda"), dmean=torch.empty(B, T, D, device="cuda"),
+                   dlogstd=torch.empty(B, T, D, device="cuda"), dvalues=torch.empty(B, T, device="cuda"))
+        ws = ip.new_workspace(B, T)
+        call = ip.prepare_loss_fwd_bwd_gaussian(t["learner_mean"], t["learner_logstd"], t["target_mean"],
+                                                t["target_logstd"], t["worker_logp"], t["actions"], t["rewards"],
+                                                t["discounts"], t["values"], t["bootstrap_values"], ip.Coefficients(),
+                                                workspace=ws, **out)
+        return call, [t[k].data_ptr() for k in sorted(t)] + [v.data_ptr() for v in out.values()] + [ws.data_ptr()]
+
+    for make in (categorical, gaussian):
+        call, addresses = make()
+        held = {x.data_ptr() for x in call._keep if isinstance(x, torch.Tensor)}
+        assert set(addresses) <= held
