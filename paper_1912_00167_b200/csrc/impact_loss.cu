@@ -934,7 +934,6 @@ __global__ void __launch_bounds__(32) impact_prefetch_kernel(const __grid_consta
 }
 constexpr int ws_tile_rows(int A) { return A > 32 ? 64 : 128; }
 constexpr int kWsMaxStages = 24;
-constexpr int kWsFewTiles = 32;  // up to this many tiles per block the producer works for latency, beyond for throughput
 constexpr int kWsGroups = 4;  // consumer groups per block at least (16 consumer warps + the producer warp)
 
 // Row passes of one step, shared by the kernels with a compile-time action count.  `zr` / `tr`
@@ -1067,7 +1066,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     using RM = RowMath<LT, A>;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kWsMaxStages], empty_bar[kWsMaxStages];
-    __shared__ __align__(8) uint64_t sums_bar[C];  // a group's final sums are in `red`
+    __shared__ unsigned int tickets_s, tag_s;  // (see dev::draw_ticket_and_publish)
     __shared__ float2 warp_agg[C][2][NTH / 32];  // (two sets, used in turn: a tile's scan has one barrier)
     __shared__ __align__(16) float red[C][NTH / 32][8];
     __shared__ int abort_s;
@@ -1118,8 +1117,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             dev::mbarrier_init_nofence(&full_bar[lane], 1);
             dev::mbarrier_init_nofence(&empty_bar[lane], NTH / 32);  // one arrival per consumer warp
         }
-        if (lane < C) dev::mbarrier_init_nofence(&sums_bar[lane], NTH / 32);
-        if (lane == 0) abort_s = 0;
+        if (lane == 0) { abort_s = 0; tickets_s = 0u; }
         dev::fence_mbarrier_init();
         __syncwarp();
 
@@ -1184,6 +1182,7 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         }
         if (sub < n_first) send_slab(first, sub, second);
         __syncthreads();  // the barriers are set up: the consumer warps may use them
+        const unsigned int tag = dev::launch_tag(p.counter);  // (asked for now, needed after the last tile has left)
         // The rest.  Tile n goes to stage n % S once that stage's previous tile has left (the "empty" phase before
         // this one) and tile n - W has landed (at most W tiles in flight).  The owners look at their barriers side by
         // side (one thread taking tile after tile through blocking waits costs a third of a microsecond per tile, too
@@ -1219,9 +1218,9 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
             }
         }
         __syncwarp();
-        // ---- then it publishes the block's sums, once every group's are final
-        if (!dev::publish_block_row<C, NTH>(sums_bar, red, &abort_s, p.counter, p.tagged_rows, n_tiles > kWsFewTiles) && lane == 0)
-            atomicExch(p.counter + 1, 1u);  // a group never delivered its sums
+        // ---- then it leaves this launch's tag for whoever publishes the block's sums, and draws its own ticket
+        if (lane == 0) tag_s = tag;
+        dev::draw_ticket_and_publish<C, NTH / 32>(&tickets_s, &tag_s, red, p.tagged_rows);
         return;
     }
 
@@ -1292,11 +1291,12 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
 
     float t_surr = 0.0f, t_val = 0.0f, t_ent = 0.0f, t_ratio = 0.0f, t_kl = 0.0f;
     int n_clip = 0, n_trunc = 0;
-    // The group's sums, once final: a butterfly per warp into `red`, then one arrival per warp tells the
-    // producer warp that the row can be published (fixed order throughout).
+    // The group's sums, once final: a butterfly per warp into `red`, then the warp's ticket; the last ticket of
+    // the block publishes its row (fixed order throughout).
     auto hand_over_sums = [&]() {
-        dev::hand_over_group_sums(t_surr, t_val, t_ent, t_ratio, t_kl, want_kl, __reduce_add_sync(0xffffffffu, n_clip),
-                                  __reduce_add_sync(0xffffffffu, n_trunc), red[grp][gwarp], &sums_bar[grp]);
+        dev::hand_over_warp_sums<C, NTH / 32>(t_surr, t_val, t_ent, t_ratio, t_kl, want_kl,
+                                              __reduce_add_sync(0xffffffffu, n_clip), __reduce_add_sync(0xffffffffu, n_trunc),
+                                              red[grp][gwarp], &tickets_s, &tag_s, red, p.tagged_rows);
     };
 
     bool pending = false;  // lane 0 of each warp: a store of this warp may still be reading its stage
@@ -1963,7 +1963,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     constexpr float kHalfLog2Pi = 0.91893853320467274178f;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     __shared__ __align__(8) uint64_t full_bar[kWsMaxStages], empty_bar[kWsMaxStages];
-    __shared__ __align__(8) uint64_t sums_bar[C];
+    __shared__ unsigned int tickets_s, tag_s;
     __shared__ float2 warp_agg[C][NT / 32];
     __shared__ __align__(16) float red[C][NT / 32][8];
     __shared__ int abort_s;
@@ -2004,8 +2004,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
             dev::mbarrier_init_nofence(&full_bar[lane], 1);
             dev::mbarrier_init_nofence(&empty_bar[lane], NT / 32);
         }
-        if (lane < C) dev::mbarrier_init_nofence(&sums_bar[lane], NT / 32);
-        if (lane == 0) abort_s = 0;
+        if (lane == 0) { abort_s = 0; tickets_s = 0u; }
         dev::fence_mbarrier_init();
         __syncwarp();
 
@@ -2055,6 +2054,7 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
         for (int base = 4; base < n_first; base += 4)
             if (sends && base + sub < n_first) send_slab(request_for(place_of(base + sub), base + sub), base + sub, q_lane);
         __syncthreads();  // the barriers are set up: the consumer warps may use them
+        const unsigned int tag = dev::launch_tag(p.counter);  // (asked for now, needed after the last tile has left)
         for (int base = n_first; base < n_tiles; base += lanes) {
             const int n = base + sub;
             bool pending = sends && sub < lanes && n < n_tiles;
@@ -2084,9 +2084,9 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
             }
         }
         __syncwarp();
-        // the block's sums, once every group's are final
-        if (!dev::publish_block_row<C, NT>(sums_bar, red, &abort_s, p.counter, p.tagged_rows, n_tiles > kWsFewTiles) && lane == 0)
-            atomicExch(p.counter + 1, 1u);
+        // this launch's tag for whoever publishes the block's sums, and the warp's own ticket
+        if (lane == 0) tag_s = tag;
+        dev::draw_ticket_and_publish<C, NT / 32>(&tickets_s, &tag_s, red, p.tagged_rows);
         return;
     }
 
@@ -2132,8 +2132,8 @@ impact_loss_gaussian_ws_kernel(const __grid_constant__ GaussParams p, const int 
     float t_surr = 0.0f, t_val = 0.0f, t_ent = 0.0f, t_ratio = 0.0f, t_kl = 0.0f;
     int n_clip = 0, n_trunc = 0;
     auto hand_over_sums = [&]() {
-        dev::hand_over_group_sums(t_surr, t_val, t_ent, t_ratio, t_kl, want_kl, n_clip, n_trunc, red[grp][gwarp],
-                                  &sums_bar[grp]);
+        dev::hand_over_warp_sums<C, NT / 32>(t_surr, t_val, t_ent, t_ratio, t_kl, want_kl, n_clip, n_trunc, red[grp][gwarp],
+                                             &tickets_s, &tag_s, red, p.tagged_rows);
     };
     bool pending = false;
     int pending_stage = 0;
