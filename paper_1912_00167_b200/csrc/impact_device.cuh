@@ -899,6 +899,7 @@ __device__ __noinline__ bool reduce_tagged_rows(const unsigned long long* rows, 
     __shared__ float fred[NT / 32][8];
     constexpr int kStride = NT / 8, kU = 10;
     const int col = gtid & 7, rc = gtid >> 3;
+    const double inv_m = 1.0 / M;  // (a long division: done while the rows are still on their way)
     float acc = 0.0f;
     bool missing = false;
     for (int base = rc; base < nrows && !missing; base += kStride * kU) {
@@ -929,26 +930,18 @@ __device__ __noinline__ bool reduce_tagged_rows(const unsigned long long* rows, 
     acc += __shfl_xor_sync(0xffffffffu, acc, 16);
     if (lane < 8) fred[warp][lane] = acc;
     asm volatile("bar.sync %0, %1;" ::"r"(bar_id), "n"(NT) : "memory");
-    if (gtid == 0) {
-        const double inv_m = 1.0 / M;
-        double t[kNumSums];
+    // the last steps sit between the slowest block's row and the end of the launch: a lane per column
+    if (gtid < 8) {
+        float x = 0.0f;
 #pragma unroll
-        for (int j = 0; j < kNumSums; ++j) {
-            float x = 0.0f;
-#pragma unroll
-            for (int w = 0; w < NT / 32; ++w) x += fred[w][j];
-            t[j] = (double)x * inv_m;
+        for (int w = 0; w < NT / 32; ++w) x += fred[w][gtid];
+        const double t = (double)x * inv_m;  // columns: surrogate, value, entropy, kl, clipped, truncated, ratio
+        const double t1 = __shfl_sync(0xffu, t, 1), t2 = __shfl_sync(0xffu, t, 2), t3 = __shfl_sync(0xffu, t, 3);
+        if (gtid == 0) {
+            loss_terms[0] = (float)(-t + (double)vf_coef * t1 - (double)ent_coef * t2 + (double)kl_coef * t3);
+            counter_words[2] = tag;
         }
-        const double l_pi = -t[0], l_v = t[1], ent = t[2], kl = t[3];
-        loss_terms[0] = (float)(l_pi + (double)vf_coef * l_v - (double)ent_coef * ent + (double)kl_coef * kl);
-        loss_terms[1] = (float)l_pi;
-        loss_terms[2] = (float)l_v;
-        loss_terms[3] = (float)ent;
-        loss_terms[4] = (float)kl;
-        loss_terms[5] = (float)t[4];
-        loss_terms[6] = (float)t[5];
-        loss_terms[7] = (float)t[6];
-        counter_words[2] = tag;
+        if (gtid < kNumSums) loss_terms[gtid + 1] = (float)(gtid == 0 ? -t : t);
     }
     return *reinterpret_cast<volatile int*>(abort_flag) == 0;
 }
