@@ -205,8 +205,8 @@ def compare(gpu, ref, ref_flipped, near, M, grad_keys, kl_coef, sens, vf_coef, r
 
 
 def _log_report(report):
-    """With IMPACT_PARITY_REPORT=<file> every comparison appends one JSON line (test id + per-output figures): the
-    table of measured margins in the design doc is made from it."""
+    """With IMPACT_PARITY_REPORT=<file> every comparison appends one JSON line (test id + per-output figures:
+    elements, elements outside the stated bar, worst error in units of the bar, allowance used)."""
     import json, os
     path = os.environ.get("IMPACT_PARITY_REPORT")
     if path:
