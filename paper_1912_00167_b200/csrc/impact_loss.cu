@@ -1083,10 +1083,10 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     auto place_of = [&](int n) { return tile_place<kLong, NT>(g, n, rows_full, total_rows); };
     // The tensors this launch reads: the call's own arguments (kernel parameters, read where they are used), or --
     // kIndirect: the call names a record in device memory that an earlier kernel of the stream fills (the circular
-    // buffer's bookkeeping on the device) -- that record's, fetched by every thread once the stream dependency has
-    // resolved
-    // (kept in shared memory, not in registers: every warp's lane 0 fetches the record and stores the same nine
-    // pointers there)
+    // buffer's bookkeeping on the device) -- that record's, fetched once the stream dependency has resolved
+    // (kept in shared memory, not in registers; the producer warp alone fetches the record, before the block-wide
+    // barrier that releases the consumer warps: with every warp of the grid fetching it -- 3 000 warps asking one
+    // cache line at the same moment -- the first tile was requested 3.6 us late)
     __shared__ LossInputPointers in_s;
 #define IMPACT_IN(field) (kIndirect ? in_s.field : p.field)
 
@@ -1277,14 +1277,17 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
         StepRaw x;
         x.a = 0; x.l_worker = 0.0f; x.reward = 0.0f; x.discount = 0.0f; x.value = 0.0f; x.value_next = 0.0f;
         if (has && tr[i] < pc.nrows) {
+            // (loads that name the global space: a pointer taken from the device record is a generic one to the
+            // compiler, and a generic load has to be complete before the next store to shared memory -- that put the
+            // whole trip to L2 into every tile, 10.9 us a launch against 6.8)
             const long long r = pc.row0 + tr[i];
-            const int a = IMPACT_IN(actions)[r];
+            const int a = __ldg(IMPACT_IN(actions) + r);
             x.a = min(max(a, 0), A - 1);
-            x.l_worker = IMPACT_IN(worker_logp)[r];
-            x.reward = IMPACT_IN(rewards)[r];
-            x.discount = IMPACT_IN(discounts)[r];
-            x.value = IMPACT_IN(values)[r];
-            x.value_next = ends_trajectory(pc, i) ? IMPACT_IN(bootstrap)[pc.traj + q[i]] : IMPACT_IN(values)[r + 1];
+            x.l_worker = __ldg(IMPACT_IN(worker_logp) + r);
+            x.reward = __ldg(IMPACT_IN(rewards) + r);
+            x.discount = __ldg(IMPACT_IN(discounts) + r);
+            x.value = __ldg(IMPACT_IN(values) + r);
+            x.value_next = ends_trajectory(pc, i) ? __ldg(IMPACT_IN(bootstrap) + pc.traj + q[i]) : __ldg(IMPACT_IN(values) + r + 1);
         }
         return x;
     };
@@ -1303,15 +1306,17 @@ impact_loss_categorical_ws_kernel(const __grid_constant__ CatParams p, const int
     int pending_stage = 0;
 
     grid_dependency_wait();
-    if (kIndirect) {
-        if (lane == 0) in_s = fetch_loss_inputs(p.indirect);
-        __syncwarp();
-    }
     Place pc = place_of(grp < n_tiles ? grp : 0);
     StepRaw cur[R];
+    if (!kIndirect) {
 #pragma unroll
-    for (int i = 0; i < R; ++i) cur[i] = load_scalars(pc, grp < n_tiles, i);
-    __syncthreads();  // the producer warp has set up the barriers
+        for (int i = 0; i < R; ++i) cur[i] = load_scalars(pc, grp < n_tiles, i);
+    }
+    __syncthreads();  // the producer warp has set up the barriers (and fetched the device record)
+    if (kIndirect) {
+#pragma unroll
+        for (int i = 0; i < R; ++i) cur[i] = load_scalars(pc, grp < n_tiles, i);
+    }
     int s = grp % S;
     uint32_t ph = (uint32_t)(grp / S) & 1u;
     int turn = 0;  // which of the group's two sets of warp aggregates this tile uses
