@@ -158,9 +158,11 @@ __global__ void __launch_bounds__(32) ring_step_kernel(const RingDeviceView v, c
     // the slots' flags and counts are staged in shared memory by the whole warp (one trip to L2 instead of one per
     // slot); lane 0 then walks them exactly as the host code does and writes back what it changed
     __shared__ int32_t valid_s[kMaxDeviceSlots], count_s[kMaxDeviceSlots];
+    __shared__ uint64_t fresh_s[kMaxDeviceSlots];
     for (int32_t i = threadIdx.x; i < v.N; i += 32) {
         valid_s[i] = v.valid[i];
         count_s[i] = v.count[i];
+        fresh_s[i] = v.fresh[i];
     }
     RingDeviceHeader hd = *v.hd;
     // (the candidate's pointers too: lane f fetches the f-th, all at once)
@@ -191,6 +193,7 @@ __global__ void __launch_bounds__(32) ring_step_kernel(const RingDeviceView v, c
             }
             v.plan->n = n;
             v.fresh[slot] = reinterpret_cast<uint64_t>(cand[v.n_fields]);
+            fresh_s[slot] = reinterpret_cast<uint64_t>(cand[v.n_fields]);
             valid_s[slot] = 1;
             count_s[slot] = 0;
             v.valid[slot] = 1;
@@ -238,7 +241,7 @@ __global__ void __launch_bounds__(32) ring_step_kernel(const RingDeviceView v, c
             in.discounts = static_cast<const float*>(field(map.discounts));
             in.worker_logp = static_cast<const float*>(field(map.worker_logp));
             const void* in_slot = field(map.target_logits);
-            const void* fresh = reinterpret_cast<const void*>(v.fresh[pick]);
+            const void* fresh = reinterpret_cast<const void*>(fresh_s[pick]);
             if (k_before == 0 && fresh && in_slot) {  // first traversal: the target network's output is appended now
                 in.target_logits = fresh;
                 in.target_logits_copy = const_cast<void*>(in_slot);
@@ -262,6 +265,16 @@ __global__ void __launch_bounds__(32) ring_step_kernel(const RingDeviceView v, c
 // multi_copy_kernel with its segments read from device memory (an empty plan copies nothing).
 __global__ void __launch_bounds__(256) multi_copy_planned_kernel(const CopySegments* plan) {
     grid_dependency_wait();
+    // the plan is staged in shared memory by the block's first threads, eight bytes each: one trip to L2 instead of
+    // one for the count, one for the segment ends and one for the addresses
+    __shared__ CopySegments plan_s;
+    constexpr int kWords = (int)(sizeof(CopySegments) / 8);
+    static_assert(sizeof(CopySegments) % 8 == 0 && kWords <= 256, "staged by one pass of the block");
+    if ((int)threadIdx.x < kWords)
+        reinterpret_cast<unsigned long long*>(&plan_s)[threadIdx.x] =
+            reinterpret_cast<const unsigned long long*>(plan)[threadIdx.x];  // (through L1: the blocks of an SM share the lines)
+    __syncthreads();
+    plan = &plan_s;
     const int n = plan->n;
     if (n == 0) return;
     const unsigned long long total = plan->vec_end[n - 1];
